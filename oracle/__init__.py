@@ -1,0 +1,252 @@
+"""ctypes front-end of the float64 CPU oracle (``gbs_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY.  The oracle restates, by the definition and in double
+precision, what the rotate-and-quantize path of arXiv 2504.13989 computes
+(Section 2.1 quantizer, Section 3.1 clip ratio, Eq. (1) Sylvester recursion,
+Algorithm 2 Paley construction, Section 4.2 zero-pad expansion).  It shares no
+code with the CUDA library and must never be imported by the product package;
+only the tests, the smoke check and the CPU-baseline / reference leg of the
+benchmark use it.
+
+The shared object is compiled on first use with gcc (``build()``).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gbs_oracle.c")
+_LIB_PATH = os.path.join(_HERE, "libgbs_oracle.so")
+_lib = None
+
+F32 = 0
+BF16 = 1
+
+
+def build(force: bool = False) -> str:
+    """Compile gbs_oracle.c into libgbs_oracle.so next to it (gcc, OpenMP)."""
+    stale = (not os.path.exists(_LIB_PATH)
+             or os.path.getmtime(_LIB_PATH) < os.path.getmtime(_SRC))
+    if force or stale:
+        tmp = _LIB_PATH + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-fopenmp", "-fPIC", "-shared",
+                               _SRC, "-o", tmp, "-lm"])
+        os.replace(tmp, _LIB_PATH)
+    return _LIB_PATH
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        c_dp = ctypes.POINTER(ctypes.c_double)
+        lib.oracle_legendre.argtypes = [ctypes.c_long, ctypes.c_int]
+        lib.oracle_legendre.restype = ctypes.c_int
+        lib.oracle_gf27_chi.argtypes = [ctypes.c_int]
+        lib.oracle_gf27_chi.restype = ctypes.c_int
+        lib.oracle_gf27_mul.argtypes = [ctypes.c_int, ctypes.c_int]
+        lib.oracle_gf27_mul.restype = ctypes.c_int
+        lib.oracle_gf27_sub.argtypes = [ctypes.c_int, ctypes.c_int]
+        lib.oracle_gf27_sub.restype = ctypes.c_int
+        lib.oracle_hadamard_m.argtypes = [ctypes.c_int, ctypes.c_void_p]
+        lib.oracle_hadamard_m.restype = ctypes.c_int
+        lib.oracle_sylvester.argtypes = [ctypes.c_int, ctypes.c_void_p]
+        lib.oracle_sylvester.restype = ctypes.c_int
+        lib.oracle_rotate_dense.argtypes = [c_dp, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                            ctypes.c_int, c_dp]
+        lib.oracle_rotate_dense.restype = ctypes.c_int
+        lib.oracle_rotate_fast.argtypes = lib.oracle_rotate_dense.argtypes
+        lib.oracle_rotate_fast.restype = ctypes.c_int
+        lib.oracle_levels.argtypes = [ctypes.c_int, ctypes.c_int]
+        lib.oracle_levels.restype = ctypes.c_int
+        lib.oracle_quantize.argtypes = [c_dp, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                        ctypes.c_double, ctypes.c_int, ctypes.c_void_p, c_dp]
+        lib.oracle_quantize.restype = ctypes.c_int
+        lib.oracle_clip_error.argtypes = [c_dp, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+                                          ctypes.c_double, ctypes.c_int]
+        lib.oracle_clip_error.restype = ctypes.c_double
+        lib.oracle_pack.argtypes = [ctypes.c_void_p, ctypes.c_long, ctypes.c_int, ctypes.c_void_p]
+        lib.oracle_pack.restype = None
+        lib.oracle_unpack.argtypes = [ctypes.c_void_p, ctypes.c_long, ctypes.c_int, ctypes.c_void_p]
+        lib.oracle_unpack.restype = None
+        lib.oracle_rotate_quantize_rows.argtypes = [
+            ctypes.c_void_p, ctypes.c_int, ctypes.c_long, ctypes.c_long,
+            ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_double,
+            ctypes.c_int, ctypes.c_int,
+            ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int]
+        lib.oracle_rotate_quantize_rows.restype = ctypes.c_int
+        lib.oracle_clip_error_rows.argtypes = [
+            ctypes.c_void_p, ctypes.c_int, ctypes.c_long, ctypes.c_long,
+            ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+            c_dp, ctypes.c_int, c_dp, ctypes.c_void_p, ctypes.c_int]
+        lib.oracle_clip_error_rows.restype = ctypes.c_int
+        lib.oracle_dequantize_rows.argtypes = [
+            ctypes.c_void_p, c_dp, ctypes.c_long,
+            ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int,
+            c_dp, ctypes.c_int]
+        lib.oracle_dequantize_rows.restype = ctypes.c_int
+        lib.oracle_max_threads.argtypes = []
+        lib.oracle_max_threads.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _dp(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.POINTER(ctypes.c_double))
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise ValueError("oracle: %s failed (rc=%d: %s)" %
+                         (what, rc, "bad arguments" if rc == -1 else "out of memory"))
+
+
+def max_threads() -> int:
+    return _load().oracle_max_threads()
+
+
+def legendre(a: int, p: int) -> int:
+    """Legendre symbol (a/p) by exhaustive squaring (Section 2.3.3)."""
+    return _load().oracle_legendre(a, p)
+
+
+def gf27_chi(e: int) -> int:
+    return _load().oracle_gf27_chi(e)
+
+
+def gf27_mul(e: int, f: int) -> int:
+    return _load().oracle_gf27_mul(e, f)
+
+
+def gf27_sub(e: int, f: int) -> int:
+    return _load().oracle_gf27_sub(e, f)
+
+
+def hadamard_m(m: int) -> np.ndarray:
+    """H_m (int8, m x m): [1], Algorithm 2 for prime m-1 = 3 (mod 4), GF(27) for m = 28."""
+    H = np.zeros((m, m), dtype=np.int8)
+    _check(_load().oracle_hadamard_m(m, H.ctypes.data), "hadamard_m(%d)" % m)
+    return H
+
+
+def sylvester(n: int) -> np.ndarray:
+    """H_n by the recursion of Eq. (1)."""
+    H = np.zeros((n, n), dtype=np.int8)
+    _check(_load().oracle_sylvester(n, H.ctypes.data), "sylvester(%d)" % n)
+    return H
+
+
+def hadamard_full(m: int, k: int) -> np.ndarray:
+    """Dense H_m (x) H_{2^k} as int8 (small sizes only)."""
+    return np.kron(hadamard_m(m).astype(np.int64), sylvester(1 << k).astype(np.int64)).astype(np.int8)
+
+
+def levels(bits: int, literal: bool = False) -> int:
+    return _load().oracle_levels(bits, int(literal))
+
+
+def rotate(x, d_pad: int, m: int = 1, dense: bool = True, transpose: bool = False) -> np.ndarray:
+    """y = H_{d'} pad(x) / sqrt(d') for one row (x: 1-D float64 of length d <= d')."""
+    x = np.ascontiguousarray(x, dtype=np.float64)
+    y = np.empty(d_pad, dtype=np.float64)
+    fn = _load().oracle_rotate_dense if dense else _load().oracle_rotate_fast
+    _check(fn(_dp(x), x.shape[0], d_pad, m, int(transpose), _dp(y)), "rotate")
+    return y
+
+
+def quantize(y, bits: int, group: int = 0, alpha: float = 1.0, literal: bool = False):
+    """Codes (int32) and scaling factors Delta (float64) of one rotated row."""
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    n = y.shape[0]
+    q = np.empty(n, dtype=np.int32)
+    delta = np.empty(n // group if group else 1, dtype=np.float64)
+    _check(_load().oracle_quantize(_dp(y), n, bits, group, float(alpha), int(literal),
+                                   q.ctypes.data, _dp(delta)), "quantize")
+    return q, delta
+
+
+def clip_error(y, bits: int, group: int = 0, alpha: float = 1.0, literal: bool = False) -> float:
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    return float(_load().oracle_clip_error(_dp(y), y.shape[0], bits, group, float(alpha), int(literal)))
+
+
+def pack(q, bits: int) -> np.ndarray:
+    q = np.ascontiguousarray(q, dtype=np.int32).ravel()
+    out = np.zeros((q.shape[0] * bits + 7) // 8, dtype=np.uint8)
+    _load().oracle_pack(q.ctypes.data, q.shape[0], bits, out.ctypes.data)
+    return out
+
+
+def unpack(buf, n: int, bits: int) -> np.ndarray:
+    buf = np.ascontiguousarray(buf, dtype=np.uint8).ravel()
+    q = np.empty(n, dtype=np.int32)
+    _load().oracle_unpack(buf.ctypes.data, n, bits, q.ctypes.data)
+    return q
+
+
+def _as_input(x):
+    """Accept a 2-D float32 array, or a 2-D uint16 array holding bf16 bit patterns."""
+    x = np.asarray(x)
+    if x.ndim != 2:
+        raise ValueError("oracle: x must be 2-D [rows, >=d]")
+    if x.dtype == np.float32:
+        return np.ascontiguousarray(x), F32
+    if x.dtype == np.uint16:
+        return np.ascontiguousarray(x), BF16
+    raise ValueError("oracle: x must be float32 or uint16 (bf16 bits), got %s" % x.dtype)
+
+
+def rotate_quantize_rows(x, d: int, d_pad: int, m: int, bits: int, group: int, alpha: float,
+                         literal: bool = False, dense: bool = False, want_y: bool = True,
+                         want_q: bool = True, want_packed: bool = True, nthreads: int = 0):
+    """Batched pad -> rotate -> quantize -> pack.
+
+    Returns dict(y=[n,d'] f64, q=[n,d'] i32, packed=[n,d'*bits/8] u8, delta=[n,spr] f64).
+    """
+    x, dtype = _as_input(x)
+    n, stride = x.shape
+    spr = d_pad // group if group else 1
+    y = np.empty((n, d_pad), dtype=np.float64) if want_y else None
+    q = np.empty((n, d_pad), dtype=np.int32) if want_q else None
+    packed = np.empty((n, d_pad * bits // 8), dtype=np.uint8) if want_packed else None
+    delta = np.empty((n, spr), dtype=np.float64)
+    rc = _load().oracle_rotate_quantize_rows(
+        x.ctypes.data, dtype, n, stride, d, d_pad, m, bits, group, float(alpha),
+        int(literal), int(dense),
+        y.ctypes.data if want_y else None, q.ctypes.data if want_q else None,
+        packed.ctypes.data if want_packed else None, delta.ctypes.data, nthreads)
+    _check(rc, "rotate_quantize_rows")
+    return dict(y=y, q=q, packed=packed, delta=delta)
+
+
+def clip_error_rows(x, d: int, d_pad: int, m: int, bits: int, group: int, alphas,
+                    literal: bool = False, want_rows: bool = False, nthreads: int = 0):
+    """E_k = sum over rows and coordinates of (y - yhat_k)^2 for each alpha_k."""
+    x, dtype = _as_input(x)
+    n, stride = x.shape
+    alphas = np.ascontiguousarray(alphas, dtype=np.float64)
+    K = alphas.shape[0]
+    err = np.empty(K, dtype=np.float64)
+    rows = np.empty((n, K), dtype=np.float64) if want_rows else None
+    rc = _load().oracle_clip_error_rows(
+        x.ctypes.data, dtype, n, stride, d, d_pad, m, bits, group, int(literal),
+        _dp(alphas), K, _dp(err), rows.ctypes.data if want_rows else None, nthreads)
+    _check(rc, "clip_error_rows")
+    return (err, rows) if want_rows else err
+
+
+def dequantize_rows(packed, delta, d: int, d_pad: int, m: int, bits: int, group: int,
+                    inverse: bool = False, nthreads: int = 0) -> np.ndarray:
+    """yhat = q * Delta (width d'), or with inverse: xhat = (H^T yhat / sqrt(d'))[:d]."""
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    delta = np.ascontiguousarray(delta, dtype=np.float64)
+    n = packed.shape[0]
+    out = np.empty((n, d if inverse else d_pad), dtype=np.float64)
+    rc = _load().oracle_dequantize_rows(packed.ctypes.data, _dp(delta), n, d, d_pad, m, bits, group,
+                                        int(inverse), _dp(out), nthreads)
+    _check(rc, "dequantize_rows")
+    return out
