@@ -1,0 +1,149 @@
+/*
+ * gbs.h -- C ABI of the B200 (sm_100a) rotate-and-quantize library.
+ *
+ * The library implements the online activation / KV path of "Gradual Binary Search and
+ * Dimension Expansion" (arXiv 2504.13989): every token row of width d is zero-padded to
+ * d' = m * 2^k (Section 4.2, Eq. (2)), rotated by the normalised Hadamard matrix
+ * H_{d'} = H_m (x) H_{2^k} / sqrt(d')  (Sylvester recursion of Eq. (1) for the power of two,
+ * Paley's Algorithm 2 for the factor m, 1/sqrt(n) normalisation of Appendix A), quantized per
+ * token or per group with the symmetric uniform quantizer of Section 2.1 under the clip ratio
+ * alpha of Section 3.1, and bit-packed.  A companion call scores K candidate clip ratios by
+ * quantization error, the quantity a clip-ratio search such as Algorithm 1 queries.
+ *
+ * Conventions
+ *   - Every function returns an int status: GBS_OK (0) or a negative GBS_ERR_* code.
+ *     Nothing throws, prints, or synchronises the device.  Argument errors are detected on
+ *     the host before any kernel is launched; no call can fault the device through a bad
+ *     size (pointers themselves cannot be validated and are the caller's responsibility).
+ *   - "device pointer" = memory of the CUDA device that was current when the plan was
+ *     created.  The caller owns all buffers; the library never allocates per call.
+ *   - Work is enqueued on the CUDA stream passed as `cuda_stream` (a cudaStream_t cast to
+ *     void*; NULL = the legacy default stream) and the call returns without waiting.
+ *   - Rotated coordinate i of a row is i = a * 2^k + c with a in [0,m), c in [0,2^k):
+ *     y[i] = (1/sqrt(d')) * sum_{a',c'} H_m[a,a'] * (-1)^popcount(c & c') * x_pad[a'*2^k + c'].
+ *   - Quantizer: per token (group = 0) or per run of `group` consecutive rotated coordinates,
+ *     M = max|y|, Delta = alpha * M / D with D = 2^(bits-1) - 1, code q = clamp(rint(y/Delta),
+ *     -D, D) (round half to even); M = 0 gives codes 0 and Delta 0.  (Read with `bits` as the
+ *     number of magnitude bits, this is the printed formula Delta = max|X| / (2^b - 1): the
+ *     printed formula at b equals this one at bits = b + 1.)
+ *   - Packed codes: element j of a row occupies bits [j*bits, (j+1)*bits) of the row's
+ *     little-endian bit stream and holds the low `bits` bits of the two's-complement code
+ *     (bits = 4: even index in the low nibble).  Row r starts at byte r * d' * bits / 8.
+ *   - Scales: fp32 Delta, layout [n_rows, scales_per_row], scales_per_row = group ? d'/group : 1.
+ */
+#ifndef GBS_H_
+#define GBS_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* status codes */
+#define GBS_OK 0
+#define GBS_ERR_INVALID_ARG (-1) /* a size, pointer or parameter is out of its documented range */
+#define GBS_ERR_UNSUPPORTED (-2) /* no Hadamard construction for this m, or d' too large */
+#define GBS_ERR_ALIGNMENT (-3)   /* a pointer or stride violates the stated alignment */
+#define GBS_ERR_CUDA (-4)        /* a CUDA runtime call failed (e.g. no device, launch error) */
+#define GBS_ERR_ALLOC (-5)       /* host or device allocation for the plan failed */
+
+/* element types of activation inputs / dequantized outputs */
+#define GBS_DTYPE_F32 0
+#define GBS_DTYPE_BF16 1
+
+/* gbs_dequantize flags */
+#define GBS_INVERSE_ROTATE 1
+
+/* largest padded width and largest number of clip-ratio candidates per call */
+#define GBS_MAX_D_PAD 32768
+#define GBS_MAX_CANDIDATES 64
+
+typedef struct gbs_plan gbs_plan_t;
+
+typedef struct gbs_plan_info {
+    int d, d_pad, m, k;            /* d' = m * 2^k                                   */
+    int bits, group;               /* group = 0: one scale per token                  */
+    float alpha;
+    int levels;                    /* D = 2^(bits-1) - 1; codes lie in [-D, D]        */
+    int q_lo, q_hi;                /* -D, +D                                          */
+    int64_t code_bytes_per_row;    /* d' * bits / 8                                   */
+    int scales_per_row;            /* group ? d'/group : 1                            */
+    int variant;                   /* kernel family chosen for bf16 rows: 0 = generic */
+} gbs_plan_info_t;
+
+/*
+ * Create a plan (Section 4.2 for d -> d'; Eq. (1) and Algorithm 2 for the rotation;
+ * Section 2.1 / 3.1 for bits and alpha).
+ *   d       row width, 1 <= d <= d_pad
+ *   d_pad   d' = m * 2^k with 2^k >= 8 and d' <= GBS_MAX_D_PAD
+ *   m       1 (pure Sylvester), or 12, 20, 24 (Algorithm 2 with p = m-1), or 28 (Algorithm 2
+ *           over GF(27) = GF(3)[x]/(x^3+2x+1), elements indexed c0 + 3 c1 + 9 c2)
+ *   bits    3 or 4
+ *   group   0, or a power of two >= 8 dividing 2^k (so a group never straddles a block of H_m)
+ *   alpha   0 < alpha <= 1
+ * The plan owns small device tables (the signs of H_m) on the current device, is immutable
+ * and may be used from several threads / streams at once.  *out is written only on success.
+ */
+int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bits, int group, float alpha);
+
+/* Free a plan.  NULL is accepted.  Work already enqueued with the plan must have finished. */
+int gbs_plan_destroy(gbs_plan_t* plan);
+
+/* Report the derived sizes of a plan. */
+int gbs_plan_info(const gbs_plan_t* plan, gbs_plan_info_t* out);
+
+/*
+ * Fused pad -> rotate -> per-token/group absmax -> scale -> round/clip -> pack
+ * (Section 4.2, Eq. (1), Algorithm 2, Section 2.1, Section 3.1), one pass over x.
+ *   x            device, n_rows rows of d elements of x_dtype; row r starts at element
+ *                r * x_row_stride.  Must be 16-byte aligned with x_row_stride * sizeof(elem)
+ *                a multiple of 16, x_row_stride >= d.
+ *   codes        device, n_rows * d' * bits / 8 bytes, 16-byte aligned
+ *   scales       device, n_rows * scales_per_row floats
+ *   y_opt        NULL, or device n_rows * d' floats receiving the rotated normalised values
+ *                (16-byte aligned)
+ * n_rows = 0 is a successful no-op.
+ */
+int gbs_rotate_quantize(const gbs_plan_t* plan, const void* x, int x_dtype, int64_t n_rows,
+                        int64_t x_row_stride, void* codes, float* scales, float* y_opt,
+                        void* cuda_stream);
+
+/*
+ * Inverse of the quantizer: yhat = q * Delta (Section 2.1) in the rotated domain, width d';
+ * with GBS_INVERSE_ROTATE also xhat = (H_{d'}^T yhat / sqrt(d'))[0:d] (rotations are undone by
+ * the transpose, Section 2.3.1), width d.
+ *   codes, scales  device, layouts as written by gbs_rotate_quantize
+ *   out            device, n_rows * (d' or d) elements of out_dtype, rows contiguous,
+ *                  16-byte aligned
+ */
+int gbs_dequantize(const gbs_plan_t* plan, const void* codes, const float* scales, int64_t n_rows,
+                   void* out, int out_dtype, int flags, void* cuda_stream);
+
+/*
+ * Score K clip ratios: for each alpha_k, err_sum[k] += sum over rows and rotated coordinates of
+ * (y - yhat_k)^2, yhat_k being the quantizer output (Section 2.1) under clip ratio alpha_k
+ * (Section 3.1).  The plan's own alpha is ignored; bits and group are honoured.
+ *   x, x_dtype, n_rows, x_row_stride   as for gbs_rotate_quantize
+ *   alphas_host   HOST pointer to K floats, each in (0, 1]; copied at call time
+ *   K             1 .. GBS_MAX_CANDIDATES
+ *   err_sum       device, K doubles, ACCUMULATED into (the caller zeroes them)
+ *   err_rows_opt  NULL, or device n_rows * K floats receiving the per-row sums
+ */
+int gbs_clip_error(const gbs_plan_t* plan, const void* x, int x_dtype, int64_t n_rows,
+                   int64_t x_row_stride, const float* alphas_host, int K, double* err_sum,
+                   float* err_rows_opt, void* cuda_stream);
+
+/*
+ * Host-only helper: write the m x m sign matrix H_m (row-major, +1 / -1) the plans use
+ * (Algorithm 2).  `out_host` must hold m*m bytes.  Needs no device.
+ */
+int gbs_hadamard_m(int m, int8_t* out_host);
+
+/* Human-readable name of a status code (static string). */
+const char* gbs_status_string(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GBS_H_ */

@@ -1,0 +1,253 @@
+"""Thin ctypes binding of libgbs.so (the C ABI declared in include/gbs.h).
+
+Argument marshalling only: every step of the path runs in the library's CUDA kernels.
+PyTorch is used for device memory and streams.  There is no CPU fallback: if the shared
+library is missing or a call fails, a GbsError is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_PKG, "libgbs.so")
+
+GBS_OK = 0
+GBS_ERR_INVALID_ARG = -1
+GBS_ERR_UNSUPPORTED = -2
+GBS_ERR_ALIGNMENT = -3
+GBS_ERR_CUDA = -4
+GBS_ERR_ALLOC = -5
+GBS_DTYPE_F32 = 0
+GBS_DTYPE_BF16 = 1
+GBS_INVERSE_ROTATE = 1
+GBS_MAX_D_PAD = 32768
+GBS_MAX_CANDIDATES = 64
+
+EXPORTS = ("gbs_plan_create", "gbs_plan_destroy", "gbs_plan_info", "gbs_rotate_quantize",
+           "gbs_dequantize", "gbs_clip_error", "gbs_hadamard_m", "gbs_status_string")
+
+
+class GbsError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__("%s failed: %s" % (what, status_string(status)))
+
+
+class PlanInfo(ctypes.Structure):
+    _fields_ = [("d", ctypes.c_int), ("d_pad", ctypes.c_int), ("m", ctypes.c_int), ("k", ctypes.c_int),
+                ("bits", ctypes.c_int), ("group", ctypes.c_int), ("alpha", ctypes.c_float),
+                ("levels", ctypes.c_int), ("q_lo", ctypes.c_int), ("q_hi", ctypes.c_int),
+                ("code_bytes_per_row", ctypes.c_int64), ("scales_per_row", ctypes.c_int),
+                ("variant", ctypes.c_int)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """Load libgbs.so (built in-tree by paper_2504_13989_b200.build); fail loudly if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise GbsErrorMissing("libgbs.so not found at %s -- run `python -m paper_2504_13989_b200.build` "
+                                  "(or __graft_entry__.build()); there is no CPU fallback" % _LIB_PATH)
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i32, i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
+        L.gbs_plan_create.argtypes = [ctypes.POINTER(vp), i32, i32, i32, i32, i32, ctypes.c_float]
+        L.gbs_plan_create.restype = i32
+        L.gbs_plan_destroy.argtypes = [vp]
+        L.gbs_plan_destroy.restype = i32
+        L.gbs_plan_info.argtypes = [vp, ctypes.POINTER(PlanInfo)]
+        L.gbs_plan_info.restype = i32
+        L.gbs_rotate_quantize.argtypes = [vp, vp, i32, i64, i64, vp, vp, vp, vp]
+        L.gbs_rotate_quantize.restype = i32
+        L.gbs_dequantize.argtypes = [vp, vp, vp, i64, vp, i32, i32, vp]
+        L.gbs_dequantize.restype = i32
+        L.gbs_clip_error.argtypes = [vp, vp, i32, i64, i64, ctypes.POINTER(ctypes.c_float), i32, vp, vp, vp]
+        L.gbs_clip_error.restype = i32
+        L.gbs_hadamard_m.argtypes = [i32, vp]
+        L.gbs_hadamard_m.restype = i32
+        L.gbs_status_string.argtypes = [i32]
+        L.gbs_status_string.restype = ctypes.c_char_p
+        _lib = L
+    return _lib
+
+
+class GbsErrorMissing(RuntimeError):
+    pass
+
+
+def status_string(status: int) -> str:
+    return lib().gbs_status_string(int(status)).decode()
+
+
+def _check(status: int, what: str):
+    if status != GBS_OK:
+        raise GbsError(status, what)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return GBS_DTYPE_F32
+    if t.dtype == torch.bfloat16:
+        return GBS_DTYPE_BF16
+    raise TypeError("gbs: tensors must be float32 or bfloat16, got %s" % t.dtype)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream)
+
+
+def _rows_view(x: torch.Tensor, d: int):
+    """(pointer, n_rows, row stride in elements) of a [..., d] tensor whose leading dims are contiguous rows."""
+    if not x.is_cuda:
+        raise ValueError("gbs: x must be a CUDA tensor (device pointer); there is no CPU path")
+    if x.dim() < 1 or x.shape[-1] != d:
+        raise ValueError("gbs: last dimension of x must be d=%d, got shape %s" % (d, tuple(x.shape)))
+    if x.dim() == 1:
+        x = x.unsqueeze(0)
+    if x.stride(-1) != 1:
+        raise ValueError("gbs: the last dimension of x must be contiguous")
+    if x.dim() > 2:
+        x = x.reshape(-1, d) if x.is_contiguous() else x.flatten(0, -2)
+    return x, x.shape[0], (x.stride(0) if x.shape[0] > 1 else max(x.stride(0), d))
+
+
+# ----------------------------------------------------------------------------------------------
+# functions named after the C entry points
+# ----------------------------------------------------------------------------------------------
+def gbs_plan_create(d: int, d_pad: int, m: int, bits: int, group: int, alpha: float) -> int:
+    """Returns an opaque plan handle (int).  See include/gbs.h for the argument ranges."""
+    h = ctypes.c_void_p()
+    _check(lib().gbs_plan_create(ctypes.byref(h), d, d_pad, m, bits, group, alpha), "gbs_plan_create")
+    return h.value
+
+
+def gbs_plan_destroy(plan: int) -> None:
+    _check(lib().gbs_plan_destroy(ctypes.c_void_p(plan)), "gbs_plan_destroy")
+
+
+def gbs_plan_info(plan: int) -> PlanInfo:
+    info = PlanInfo()
+    _check(lib().gbs_plan_info(ctypes.c_void_p(plan), ctypes.byref(info)), "gbs_plan_info")
+    return info
+
+
+def gbs_hadamard_m(m: int) -> torch.Tensor:
+    """The m x m sign matrix H_m the plans use (host computation, int8)."""
+    out = torch.zeros((m, m), dtype=torch.int8)
+    _check(lib().gbs_hadamard_m(m, out.data_ptr()), "gbs_hadamard_m")
+    return out
+
+
+def gbs_rotate_quantize(plan: int, x: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor,
+                        y_opt: torch.Tensor | None = None, stream=None) -> None:
+    info = gbs_plan_info(plan)
+    xv, n_rows, stride = _rows_view(x, info.d)
+    _check(lib().gbs_rotate_quantize(ctypes.c_void_p(plan), xv.data_ptr(), _dtype_code(xv), n_rows, stride,
+                                     codes.data_ptr(), scales.data_ptr(),
+                                     y_opt.data_ptr() if y_opt is not None else None, _stream_ptr(stream)),
+           "gbs_rotate_quantize")
+
+
+def gbs_dequantize(plan: int, codes: torch.Tensor, scales: torch.Tensor, n_rows: int, out: torch.Tensor,
+                   flags: int = 0, stream=None) -> None:
+    _check(lib().gbs_dequantize(ctypes.c_void_p(plan), codes.data_ptr(), scales.data_ptr(), n_rows,
+                                out.data_ptr(), _dtype_code(out), flags, _stream_ptr(stream)),
+           "gbs_dequantize")
+
+
+def gbs_clip_error(plan: int, x: torch.Tensor, alphas, err_sum: torch.Tensor,
+                   err_rows_opt: torch.Tensor | None = None, stream=None) -> None:
+    info = gbs_plan_info(plan)
+    xv, n_rows, stride = _rows_view(x, info.d)
+    alphas = [float(a) for a in alphas]
+    arr = (ctypes.c_float * len(alphas))(*alphas)
+    if err_sum.dtype != torch.float64:
+        raise TypeError("gbs: err_sum must be float64")
+    _check(lib().gbs_clip_error(ctypes.c_void_p(plan), xv.data_ptr(), _dtype_code(xv), n_rows, stride,
+                                arr, len(alphas), err_sum.data_ptr(),
+                                err_rows_opt.data_ptr() if err_rows_opt is not None else None,
+                                _stream_ptr(stream)),
+           "gbs_clip_error")
+
+
+# ----------------------------------------------------------------------------------------------
+# convenience object: owns a plan handle and allocates outputs with torch
+# ----------------------------------------------------------------------------------------------
+class Plan:
+    """RAII wrapper of a gbs plan; allocates output tensors with torch and forwards to the C ABI."""
+
+    def __init__(self, d: int, d_pad: int | None = None, m: int = 1, bits: int = 4, group: int = 0,
+                 alpha: float = 1.0):
+        d_pad = d if d_pad is None else d_pad
+        self.handle = gbs_plan_create(d, d_pad, m, bits, group, alpha)
+        self.info = gbs_plan_info(self.handle)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            gbs_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+
+    def alloc_outputs(self, n_rows: int, device, want_y: bool = False):
+        codes = torch.empty((n_rows, self.info.code_bytes_per_row), dtype=torch.uint8, device=device)
+        scales = torch.empty((n_rows, self.info.scales_per_row), dtype=torch.float32, device=device)
+        y = torch.empty((n_rows, self.info.d_pad), dtype=torch.float32, device=device) if want_y else None
+        return codes, scales, y
+
+    def rotate_quantize(self, x: torch.Tensor, want_y: bool = False, out=None, stream=None):
+        n_rows = x.numel() // self.info.d
+        codes, scales, y = out if out is not None else self.alloc_outputs(n_rows, x.device, want_y)
+        gbs_rotate_quantize(self.handle, x, codes, scales, y, stream)
+        return codes, scales, y
+
+    def dequantize(self, codes: torch.Tensor, scales: torch.Tensor, inverse: bool = False,
+                   dtype=torch.float32, out=None, stream=None) -> torch.Tensor:
+        n_rows = codes.shape[0]
+        width = self.info.d if inverse else self.info.d_pad
+        if out is None:
+            out = torch.empty((n_rows, width), dtype=dtype, device=codes.device)
+        gbs_dequantize(self.handle, codes, scales, n_rows, out, GBS_INVERSE_ROTATE if inverse else 0, stream)
+        return out
+
+    def clip_error(self, x: torch.Tensor, alphas, want_rows: bool = False, err_sum=None, stream=None):
+        n_rows = x.numel() // self.info.d
+        K = len(alphas)
+        if err_sum is None:
+            err_sum = torch.zeros(K, dtype=torch.float64, device=x.device)
+        rows = torch.empty((n_rows, K), dtype=torch.float32, device=x.device) if want_rows else None
+        gbs_clip_error(self.handle, x, alphas, err_sum, rows, stream)
+        return (err_sum, rows) if want_rows else err_sum
+
+    def rotate_quantize_host(self, x_host: torch.Tensor, codes_host: torch.Tensor, scales_host: torch.Tensor,
+                             device="cuda:0", stream=None):
+        """End-to-end call for host-resident data: pinned host -> device, rotate_quantize, device -> host.
+
+        x_host / codes_host / scales_host are (ideally pinned) CPU tensors; the copies are enqueued on
+        the same stream as the kernel.  Returns after the stream has been synchronised.
+        """
+        s = stream or torch.cuda.current_stream()
+        with torch.cuda.stream(s):
+            x = x_host.to(device, non_blocking=True)
+            codes, scales, _ = self.rotate_quantize(x, stream=s)
+            codes_host.copy_(codes, non_blocking=True)
+            scales_host.copy_(scales, non_blocking=True)
+        s.synchronize()
+        return codes_host, scales_host

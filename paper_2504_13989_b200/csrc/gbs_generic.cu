@@ -1,0 +1,693 @@
+// Generic kernel family: works for every supported (m, k), fp32 or bf16 rows, 3 or 4 bits, per-token
+// or per-group scales.  A team of up to 256 threads owns one token row; the padded row lives in
+// shared memory as fp32.
+//
+//   S0/S1  load the row, append zeros up to d'                     (Section 4.2, Eq. (2))
+//   S3     Sylvester butterflies inside each block of 2^k          (Eq. (1))
+//   S2     m x m Paley mix across the m blocks                     (Algorithm 2)
+//   S4-S8  1/sqrt(d'), absmax, Delta, round/clip, pack, store      (Appendix A; Sections 2.1, 3.1)
+//
+// The two factors of H_m (x) H_{2^k} act on different index digits and commute; the butterflies
+// run first because the first three stages are done in registers straight from the global load.
+//
+// The specialised tensor-core families reuse none of this file; it is the fallback and the path for
+// fp32 inputs.
+#include <cuda_bf16.h>
+
+#include "gbs_internal.h"
+
+namespace {
+
+constexpr int NT = 256;             // threads per block
+constexpr unsigned FULL = 0xffffffffu;
+
+struct GenericParams {
+    int d, d_pad, k, m, n2;          // n2 = 2^k
+    int group, G, spr;               // G = group ? group : d_pad ; spr = scales per row
+    int levels;
+    float norm, c_scale, c_inv;
+    int tt_log2, rows_per_cta;       // team = 1 << tt_log2 threads per row
+    int chunks;                      // d_pad / 8
+    int red_mode, seg_lanes;         // absmax reduction strategy (see reduce_group_max)
+    int row_floats;                  // d_pad + d_pad/32 (one pad word per 32)
+    int row_bytes;                   // d_pad * bits / 8
+    int stage_bytes;                 // row_bytes rounded up to 16
+    int n_pass;
+    int pass_s[8], pass_r[8];        // butterfly passes over bits [s, s+r) in shared memory
+    long long n_rows, stride;
+    const float* hm;                 // device H_m (forward) or H_m^T (inverse), m*m floats
+};
+
+__device__ __forceinline__ int pidx(int i) { return i + (i >> 5); }
+
+// ---- global loads of one chunk of 8 consecutive elements, zero beyond d ---------------------------
+__device__ __forceinline__ void load_chunk8(const float* xrow, int idx, int d, float v[8])
+{
+    if (idx + 8 <= d) {
+        float4 a = __ldg(reinterpret_cast<const float4*>(xrow + idx));
+        float4 b = __ldg(reinterpret_cast<const float4*>(xrow + idx + 4));
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+        v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    } else {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) v[e] = (idx + e < d) ? __ldg(xrow + idx + e) : 0.f;
+    }
+}
+
+__device__ __forceinline__ void load_chunk8(const __nv_bfloat16* xrow, int idx, int d, float v[8])
+{
+    if (idx + 8 <= d) {
+        uint4 r = __ldg(reinterpret_cast<const uint4*>(xrow + idx));
+        unsigned w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            v[2 * e] = __uint_as_float(w[e] << 16);
+            v[2 * e + 1] = __uint_as_float(w[e] & 0xffff0000u);
+        }
+    } else {
+        const unsigned short* xs = reinterpret_cast<const unsigned short*>(xrow);
+#pragma unroll
+        for (int e = 0; e < 8; ++e)
+            v[e] = (idx + e < d) ? __uint_as_float(((unsigned)__ldg(xs + idx + e)) << 16) : 0.f;
+    }
+}
+
+template <int N>
+__device__ __forceinline__ void butterflies(float v[N])
+{
+#pragma unroll
+    for (int h = 1; h < N; h <<= 1)
+#pragma unroll
+        for (int i = 0; i < N; ++i)
+            if ((i & h) == 0) {
+                float a = v[i], b = v[i + h];
+                v[i] = a + b;
+                v[i + h] = a - b;
+            }
+}
+
+// One butterfly pass over index bits [s, s+R) of a row held in shared memory.
+template <int R>
+__device__ __forceinline__ void fwht_pass(float* row, int s, int d_pad, int j, int tt)
+{
+    const int items = d_pad >> R;
+    for (int w = j; w < items; w += tt) {
+        int low = w & ((1 << s) - 1);
+        int base = ((w >> s) << (s + R)) | low;
+        float v[1 << R];
+#pragma unroll
+        for (int t = 0; t < (1 << R); ++t) v[t] = row[pidx(base + (t << s))];
+        butterflies<(1 << R)>(v);
+#pragma unroll
+        for (int t = 0; t < (1 << R); ++t) row[pidx(base + (t << s))] = v[t];
+    }
+}
+
+// U = H_m * X_mat: thread-owned columns, signs (as +-1.0f) read from shared memory.
+template <int M>
+__device__ __forceinline__ void paley_mix(float* row, const float* hm_s, int n2, int j, int tt)
+{
+    for (int c = j; c < n2; c += tt) {
+        float u[M];
+#pragma unroll
+        for (int a = 0; a < M; ++a) u[a] = row[pidx(a * n2 + c)];
+#pragma unroll 4
+        for (int a = 0; a < M; ++a) {
+            const float4* hr = reinterpret_cast<const float4*>(hm_s + a * M);
+            float acc = 0.f;
+#pragma unroll
+            for (int q = 0; q < M / 4; ++q) {
+                float4 h = hr[q];
+                acc = fmaf(h.x, u[4 * q], acc);
+                acc = fmaf(h.y, u[4 * q + 1], acc);
+                acc = fmaf(h.z, u[4 * q + 2], acc);
+                acc = fmaf(h.w, u[4 * q + 3], acc);
+            }
+            row[pidx(a * n2 + c)] = acc;
+        }
+    }
+}
+
+__device__ __forceinline__ void run_passes_and_mix(const GenericParams& P, float* row, const float* hm_s,
+                                                   int j, int tt)
+{
+    for (int ps = 0; ps < P.n_pass; ++ps) {
+        __syncthreads();
+        const int s = P.pass_s[ps];
+        switch (P.pass_r[ps]) {
+            case 1: fwht_pass<1>(row, s, P.d_pad, j, tt); break;
+            case 2: fwht_pass<2>(row, s, P.d_pad, j, tt); break;
+            case 3: fwht_pass<3>(row, s, P.d_pad, j, tt); break;
+            default: fwht_pass<4>(row, s, P.d_pad, j, tt); break;
+        }
+    }
+    if (P.m > 1) {
+        __syncthreads();
+        switch (P.m) {
+            case 12: paley_mix<12>(row, hm_s, P.n2, j, tt); break;
+            case 20: paley_mix<20>(row, hm_s, P.n2, j, tt); break;
+            case 24: paley_mix<24>(row, hm_s, P.n2, j, tt); break;
+            default: paley_mix<28>(row, hm_s, P.n2, j, tt); break;
+        }
+    }
+    __syncthreads();
+}
+
+// Load + pad + first three butterfly stages in registers -> shared memory, then the rest.
+template <typename InT>
+__device__ __forceinline__ void rotate_row_to_smem(const GenericParams& P, const InT* x, long long row,
+                                                   bool active, float* rowbuf, const float* hm_s, int j,
+                                                   int tt)
+{
+    if (active) {
+        const InT* xrow = x + row * P.stride;
+        for (int ch = j; ch < P.chunks; ch += tt) {
+            float v[8];
+            load_chunk8(xrow, ch * 8, P.d, v);
+            butterflies<8>(v);
+            const int p = ch * 8 + (ch >> 2);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) rowbuf[p + e] = v[e];
+        }
+    }
+    run_passes_and_mix(P, rowbuf, hm_s, j, tt);
+}
+
+// max|.| of a group of G consecutive values, each thread holding the max of its 8-value chunk.
+//   mode 1: G is a power of two <= 256: xor-shuffle over the G/8 adjacent lanes, leader stores
+//   mode 2: G is a multiple of 256: the whole warp shares one group: warp max, one atomic
+//   mode 3: anything else: one shared-memory atomic per chunk
+__device__ __forceinline__ void reduce_group_max(const GenericParams& P, float amax, int ch, bool valid,
+                                                 unsigned* gmax)
+{
+    const int lane = threadIdx.x & 31;
+    if (P.red_mode == 1) {
+        for (int o = P.seg_lanes >> 1; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, o));
+        if (valid && (lane & (P.seg_lanes - 1)) == 0) gmax[(ch * 8) / P.G] = __float_as_uint(amax);
+    } else if (P.red_mode == 2) {
+        for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(FULL, amax, o));
+        if (valid && lane == 0) atomicMax(&gmax[(ch * 8) / P.G], __float_as_uint(amax));
+    } else {
+        if (valid) atomicMax(&gmax[(ch * 8) / P.G], __float_as_uint(amax));
+    }
+}
+
+__device__ __forceinline__ void read_chunk_smem(const float* rowbuf, int ch, float v[8])
+{
+    const int p = ch * 8 + (ch >> 2);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = rowbuf[p + e];
+}
+
+// Team-wide absmax of the rotated row into gmax[0 .. spr).  Ends with a block barrier.
+__device__ __forceinline__ void row_group_max(const GenericParams& P, const float* rowbuf, unsigned* gmax,
+                                              bool active, int j, int tt)
+{
+    const int iters = (P.chunks + tt - 1) / tt;
+    for (int it = 0; it < iters; ++it) {
+        const int ch = j + it * tt;
+        const bool valid = active && ch < P.chunks;
+        float amax = 0.f;
+        if (valid) {
+            float v[8];
+            read_chunk_smem(rowbuf, ch, v);
+#pragma unroll
+            for (int e = 0; e < 8; ++e) amax = fmaxf(amax, fabsf(v[e]));
+        }
+        reduce_group_max(P, amax, valid ? ch : 0, valid, gmax);
+    }
+    __syncthreads();
+}
+
+struct SmemLayout {
+    float* rowbuf;      // [R][row_floats]
+    unsigned* gmax;     // [R][spr]
+    float* hm_s;        // [m*m]
+    unsigned char* tail;  // kernel-specific
+};
+
+__device__ __forceinline__ SmemLayout carve(const GenericParams& P, unsigned char* smem)
+{
+    SmemLayout L;
+    L.rowbuf = reinterpret_cast<float*>(smem);
+    size_t off = sizeof(float) * (size_t)P.rows_per_cta * P.row_floats;
+    L.gmax = reinterpret_cast<unsigned*>(smem + off);
+    off += sizeof(unsigned) * (size_t)P.rows_per_cta * P.spr;
+    off = (off + 15) & ~(size_t)15;
+    L.hm_s = reinterpret_cast<float*>(smem + off);
+    off += sizeof(float) * (size_t)((P.m > 1) ? P.m * P.m : 0);
+    off = (off + 15) & ~(size_t)15;
+    L.tail = smem + off;
+    return L;
+}
+
+__device__ __forceinline__ void stage_hm(const GenericParams& P, float* hm_s)
+{
+    if (P.m > 1)
+        for (int i = threadIdx.x; i < P.m * P.m; i += NT) hm_s[i] = P.hm[i];
+}
+
+__device__ __forceinline__ void clear_gmax(const GenericParams& P, unsigned* gmax)
+{
+    for (int i = threadIdx.x; i < P.rows_per_cta * P.spr; i += NT) gmax[i] = 0u;
+}
+
+// ======================================================================================
+// rotate + quantize + pack
+// ======================================================================================
+template <typename InT, int BITS>
+__global__ void __launch_bounds__(NT) k_rotate_quantize(GenericParams P, const InT* __restrict__ x,
+                                                        unsigned char* __restrict__ codes,
+                                                        float* __restrict__ scales, float* __restrict__ y_opt)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    SmemLayout L = carve(P, smem);
+    unsigned char* stage_all = L.tail;
+    stage_hm(P, L.hm_s);
+
+    const int tt = 1 << P.tt_log2;
+    const int team = threadIdx.x >> P.tt_log2;
+    const int j = threadIdx.x & (tt - 1);
+    float* rowbuf = L.rowbuf + (size_t)team * P.row_floats;
+    unsigned* gmax = L.gmax + (size_t)team * P.spr;
+    unsigned char* stage = stage_all + (size_t)team * P.stage_bytes;
+    const float fD = (float)P.levels;
+
+    for (long long row0 = (long long)blockIdx.x * P.rows_per_cta; row0 < P.n_rows;
+         row0 += (long long)gridDim.x * P.rows_per_cta) {
+        const long long row = row0 + team;
+        const bool active = row < P.n_rows;
+        clear_gmax(P, L.gmax);
+        rotate_row_to_smem<InT>(P, x, row, active, rowbuf, L.hm_s, j, tt);
+        row_group_max(P, rowbuf, gmax, active, j, tt);
+
+        if (active) {
+            for (int ch = j; ch < P.chunks; ch += tt) {
+                float v[8];
+                read_chunk_smem(rowbuf, ch, v);
+                const int g = (ch * 8) / P.G;
+                const float M = __uint_as_float(gmax[g]);
+                const float delta = P.c_scale * M;
+                const float inv = (M > 0.f) ? (P.c_inv / M) : 0.f;
+                if ((ch * 8) % P.G == 0) scales[row * P.spr + g] = delta;
+                unsigned word = 0;
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                    float t = fminf(fmaxf(v[e] * inv, -fD), fD);
+                    int q = __float2int_rn(t);
+                    word |= ((unsigned)q & ((1u << BITS) - 1u)) << (BITS * e);
+                }
+                if (BITS == 4) {
+                    *reinterpret_cast<unsigned*>(stage + ch * 4) = word;
+                } else {
+                    stage[ch * 3] = (unsigned char)(word & 0xff);
+                    stage[ch * 3 + 1] = (unsigned char)((word >> 8) & 0xff);
+                    stage[ch * 3 + 2] = (unsigned char)((word >> 16) & 0xff);
+                }
+                if (y_opt) {
+                    float4* yo = reinterpret_cast<float4*>(y_opt + row * P.d_pad + ch * 8);
+                    yo[0] = make_float4(v[0] * P.norm, v[1] * P.norm, v[2] * P.norm, v[3] * P.norm);
+                    yo[1] = make_float4(v[4] * P.norm, v[5] * P.norm, v[6] * P.norm, v[7] * P.norm);
+                }
+            }
+        }
+        __syncthreads();
+        if (active) {
+            unsigned char* dst = codes + row * P.row_bytes;
+            if ((P.row_bytes & 15) == 0) {
+                const uint4* s4 = reinterpret_cast<const uint4*>(stage);
+                uint4* d4 = reinterpret_cast<uint4*>(dst);
+                for (int i = j; i < (P.row_bytes >> 4); i += tt) d4[i] = s4[i];
+            } else {
+                for (int i = j; i < P.row_bytes; i += tt) dst[i] = stage[i];
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// ======================================================================================
+// clip-ratio scoring
+// ======================================================================================
+constexpr int KT = 8;   // candidates scored per sweep over the row
+
+struct ClipConsts {
+    float c_scale[GBS_MAX_CANDIDATES];   // alpha_k / (D sqrt(d'))
+    float c_inv[GBS_MAX_CANDIDATES];     // D / alpha_k
+};
+
+template <typename InT>
+__global__ void __launch_bounds__(NT) k_clip_error(GenericParams P, ClipConsts C, int K,
+                                                   const InT* __restrict__ x, double* __restrict__ err_sum,
+                                                   float* __restrict__ err_rows)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    SmemLayout L = carve(P, smem);
+    // tail: double cta_sum[K]; float row_err[R][K]
+    double* cta_sum = reinterpret_cast<double*>(L.tail);
+    float* row_err_all = reinterpret_cast<float*>(L.tail + sizeof(double) * GBS_MAX_CANDIDATES);
+    stage_hm(P, L.hm_s);
+    for (int i = threadIdx.x; i < K; i += NT) cta_sum[i] = 0.0;
+
+    const int tt = 1 << P.tt_log2;
+    const int team = threadIdx.x >> P.tt_log2;
+    const int j = threadIdx.x & (tt - 1);
+    const int lane = threadIdx.x & 31;
+    float* rowbuf = L.rowbuf + (size_t)team * P.row_floats;
+    unsigned* gmax = L.gmax + (size_t)team * P.spr;
+    float* row_err = row_err_all + (size_t)team * GBS_MAX_CANDIDATES;
+    const float fD = (float)P.levels;
+    const float MAGIC = 12582912.f;   // 1.5 * 2^23: adding and subtracting rounds to nearest-even integer
+
+    for (long long row0 = (long long)blockIdx.x * P.rows_per_cta; row0 < P.n_rows;
+         row0 += (long long)gridDim.x * P.rows_per_cta) {
+        const long long row = row0 + team;
+        const bool active = row < P.n_rows;
+        clear_gmax(P, L.gmax);
+        for (int i = threadIdx.x; i < P.rows_per_cta * GBS_MAX_CANDIDATES; i += NT) row_err_all[i] = 0.f;
+        rotate_row_to_smem<InT>(P, x, row, active, rowbuf, L.hm_s, j, tt);
+        row_group_max(P, rowbuf, gmax, active, j, tt);
+
+        for (int k0 = 0; k0 < K; k0 += KT) {
+            float acc[KT];
+#pragma unroll
+            for (int kk = 0; kk < KT; ++kk) acc[kk] = 0.f;
+            if (active) {
+                for (int ch = j; ch < P.chunks; ch += tt) {
+                    float v[8];
+                    read_chunk_smem(rowbuf, ch, v);
+                    const float M = __uint_as_float(gmax[(ch * 8) / P.G]);
+                    // y / Delta_k = Y * (D / alpha_k) / max|Y| and y = Y * norm, so on y the factor is
+                    // (D / alpha_k) * sM with sM = 1 / (max|Y| * norm)
+                    const float sM = (M > 0.f) ? (1.f / (M * P.norm)) : 0.f;
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) v[e] *= P.norm;          // y = Y / sqrt(d')
+#pragma unroll
+                    for (int kk = 0; kk < KT; ++kk) {
+                        if (k0 + kk < K) {
+                            const float delta = C.c_scale[k0 + kk] * M;   // Delta_k = c_scale_k * max|Y|
+                            const float inv = C.c_inv[k0 + kk] * sM;
+#pragma unroll
+                            for (int e = 0; e < 8; ++e) {
+                                float t = fminf(fmaxf(v[e] * inv, -fD), fD);
+                                float q = (t + MAGIC) - MAGIC;
+                                float err = fmaf(-q, delta, v[e]);
+                                acc[kk] = fmaf(err, err, acc[kk]);
+                            }
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int kk = 0; kk < KT; ++kk) {
+                float a = acc[kk];
+                if (tt >= 32) {
+                    for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(FULL, a, o);
+                    if (active && lane == 0 && k0 + kk < K) atomicAdd(&row_err[k0 + kk], a);
+                } else {
+                    for (int o = tt >> 1; o > 0; o >>= 1) a += __shfl_xor_sync(FULL, a, o);
+                    if (active && j == 0 && k0 + kk < K) row_err[k0 + kk] = a;
+                }
+            }
+        }
+        __syncthreads();
+        // per-row results out, block totals in double
+        for (int i = threadIdx.x; i < P.rows_per_cta * K; i += NT) {
+            const int t = i / K, kx = i - t * K;
+            const long long r = row0 + t;
+            if (r < P.n_rows && err_rows) err_rows[r * K + kx] = row_err_all[t * GBS_MAX_CANDIDATES + kx];
+        }
+        if (threadIdx.x < K) {
+            double s = 0.0;
+            for (int t = 0; t < P.rows_per_cta; ++t)
+                if (row0 + t < P.n_rows) s += (double)row_err_all[t * GBS_MAX_CANDIDATES + threadIdx.x];
+            cta_sum[threadIdx.x] += s;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x < K) atomicAdd(&err_sum[threadIdx.x], cta_sum[threadIdx.x]);
+}
+
+// ======================================================================================
+// dequantize
+// ======================================================================================
+template <int BITS>
+__device__ __forceinline__ void unpack8(const unsigned char* src, float delta, float v[8])
+{
+    unsigned word;
+    if (BITS == 4) word = (unsigned)src[0] | ((unsigned)src[1] << 8) | ((unsigned)src[2] << 16) | ((unsigned)src[3] << 24);
+    else word = (unsigned)src[0] | ((unsigned)src[1] << 8) | ((unsigned)src[2] << 16);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) {
+        int f = (int)((word >> (BITS * e)) & ((1u << BITS) - 1u));
+        f = (f << (32 - BITS)) >> (32 - BITS);    // sign-extend
+        v[e] = (float)f * delta;
+    }
+}
+
+__device__ __forceinline__ void store8(float* dst, const float v[8])
+{
+    reinterpret_cast<float4*>(dst)[0] = make_float4(v[0], v[1], v[2], v[3]);
+    reinterpret_cast<float4*>(dst)[1] = make_float4(v[4], v[5], v[6], v[7]);
+}
+
+__device__ __forceinline__ void store8(__nv_bfloat16* dst, const float v[8])
+{
+    unsigned w[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+        w[e] = *reinterpret_cast<unsigned*>(&h);
+    }
+    *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+__device__ __forceinline__ void store1(float* dst, float v) { *dst = v; }
+__device__ __forceinline__ void store1(__nv_bfloat16* dst, float v) { *dst = __float2bfloat16_rn(v); }
+
+// yhat = q * Delta, rotated domain: pure streaming, one thread per chunk of 8 codes.
+template <typename OutT, int BITS>
+__global__ void __launch_bounds__(NT) k_dequantize_plain(int d_pad, int G, int spr, long long n_chunks,
+                                                         const unsigned char* __restrict__ codes,
+                                                         const float* __restrict__ scales,
+                                                         OutT* __restrict__ out)
+{
+    const int chunks = d_pad >> 3;
+    for (long long g = (long long)blockIdx.x * NT + threadIdx.x; g < n_chunks; g += (long long)gridDim.x * NT) {
+        const long long row = g / chunks;
+        const int ch = (int)(g - row * chunks);
+        const float delta = __ldg(scales + row * spr + (ch * 8) / G);
+        float v[8];
+        unpack8<BITS>(codes + g * BITS, delta, v);
+        store8(out + g * 8, v);
+    }
+}
+
+// xhat = (H^T yhat / sqrt(d'))[0:d]: same shared-memory machinery with the transposed H_m.
+template <typename OutT, int BITS>
+__global__ void __launch_bounds__(NT) k_dequantize_inverse(GenericParams P, const unsigned char* __restrict__ codes,
+                                                           const float* __restrict__ scales,
+                                                           OutT* __restrict__ out)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    SmemLayout L = carve(P, smem);
+    stage_hm(P, L.hm_s);
+    const int tt = 1 << P.tt_log2;
+    const int team = threadIdx.x >> P.tt_log2;
+    const int j = threadIdx.x & (tt - 1);
+    float* rowbuf = L.rowbuf + (size_t)team * P.row_floats;
+
+    for (long long row0 = (long long)blockIdx.x * P.rows_per_cta; row0 < P.n_rows;
+         row0 += (long long)gridDim.x * P.rows_per_cta) {
+        const long long row = row0 + team;
+        const bool active = row < P.n_rows;
+        if (active) {
+            const unsigned char* crow = codes + row * P.row_bytes;
+            for (int ch = j; ch < P.chunks; ch += tt) {
+                float v[8];
+                unpack8<BITS>(crow + ch * BITS, __ldg(scales + row * P.spr + (ch * 8) / P.G), v);
+                butterflies<8>(v);
+                const int p = ch * 8 + (ch >> 2);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) rowbuf[p + e] = v[e];
+            }
+        }
+        run_passes_and_mix(P, rowbuf, L.hm_s, j, tt);
+        if (active) {
+            OutT* orow = out + row * P.d;
+            for (int i = j; i < P.d; i += tt) store1(orow + i, rowbuf[pidx(i)] * P.norm);
+        }
+        __syncthreads();
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------------------
+int ceil_log2(int v)
+{
+    int l = 0;
+    while ((1 << l) < v) ++l;
+    return l;
+}
+
+void fill_params(const gbs_plan* p, GenericParams& P, int64_t n_rows, int64_t stride, bool inverse)
+{
+    P.d = p->d; P.d_pad = p->d_pad; P.k = p->k; P.m = p->m; P.n2 = 1 << p->k;
+    P.group = p->group; P.G = p->group ? p->group : p->d_pad;
+    P.spr = p->group ? p->d_pad / p->group : 1;
+    P.levels = p->levels;
+    P.norm = p->norm; P.c_scale = p->c_scale; P.c_inv = p->c_inv;
+    P.chunks = p->d_pad / 8;
+    int tl = ceil_log2(P.chunks);
+    if (tl > 8) tl = 8;
+    P.tt_log2 = tl;
+    P.rows_per_cta = NT >> tl;
+    if ((P.G & (P.G - 1)) == 0 && P.G <= 256) { P.red_mode = 1; P.seg_lanes = P.G / 8; }
+    else if (P.G % 256 == 0) { P.red_mode = 2; P.seg_lanes = 32; }
+    else { P.red_mode = 3; P.seg_lanes = 1; }
+    P.row_floats = p->d_pad + p->d_pad / 32 + 1;
+    P.row_bytes = p->d_pad * p->bits / 8;
+    P.stage_bytes = (P.row_bytes + 15) & ~15;
+    // butterfly passes over bits 3 .. k-1, at most 4 bits each, split evenly
+    int rem = p->k - 3, np = (rem + 3) / 4, s = 3;
+    P.n_pass = np;
+    for (int i = 0; i < np; ++i) {
+        int r = rem / np + (i < rem % np ? 1 : 0);
+        P.pass_s[i] = s; P.pass_r[i] = r; s += r;
+    }
+    P.n_rows = n_rows; P.stride = stride;
+    P.hm = p->d_hm ? (p->d_hm + (inverse ? p->m * p->m : 0)) : nullptr;
+}
+
+size_t base_smem(const GenericParams& P)
+{
+    size_t off = sizeof(float) * (size_t)P.rows_per_cta * P.row_floats;
+    off += sizeof(unsigned) * (size_t)P.rows_per_cta * P.spr;
+    off = (off + 15) & ~(size_t)15;
+    off += sizeof(float) * (size_t)((P.m > 1) ? P.m * P.m : 0);
+    off = (off + 15) & ~(size_t)15;
+    return off;
+}
+
+int grid_for(const gbs_plan* p, const GenericParams& P, size_t smem)
+{
+    long long need = (P.n_rows + P.rows_per_cta - 1) / P.rows_per_cta;
+    int per_sm = (int)((size_t)(228 * 1024) / (smem + 1024));
+    if (per_sm > 2048 / NT) per_sm = 2048 / NT;
+    if (per_sm < 1) per_sm = 1;
+    long long cap = (long long)p->sm_count * per_sm;
+    return (int)(need < cap ? need : cap);
+}
+
+template <typename KernelT>
+cudaError_t prep(KernelT kernel, size_t smem)
+{
+    if (smem > 48 * 1024)
+        return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    return cudaSuccess;
+}
+
+}  // namespace
+
+size_t gbs_generic_smem_bytes(const gbs_plan* p, int* rows_per_cta)
+{
+    GenericParams P;
+    fill_params(p, P, 0, 0, false);
+    if (rows_per_cta) *rows_per_cta = P.rows_per_cta;
+    size_t rq = base_smem(P) + (size_t)P.rows_per_cta * P.stage_bytes;
+    size_t ce = base_smem(P) + sizeof(double) * GBS_MAX_CANDIDATES +
+                sizeof(float) * (size_t)P.rows_per_cta * GBS_MAX_CANDIDATES;
+    return rq > ce ? rq : ce;
+}
+
+int gbs_generic_rotate_quantize(const gbs_plan* p, const void* x, int x_dtype, int64_t n_rows, int64_t stride,
+                                void* codes, float* scales, float* y_opt, cudaStream_t stream)
+{
+    GenericParams P;
+    fill_params(p, P, n_rows, stride, false);
+    const size_t smem = base_smem(P) + (size_t)P.rows_per_cta * P.stage_bytes;
+    const int grid = grid_for(p, P, smem);
+    cudaError_t e;
+#define LAUNCH_RQ(T, B)                                                                       \
+    do {                                                                                      \
+        e = prep(k_rotate_quantize<T, B>, smem);                                              \
+        if (e == cudaSuccess) {                                                               \
+            k_rotate_quantize<T, B><<<grid, NT, smem, stream>>>(P, (const T*)x, (unsigned char*)codes, scales, y_opt); \
+            e = cudaGetLastError();                                                           \
+        }                                                                                     \
+    } while (0)
+    if (x_dtype == GBS_DTYPE_F32) { if (p->bits == 3) LAUNCH_RQ(float, 3); else LAUNCH_RQ(float, 4); }
+    else { if (p->bits == 3) LAUNCH_RQ(__nv_bfloat16, 3); else LAUNCH_RQ(__nv_bfloat16, 4); }
+#undef LAUNCH_RQ
+    return (int)e;
+}
+
+int gbs_generic_clip_error(const gbs_plan* p, const void* x, int x_dtype, int64_t n_rows, int64_t stride,
+                           const float* c_scale_k, const float* c_inv_k, int K, double* err_sum,
+                           float* err_rows, cudaStream_t stream)
+{
+    GenericParams P;
+    fill_params(p, P, n_rows, stride, false);
+    ClipConsts C;
+    for (int i = 0; i < GBS_MAX_CANDIDATES; ++i) {
+        C.c_scale[i] = i < K ? c_scale_k[i] : 0.f;
+        C.c_inv[i] = i < K ? c_inv_k[i] : 0.f;
+    }
+    const size_t smem = base_smem(P) + sizeof(double) * GBS_MAX_CANDIDATES +
+                       sizeof(float) * (size_t)P.rows_per_cta * GBS_MAX_CANDIDATES;
+    const int grid = grid_for(p, P, smem);
+    cudaError_t e;
+    if (x_dtype == GBS_DTYPE_F32) {
+        e = prep(k_clip_error<float>, smem);
+        if (e == cudaSuccess) {
+            k_clip_error<float><<<grid, NT, smem, stream>>>(P, C, K, (const float*)x, err_sum, err_rows);
+            e = cudaGetLastError();
+        }
+    } else {
+        e = prep(k_clip_error<__nv_bfloat16>, smem);
+        if (e == cudaSuccess) {
+            k_clip_error<__nv_bfloat16><<<grid, NT, smem, stream>>>(P, C, K, (const __nv_bfloat16*)x, err_sum, err_rows);
+            e = cudaGetLastError();
+        }
+    }
+    return (int)e;
+}
+
+int gbs_generic_dequantize(const gbs_plan* p, const void* codes, const float* scales, int64_t n_rows,
+                           void* out, int out_dtype, int inverse, cudaStream_t stream)
+{
+    GenericParams P;
+    fill_params(p, P, n_rows, 0, inverse != 0);
+    cudaError_t e = cudaSuccess;
+    if (!inverse) {
+        const long long n_chunks = (long long)n_rows * P.chunks;
+        long long blocks = (n_chunks + NT - 1) / NT;
+        long long cap = (long long)p->sm_count * 8 * 4;
+        const int grid = (int)(blocks < cap ? blocks : cap);
+#define LAUNCH_DP(T, B)                                                                            \
+    do {                                                                                           \
+        k_dequantize_plain<T, B><<<grid, NT, 0, stream>>>(P.d_pad, P.G, P.spr, n_chunks,            \
+                                                          (const unsigned char*)codes, scales, (T*)out); \
+        e = cudaGetLastError();                                                                    \
+    } while (0)
+        if (out_dtype == GBS_DTYPE_F32) { if (p->bits == 3) LAUNCH_DP(float, 3); else LAUNCH_DP(float, 4); }
+        else { if (p->bits == 3) LAUNCH_DP(__nv_bfloat16, 3); else LAUNCH_DP(__nv_bfloat16, 4); }
+#undef LAUNCH_DP
+        return (int)e;
+    }
+    const size_t smem = base_smem(P);
+    const int grid = grid_for(p, P, smem);
+#define LAUNCH_DI(T, B)                                                                            \
+    do {                                                                                           \
+        e = prep(k_dequantize_inverse<T, B>, smem);                                                \
+        if (e == cudaSuccess) {                                                                    \
+            k_dequantize_inverse<T, B><<<grid, NT, smem, stream>>>(P, (const unsigned char*)codes, scales, (T*)out); \
+            e = cudaGetLastError();                                                                \
+        }                                                                                          \
+    } while (0)
+    if (out_dtype == GBS_DTYPE_F32) { if (p->bits == 3) LAUNCH_DI(float, 3); else LAUNCH_DI(float, 4); }
+    else { if (p->bits == 3) LAUNCH_DI(__nv_bfloat16, 3); else LAUNCH_DI(__nv_bfloat16, 4); }
+#undef LAUNCH_DI
+    return (int)e;
+}

@@ -1,0 +1,216 @@
+// C-ABI entry points: argument validation, plan construction, kernel-family dispatch.
+// Every argument error is caught here, on the host, before anything is launched.
+#include <math.h>
+#include <new>
+#include <stdlib.h>
+#include <string.h>
+
+#include "gbs_internal.h"
+
+namespace {
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int log2_exact(int v)
+{
+    if (v < 1 || (v & (v - 1))) return -1;
+    int l = 0;
+    while ((1 << l) < v) ++l;
+    return l;
+}
+
+bool supported_m(int m) { return m == 1 || m == 12 || m == 20 || m == 24 || m == 28; }
+
+int elem_size(int dtype) { return dtype == GBS_DTYPE_F32 ? 4 : 2; }
+
+// shared validation of (x, dtype, n_rows, stride)
+int check_rows(const gbs_plan* p, const void* x, int x_dtype, int64_t n_rows, int64_t stride)
+{
+    if (!p) return GBS_ERR_INVALID_ARG;
+    if (x_dtype != GBS_DTYPE_F32 && x_dtype != GBS_DTYPE_BF16) return GBS_ERR_INVALID_ARG;
+    if (n_rows < 0) return GBS_ERR_INVALID_ARG;
+    if (n_rows == 0) return GBS_OK;
+    if (!x) return GBS_ERR_INVALID_ARG;
+    if (stride < p->d) return GBS_ERR_INVALID_ARG;
+    if (!aligned16(x) || ((stride * elem_size(x_dtype)) & 15) != 0) return GBS_ERR_ALIGNMENT;
+    return GBS_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool switched = false;
+    cudaError_t enter(int dev)
+    {
+        cudaError_t e = cudaGetDevice(&prev);
+        if (e != cudaSuccess) return e;
+        if (prev != dev) {
+            e = cudaSetDevice(dev);
+            switched = (e == cudaSuccess);
+        }
+        return e;
+    }
+    ~DeviceGuard()
+    {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+extern "C" int gbs_hadamard_m(int m, int8_t* out_host)
+{
+    if (!out_host || m < 1) return GBS_ERR_INVALID_ARG;
+    if (!supported_m(m)) return GBS_ERR_UNSUPPORTED;
+    return gbs_build_hadamard_m(m, out_host);
+}
+
+extern "C" const char* gbs_status_string(int status)
+{
+    switch (status) {
+        case GBS_OK: return "GBS_OK";
+        case GBS_ERR_INVALID_ARG: return "GBS_ERR_INVALID_ARG: argument out of its documented range";
+        case GBS_ERR_UNSUPPORTED: return "GBS_ERR_UNSUPPORTED: no Hadamard construction for this m, or d' too large";
+        case GBS_ERR_ALIGNMENT: return "GBS_ERR_ALIGNMENT: pointer or stride not 16-byte aligned";
+        case GBS_ERR_CUDA: return "GBS_ERR_CUDA: a CUDA runtime call failed";
+        case GBS_ERR_ALLOC: return "GBS_ERR_ALLOC: allocation failed";
+        default: return "GBS: unknown status";
+    }
+}
+
+extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bits, int group, float alpha)
+{
+    if (!out) return GBS_ERR_INVALID_ARG;
+    if (d < 1 || d_pad < d || m < 1) return GBS_ERR_INVALID_ARG;
+    if (bits != 3 && bits != 4) return GBS_ERR_INVALID_ARG;
+    if (!(alpha > 0.f) || !(alpha <= 1.f)) return GBS_ERR_INVALID_ARG;     // also rejects NaN
+    if (d_pad % m != 0) return GBS_ERR_INVALID_ARG;
+    const int k = log2_exact(d_pad / m);
+    if (k < 3) return GBS_ERR_INVALID_ARG;                                  // 2^k >= 8
+    if (group != 0) {
+        if (group < 8 || log2_exact(group) < 0 || (1 << k) % group != 0) return GBS_ERR_INVALID_ARG;
+    }
+    if (!supported_m(m)) return GBS_ERR_UNSUPPORTED;
+    if (d_pad > GBS_MAX_D_PAD) return GBS_ERR_UNSUPPORTED;
+
+    gbs_plan* p = new (std::nothrow) gbs_plan;
+    if (!p) return GBS_ERR_ALLOC;
+    memset(p, 0, sizeof(*p));
+    p->d = d; p->d_pad = d_pad; p->m = m; p->k = k; p->bits = bits; p->group = group; p->alpha = alpha;
+    p->levels = (1 << (bits - 1)) - 1;
+    const double rootn = sqrt((double)d_pad);
+    p->norm = (float)(1.0 / rootn);
+    p->c_scale = (float)((double)alpha / ((double)p->levels * rootn));
+    p->c_inv = (float)((double)p->levels / (double)alpha);
+    p->variant = GBS_VARIANT_GENERIC;
+    int rc = gbs_build_hadamard_m(m, p->h_hm);
+    if (rc != GBS_OK) { delete p; return rc; }
+
+    cudaError_t e = cudaGetDevice(&p->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, p->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, p->device);
+    if (e != cudaSuccess) { cudaGetLastError(); delete p; return GBS_ERR_CUDA; }
+
+    if (gbs_generic_smem_bytes(p, nullptr) > (size_t)p->smem_optin) { delete p; return GBS_ERR_UNSUPPORTED; }
+
+    if (m > 1) {
+        float h[2 * 32 * 32];
+        for (int i = 0; i < m; ++i)
+            for (int j = 0; j < m; ++j) {
+                h[i * m + j] = (float)p->h_hm[i * m + j];
+                h[m * m + j * m + i] = (float)p->h_hm[i * m + j];     // transpose, for the inverse rotation
+            }
+        e = cudaMalloc(&p->d_hm, sizeof(float) * 2 * m * m);
+        if (e != cudaSuccess) { cudaGetLastError(); delete p; return GBS_ERR_ALLOC; }
+        e = cudaMemcpy(p->d_hm, h, sizeof(float) * 2 * m * m, cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) { cudaGetLastError(); cudaFree(p->d_hm); delete p; return GBS_ERR_CUDA; }
+    }
+    *out = p;
+    return GBS_OK;
+}
+
+extern "C" int gbs_plan_destroy(gbs_plan_t* plan)
+{
+    if (!plan) return GBS_OK;
+    int rc = GBS_OK;
+    if (plan->d_hm) {
+        DeviceGuard g;
+        if (g.enter(plan->device) != cudaSuccess || cudaFree(plan->d_hm) != cudaSuccess) {
+            cudaGetLastError();
+            rc = GBS_ERR_CUDA;
+        }
+    }
+    delete plan;
+    return rc;
+}
+
+extern "C" int gbs_plan_info(const gbs_plan_t* p, gbs_plan_info_t* out)
+{
+    if (!p || !out) return GBS_ERR_INVALID_ARG;
+    out->d = p->d; out->d_pad = p->d_pad; out->m = p->m; out->k = p->k;
+    out->bits = p->bits; out->group = p->group; out->alpha = p->alpha;
+    out->levels = p->levels; out->q_lo = -p->levels; out->q_hi = p->levels;
+    out->code_bytes_per_row = (int64_t)p->d_pad * p->bits / 8;
+    out->scales_per_row = p->group ? p->d_pad / p->group : 1;
+    out->variant = p->variant;
+    return GBS_OK;
+}
+
+extern "C" int gbs_rotate_quantize(const gbs_plan_t* p, const void* x, int x_dtype, int64_t n_rows,
+                                   int64_t x_row_stride, void* codes, float* scales, float* y_opt,
+                                   void* cuda_stream)
+{
+    int rc = check_rows(p, x, x_dtype, n_rows, x_row_stride);
+    if (rc != GBS_OK || n_rows == 0) return rc;
+    if (!codes || !scales) return GBS_ERR_INVALID_ARG;
+    if (!aligned16(codes) || (y_opt && !aligned16(y_opt)) || (reinterpret_cast<uintptr_t>(scales) & 3u))
+        return GBS_ERR_ALIGNMENT;
+    DeviceGuard g;
+    if (g.enter(p->device) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
+    int e = gbs_generic_rotate_quantize(p, x, x_dtype, n_rows, x_row_stride, codes, scales, y_opt,
+                                        static_cast<cudaStream_t>(cuda_stream));
+    return e == 0 ? GBS_OK : GBS_ERR_CUDA;
+}
+
+extern "C" int gbs_dequantize(const gbs_plan_t* p, const void* codes, const float* scales, int64_t n_rows,
+                              void* out, int out_dtype, int flags, void* cuda_stream)
+{
+    if (!p) return GBS_ERR_INVALID_ARG;
+    if (out_dtype != GBS_DTYPE_F32 && out_dtype != GBS_DTYPE_BF16) return GBS_ERR_INVALID_ARG;
+    if (flags & ~GBS_INVERSE_ROTATE) return GBS_ERR_INVALID_ARG;
+    if (n_rows < 0) return GBS_ERR_INVALID_ARG;
+    if (n_rows == 0) return GBS_OK;
+    if (!codes || !scales || !out) return GBS_ERR_INVALID_ARG;
+    if (!aligned16(codes) || !aligned16(out) || (reinterpret_cast<uintptr_t>(scales) & 3u))
+        return GBS_ERR_ALIGNMENT;
+    DeviceGuard g;
+    if (g.enter(p->device) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
+    int e = gbs_generic_dequantize(p, codes, scales, n_rows, out, out_dtype, (flags & GBS_INVERSE_ROTATE) != 0,
+                                   static_cast<cudaStream_t>(cuda_stream));
+    return e == 0 ? GBS_OK : GBS_ERR_CUDA;
+}
+
+extern "C" int gbs_clip_error(const gbs_plan_t* p, const void* x, int x_dtype, int64_t n_rows,
+                              int64_t x_row_stride, const float* alphas_host, int K, double* err_sum,
+                              float* err_rows_opt, void* cuda_stream)
+{
+    int rc = check_rows(p, x, x_dtype, n_rows, x_row_stride);
+    if (rc != GBS_OK) return rc;
+    if (K < 1 || K > GBS_MAX_CANDIDATES || !alphas_host) return GBS_ERR_INVALID_ARG;
+    float c_scale[GBS_MAX_CANDIDATES], c_inv[GBS_MAX_CANDIDATES];
+    const double rootn = sqrt((double)p->d_pad);
+    for (int i = 0; i < K; ++i) {
+        const float a = alphas_host[i];
+        if (!(a > 0.f) || !(a <= 1.f)) return GBS_ERR_INVALID_ARG;
+        c_scale[i] = (float)((double)a / ((double)p->levels * rootn));
+        c_inv[i] = (float)((double)p->levels / (double)a);
+    }
+    if (n_rows == 0) return GBS_OK;
+    if (!err_sum) return GBS_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(err_sum) & 7u) || (err_rows_opt && (reinterpret_cast<uintptr_t>(err_rows_opt) & 3u)))
+        return GBS_ERR_ALIGNMENT;
+    DeviceGuard g;
+    if (g.enter(p->device) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
+    int e = gbs_generic_clip_error(p, x, x_dtype, n_rows, x_row_stride, c_scale, c_inv, K, err_sum, err_rows_opt,
+                                   static_cast<cudaStream_t>(cuda_stream));
+    return e == 0 ? GBS_OK : GBS_ERR_CUDA;
+}

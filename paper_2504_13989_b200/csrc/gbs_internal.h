@@ -1,0 +1,42 @@
+// Internal declarations shared by the translation units of libgbs (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "gbs.h"
+
+// Kernel families a plan can select for bf16 rows.
+enum gbs_variant {
+    GBS_VARIANT_GENERIC = 0,   // shared-memory FWHT on the plain ALUs; any supported (m, k), any dtype
+};
+
+struct gbs_plan {
+    int d, d_pad, m, k;
+    int bits, group;
+    float alpha;
+    int levels;            // D
+    float norm;            // 1/sqrt(d')
+    float c_scale;         // alpha / (D sqrt(d')):  Delta = c_scale * max|Y|   (Y = unnormalised rotation)
+    float c_inv;           // D / alpha:             code  = rint(Y * c_inv / max|Y|)
+    int device;
+    int sm_count;
+    int smem_optin;        // largest dynamic shared memory a block may opt in to
+    int variant;
+    float* d_hm;           // device: H_m as floats, m*m row-major, followed by H_m^T (m*m)
+    int8_t h_hm[32 * 32];  // host copy of H_m (m <= 32)
+};
+
+// gbs_paley.cu
+int gbs_build_hadamard_m(int m, int8_t* out);   // 0 or GBS_ERR_UNSUPPORTED
+
+// gbs_generic.cu : launches on `stream`; return a cudaError_t cast to int (0 = success)
+int gbs_generic_rotate_quantize(const gbs_plan* p, const void* x, int x_dtype, int64_t n_rows,
+                                int64_t stride, void* codes, float* scales, float* y_opt,
+                                cudaStream_t stream);
+int gbs_generic_clip_error(const gbs_plan* p, const void* x, int x_dtype, int64_t n_rows,
+                           int64_t stride, const float* c_scale_k, const float* c_inv_k, int K,
+                           double* err_sum, float* err_rows, cudaStream_t stream);
+int gbs_generic_dequantize(const gbs_plan* p, const void* codes, const float* scales, int64_t n_rows,
+                           void* out, int out_dtype, int inverse, cudaStream_t stream);
+size_t gbs_generic_smem_bytes(const gbs_plan* p, int* rows_per_cta);

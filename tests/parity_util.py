@@ -1,0 +1,72 @@
+"""Helpers for the GPU-vs-oracle parity tests.  The tolerances are the ones the task fixes:
+rotated fp32 values within 1e-5 relative L2 per row, scales within 1e-6 relative, integer codes
+identical except at rounding ties (mismatch fraction <= 1e-4, never more than one level),
+clip-error sums within 1e-5 relative."""
+import numpy as np
+import torch
+
+import oracle
+from paper_2504_13989_b200 import synth
+
+TOL_ROT_L2 = 1e-5
+TOL_SCALE = 1e-6
+TOL_CODE_FRAC = 1e-4
+TOL_CLIP = 1e-5
+
+
+def unpack_codes(buf: np.ndarray, n: int, bits: int) -> np.ndarray:
+    """Vectorised unpack of the little-endian bit stream (written independently of both sides)."""
+    buf = np.ascontiguousarray(buf, dtype=np.uint8)
+    rows = buf.shape[0]
+    bitsarr = np.unpackbits(buf, axis=1, bitorder="little")[:, : n * bits].reshape(rows, n, bits)
+    weights = (1 << np.arange(bits)).astype(np.int32)
+    f = (bitsarr.astype(np.int32) * weights).sum(axis=2)
+    return np.where(f >= (1 << (bits - 1)), f - (1 << bits), f).astype(np.int32)
+
+
+def compare_rotate_quantize(x: torch.Tensor, ref: dict, codes: torch.Tensor, scales: torch.Tensor,
+                            y: torch.Tensor | None, bits: int, group: int, d_pad: int, alpha: float = None):
+    """Assert the four parity conditions; returns a dict of the measured statistics."""
+    stats = {}
+    n = ref["delta"].shape[0]
+    if y is not None:
+        yg = y.detach().cpu().to(torch.float64).numpy()
+        num = np.linalg.norm(yg - ref["y"], axis=1)
+        den = np.linalg.norm(ref["y"], axis=1)
+        rel = np.where(den > 0, num / np.where(den > 0, den, 1), num)
+        stats["rot_rel_l2_max"] = float(rel.max()) if n else 0.0
+        assert np.all(rel <= TOL_ROT_L2), "rotated values: max rel L2 %.3e" % rel.max()
+    sg = scales.detach().cpu().to(torch.float64).numpy().reshape(ref["delta"].shape)
+    dref = ref["delta"]
+    srel = np.abs(sg - dref) / np.where(dref > 0, dref, 1.0)
+    stats["scale_rel_max"] = float(srel.max()) if n else 0.0
+    assert np.all(srel <= TOL_SCALE), "scales: max rel err %.3e" % srel.max()
+    assert np.all(sg[dref == 0] == 0)
+    qg = unpack_codes(codes.detach().cpu().numpy().reshape(n, -1), d_pad, bits)
+    D = 2 ** (bits - 1) - 1
+    assert qg.min(initial=0) >= -D and qg.max(initial=0) <= D, "code outside [-D, D]"
+    diff = qg != ref["q"]
+    frac = diff.mean() if diff.size else 0.0
+    stats["code_mismatch_frac"] = float(frac)
+    assert frac <= TOL_CODE_FRAC, "codes: mismatch fraction %.3e" % frac
+    if diff.any():
+        assert np.abs(qg - ref["q"])[diff].max() <= 1, "a code differs by more than one level"
+        # every mismatch must sit at a rounding tie of the oracle's own y / Delta
+        g = group or d_pad
+        dl = np.repeat(ref["delta"], g, axis=1)
+        t = ref["y"][diff] / dl[diff]
+        dist = np.abs(np.abs(t - np.floor(t)) - 0.5)
+        clip_edge = np.abs(np.abs(t) - (D + 0.5))     # |t| just around D+0.5 is also a tie (then clamped)
+        stats["tie_dist_max"] = float(dist.max())
+        assert np.all((dist < 2e-4) | (clip_edge < 2e-4)), "a mismatching code is not at a rounding tie"
+    return stats
+
+
+def oracle_rq(x: torch.Tensor, w_or_plan, bits: int, dense: bool = False, alpha: float = None, group: int = None):
+    if isinstance(w_or_plan, synth.Workload):
+        d, d_pad, m = w_or_plan.d, w_or_plan.d_pad, w_or_plan.m
+        alpha = w_or_plan.alpha if alpha is None else alpha
+        group = w_or_plan.group if group is None else group
+    else:
+        d, d_pad, m = w_or_plan
+    return oracle.rotate_quantize_rows(synth.to_oracle_array(x), d, d_pad, m, bits, group, alpha, dense=dense)

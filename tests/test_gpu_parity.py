@@ -1,0 +1,261 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the float64 CPU oracle on the same
+seeded inputs, element by element."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2504_13989_b200 import Plan, binding, synth
+from paper_2504_13989_b200 import build as gbs_build
+from parity_util import (TOL_CLIP, TOL_ROT_L2, compare_rotate_quantize, oracle_rq, unpack_codes)
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    gbs_build.build()
+    binding.lib()
+
+
+def _guarded(n_bytes, dtype, device=DEV, guard=256):
+    """Buffer with sentinel guard bands on both sides; returns (view, checker)."""
+    item = torch.empty((), dtype=dtype).element_size()
+    total = n_bytes + 2 * guard
+    raw = torch.full((total,), 0xA5, dtype=torch.uint8, device=device)
+    view = raw[guard:guard + n_bytes].view(dtype) if n_bytes else raw[guard:guard].view(dtype)
+
+    def check():
+        r = raw.cpu()
+        assert bool((r[:guard] == 0xA5).all()) and bool((r[guard + n_bytes:] == 0xA5).all()), "guard band overwritten"
+    return view, check, item
+
+
+def _run_rq(plan: Plan, x_dev, n_rows, want_y=True):
+    info = plan.info
+    codes, c1, _ = _guarded(n_rows * info.code_bytes_per_row, torch.uint8)
+    scales, c2, _ = _guarded(n_rows * info.scales_per_row * 4, torch.float32)
+    y, c3, _ = _guarded(n_rows * info.d_pad * 4, torch.float32)
+    binding.gbs_rotate_quantize(plan.handle, x_dev, codes, scales, y if want_y else None)
+    torch.cuda.synchronize()
+    c1(); c2(); c3()
+    return (codes.view(n_rows, -1) if n_rows else codes, scales.view(n_rows, -1) if n_rows else scales,
+            y.view(n_rows, info.d_pad) if (want_y and n_rows) else None)
+
+
+# ------------------------------------------------------------------------------------------
+# the tiny configuration, fully, with the dense-definition oracle
+# ------------------------------------------------------------------------------------------
+def test_tiny_config_rotate_quantize_dequantize_clip_error():
+    w = synth.WORKLOADS["tiny"]
+    x = synth.make_host("tiny")
+    ref = oracle_rq(x, w, 4, dense=True)
+    with Plan(w.d, w.d_pad, w.m, 4, w.group, w.alpha) as plan:
+        codes, scales, y = _run_rq(plan, x.to(DEV), w.n_rows)
+        compare_rotate_quantize(x, ref, codes, scales, y, 4, w.group, w.d_pad)
+        # dequantize (rotated domain) and inverse rotation
+        yhat = plan.dequantize(codes, scales)
+        want = oracle.dequantize_rows(codes.cpu().numpy(), scales.cpu().double().numpy(), w.d, w.d_pad, w.m, 4, w.group)
+        np.testing.assert_allclose(yhat.cpu().double().numpy(), want, rtol=2e-7, atol=0)
+        xhat = plan.dequantize(codes, scales, inverse=True)
+        wantx = oracle.dequantize_rows(codes.cpu().numpy(), scales.cpu().double().numpy(), w.d, w.d_pad, w.m, 4,
+                                       w.group, inverse=True)
+        rel = np.linalg.norm(xhat.cpu().double().numpy() - wantx, axis=1) / np.linalg.norm(wantx, axis=1)
+        assert rel.max() <= TOL_ROT_L2
+        # clip-error sweep, K = 8 alphas in [0.5, 1]
+        alphas = np.linspace(0.5, 1.0, 8)
+        err, rows = plan.clip_error(x.to(DEV), alphas, want_rows=True)
+        torch.cuda.synchronize()
+        eref, rref = oracle.clip_error_rows(synth.to_oracle_array(x), w.d, w.d_pad, w.m, 4, w.group, alphas,
+                                            want_rows=True)
+        np.testing.assert_allclose(err.cpu().numpy(), eref, rtol=TOL_CLIP)
+        np.testing.assert_allclose(rows.cpu().double().numpy(), rref, rtol=1e-4)
+        # accumulation semantics: a second call adds to err_sum
+        plan.clip_error(x.to(DEV), alphas, err_sum=err)
+        torch.cuda.synchronize()
+        np.testing.assert_allclose(err.cpu().numpy(), 2 * eref, rtol=TOL_CLIP)
+
+
+def test_literal_formula_at_b3_is_the_4bit_plan():
+    """Delta = max|X| / (2^b - 1) exactly as printed (Section 2.1) at b = 3 is D = 7: the bits = 4 plan."""
+    w = synth.WORKLOADS["tiny"]
+    x = synth.make_host("tiny")
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(x), w.d, w.d_pad, w.m, 3, 0, 1.0, literal=True, dense=True)
+    with Plan(w.d, w.d_pad, 1, 4, 0, 1.0) as plan:
+        codes, scales, y = _run_rq(plan, x.to(DEV), w.n_rows)
+        compare_rotate_quantize(x, ref, codes, scales, y, 4, 0, w.d_pad)
+
+
+# ------------------------------------------------------------------------------------------
+# reduced-size versions of every workload: several tiles and a ragged tail
+# ------------------------------------------------------------------------------------------
+CASES = [
+    # name, rows, bits
+    ("llama4096", 301, 3), ("llama4096", 301, 4),
+    ("qwen3584", 203, 3),
+    ("mlp18944", 37, 4),
+    ("kv128", 4099, 3),
+    ("calib4096", 150, 3),
+]
+
+
+@pytest.mark.parametrize("name,rows,bits", CASES)
+def test_workload_parity_reduced(name, rows, bits):
+    w = synth.WORKLOADS[name]
+    x = synth.make_host(name, rows)
+    ref = oracle_rq(x, w, bits)
+    with Plan(w.d, w.d_pad, w.m, bits, w.group, w.alpha) as plan:
+        codes, scales, y = _run_rq(plan, x.to(DEV), rows)
+        stats = compare_rotate_quantize(x, ref, codes, scales, y, bits, w.group, w.d_pad)
+        print(name, bits, stats)
+        # same call without the optional rotated output must give identical codes and scales
+        codes2, scales2, _ = _run_rq(plan, x.to(DEV), rows, want_y=False)
+        assert torch.equal(codes, codes2) and torch.equal(scales, scales2)
+        # dequantize of the GPU's own codes against the oracle's dequantize of the same bytes
+        sc64 = scales.cpu().double().numpy()
+        yhat = plan.dequantize(codes, scales)
+        want = oracle.dequantize_rows(codes.cpu().numpy(), sc64, w.d, w.d_pad, w.m, bits, w.group)
+        np.testing.assert_allclose(yhat.cpu().double().numpy(), want, rtol=2e-7, atol=0)
+        yhat16 = plan.dequantize(codes, scales, dtype=torch.bfloat16)
+        np.testing.assert_allclose(yhat16.cpu().double().numpy(), want, rtol=2 ** -8, atol=0)
+        xhat = plan.dequantize(codes, scales, inverse=True)
+        wantx = oracle.dequantize_rows(codes.cpu().numpy(), sc64, w.d, w.d_pad, w.m, bits, w.group, inverse=True)
+        num = np.linalg.norm(xhat.cpu().double().numpy() - wantx, axis=1)
+        den = np.linalg.norm(wantx, axis=1)
+        assert np.all(num <= TOL_ROT_L2 * den + 1e-30)
+        # clip error
+        K = 5
+        alphas = np.linspace(0.5, 1.0, K)
+        err, erows = plan.clip_error(x.to(DEV), alphas, want_rows=True)
+        torch.cuda.synchronize()
+        eref, rref = oracle.clip_error_rows(synth.to_oracle_array(x), w.d, w.d_pad, w.m, bits, w.group, alphas,
+                                            want_rows=True)
+        np.testing.assert_allclose(err.cpu().numpy(), eref, rtol=TOL_CLIP)
+        np.testing.assert_allclose(erows.cpu().double().numpy(), rref, rtol=1e-4, atol=1e-12)
+
+
+# ------------------------------------------------------------------------------------------
+# shapes: every supported m, small and large k, groups, padding, strides
+# ------------------------------------------------------------------------------------------
+SHAPES = [
+    # d, d_pad, m, bits, group, alpha, rows, dtype
+    (8, 8, 1, 3, 0, 1.0, 5, torch.float32),
+    (8, 8, 1, 4, 8, 0.7, 300, torch.bfloat16),
+    (13, 16, 1, 3, 0, 0.9, 33, torch.bfloat16),
+    (16, 16, 1, 4, 8, 1.0, 257, torch.float32),
+    (32, 32, 1, 3, 16, 0.8, 149, torch.bfloat16),
+    (64, 64, 1, 4, 0, 0.95, 147, torch.float32),
+    (96, 96, 12, 3, 0, 0.9, 21, torch.bfloat16),
+    (90, 96, 12, 4, 8, 0.9, 22, torch.float32),
+    (160, 160, 20, 3, 8, 1.0, 13, torch.bfloat16),
+    (192, 192, 24, 4, 0, 0.85, 17, torch.bfloat16),
+    (224, 224, 28, 3, 8, 0.6, 19, torch.float32),
+    (300, 384, 12, 3, 32, 0.9, 9, torch.bfloat16),
+    (256, 256, 1, 3, 256, 0.9, 64, torch.bfloat16),
+    (1024, 1024, 1, 4, 64, 0.5, 31, torch.bfloat16),
+    (1000, 1024, 1, 3, 0, 0.3, 31, torch.float32),
+    (2048, 2048, 1, 3, 512, 0.9, 12, torch.bfloat16),
+    (1536, 1536, 24, 4, 64, 0.9, 40, torch.bfloat16),
+    (1536, 1536, 12, 3, 128, 0.9, 40, torch.bfloat16),
+    (3584, 3584, 28, 4, 0, 0.9, 10, torch.float32),
+    (8192, 8192, 1, 3, 0, 0.9, 7, torch.bfloat16),
+    (30000, 32768, 1, 4, 1024, 0.9, 3, torch.bfloat16),
+    (32768, 32768, 1, 3, 0, 1.0, 2, torch.float32),
+    (20480, 20480, 20, 3, 1024, 0.9, 3, torch.bfloat16),
+    (28672, 28672, 28, 4, 0, 0.9, 2, torch.bfloat16),
+]
+
+
+@pytest.mark.parametrize("d,d_pad,m,bits,group,alpha,rows,dtype", SHAPES)
+def test_shape_sweep(d, d_pad, m, bits, group, alpha, rows, dtype):
+    rng = np.random.Generator(np.random.PCG64(d * 7 + m * 3 + bits))
+    xs = rng.standard_t(3, size=(rows, d))
+    xs[:, rng.integers(0, d, 2)] *= 30
+    if rows > 2:
+        xs[1, :] = 0.0                      # an all-zero row: codes 0, scale 0
+    x = torch.from_numpy(xs.astype(np.float32)).to(dtype)
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(x), d, d_pad, m, bits, group, alpha,
+                                      dense=(d_pad <= 2048))
+    with Plan(d, d_pad, m, bits, group, alpha) as plan:
+        codes, scales, y = _run_rq(plan, x.to(DEV), rows)
+        compare_rotate_quantize(x, ref, codes, scales, y, bits, group, d_pad)
+        if rows > 2:
+            assert int(codes[1].max()) == 0 and float(scales[1].abs().max()) == 0.0
+        alphas = [1.0, 0.8, 0.45]
+        err = plan.clip_error(x.to(DEV), alphas)
+        torch.cuda.synchronize()
+        eref = oracle.clip_error_rows(synth.to_oracle_array(x), d, d_pad, m, bits, group, np.array(alphas))
+        np.testing.assert_allclose(err.cpu().numpy(), eref, rtol=TOL_CLIP)
+        xhat = plan.dequantize(codes, scales, inverse=True)
+        wantx = oracle.dequantize_rows(codes.cpu().numpy(), scales.cpu().double().numpy(), d, d_pad, m, bits,
+                                       group, inverse=True)
+        num = np.linalg.norm(xhat.cpu().double().numpy() - wantx, axis=1)
+        den = np.linalg.norm(wantx, axis=1)
+        assert np.all(num <= TOL_ROT_L2 * den + 1e-30)
+
+
+def test_strided_rows_and_leading_dims():
+    """x_row_stride > d (a slice of a wider buffer) and KV-style [batch, heads, seq, 128] views."""
+    rng = np.random.Generator(np.random.PCG64(99))
+    big = torch.from_numpy(rng.standard_normal((50, 512)).astype(np.float32)).to(torch.bfloat16)
+    x = big[:, :256]
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(big), 256, 256, 1, 4, 0, 0.9)
+    with Plan(256, 256, 1, 4, 0, 0.9) as plan:
+        xd = big.to(DEV)[:, :256]
+        assert xd.stride(0) == 512
+        codes, scales, y = _run_rq(plan, xd, 50)
+        compare_rotate_quantize(x, ref, codes, scales, y, 4, 0, 256)
+    kv = torch.from_numpy(rng.standard_t(3, size=(2, 3, 17, 128)).astype(np.float32)).to(torch.bfloat16)
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(kv.reshape(-1, 128)), 128, 128, 1, 3, 0, 1.0)
+    with Plan(128, 128, 1, 3, 0, 1.0) as plan:
+        codes, scales, y = _run_rq(plan, kv.to(DEV), 2 * 3 * 17)
+        compare_rotate_quantize(kv.reshape(-1, 128), ref, codes, scales, y, 3, 0, 128)
+
+
+def test_empty_and_error_paths_on_device():
+    with Plan(128, 128, 1, 4, 0, 1.0) as plan:
+        x = torch.zeros((0, 128), dtype=torch.bfloat16, device=DEV)
+        codes, scales, _ = plan.alloc_outputs(0, DEV)
+        binding.gbs_rotate_quantize(plan.handle, x, codes, scales)          # n_rows = 0: no-op
+        L = binding.lib()
+        xb = torch.zeros((4, 136), dtype=torch.bfloat16, device=DEV)
+        c, s, _ = plan.alloc_outputs(4, DEV)
+        h = plan.handle
+        import ctypes
+        vp = ctypes.c_void_p
+        # misaligned base pointer / stride not a multiple of 16 bytes / stride < d / bad dtype / bad K
+        assert L.gbs_rotate_quantize(vp(h), xb.data_ptr() + 2, 1, 4, 136, c.data_ptr(), s.data_ptr(), None, None) == binding.GBS_ERR_ALIGNMENT
+        assert L.gbs_rotate_quantize(vp(h), xb.data_ptr(), 1, 4, 130, c.data_ptr(), s.data_ptr(), None, None) == binding.GBS_ERR_ALIGNMENT
+        assert L.gbs_rotate_quantize(vp(h), xb.data_ptr(), 1, 4, 64, c.data_ptr(), s.data_ptr(), None, None) == binding.GBS_ERR_INVALID_ARG
+        assert L.gbs_rotate_quantize(vp(h), xb.data_ptr(), 7, 4, 136, c.data_ptr(), s.data_ptr(), None, None) == binding.GBS_ERR_INVALID_ARG
+        assert L.gbs_rotate_quantize(vp(h), xb.data_ptr(), 1, -1, 136, c.data_ptr(), s.data_ptr(), None, None) == binding.GBS_ERR_INVALID_ARG
+        assert L.gbs_rotate_quantize(vp(h), xb.data_ptr(), 1, 4, 136, None, s.data_ptr(), None, None) == binding.GBS_ERR_INVALID_ARG
+        err = torch.zeros(4, dtype=torch.float64, device=DEV)
+        a = (ctypes.c_float * 3)(0.5, 1.2, 0.9)
+        assert L.gbs_clip_error(vp(h), xb.data_ptr(), 1, 4, 136, a, 3, err.data_ptr(), None, None) == binding.GBS_ERR_INVALID_ARG
+        assert L.gbs_clip_error(vp(h), xb.data_ptr(), 1, 4, 136, a, 0, err.data_ptr(), None, None) == binding.GBS_ERR_INVALID_ARG
+        assert L.gbs_clip_error(vp(h), xb.data_ptr(), 1, 4, 136, a, 65, err.data_ptr(), None, None) == binding.GBS_ERR_INVALID_ARG
+        assert L.gbs_dequantize(vp(h), c.data_ptr(), s.data_ptr(), 4, xb.data_ptr(), 0, 2, None) == binding.GBS_ERR_INVALID_ARG
+        torch.cuda.synchronize()            # the context is still healthy
+        assert float(err.sum()) == 0.0
+
+
+def test_quantizer_invariants_on_device():
+    """Properties that hold at any size: alpha = 1 reproduces the max (Section 2.1); the norm is preserved
+    (Section 2.3.1); Lemma 1 for a single spike."""
+    n, d = 64, 4096
+    x = synth.make_host("llama4096", n)
+    with Plan(d, d, 1, 4, 0, 1.0) as plan:
+        codes, scales, y = _run_rq(plan, x.to(DEV), n)
+        yn = y.double().norm(dim=1).cpu()
+        xn = x.double().norm(dim=1)
+        assert torch.all((yn - xn).abs() <= 1e-5 * xn)
+        q = unpack_codes(codes.cpu().numpy(), d, 4)
+        assert np.all(np.abs(q).max(axis=1) == 7)
+        amax = y.abs().max(dim=1).values.cpu().double()
+        np.testing.assert_allclose((scales[:, 0].cpu().double() * 7).numpy(), amax.numpy(), rtol=3e-7)
+        spike = torch.zeros((3, d), dtype=torch.float32)
+        spike[0, 0] = 200.0; spike[1, 1777] = 200.0; spike[2, d - 1] = -200.0
+        _, _, ys = _run_rq(plan, spike.to(DEV), 3)
+        np.testing.assert_allclose(ys.abs().cpu().numpy(), 200.0 / 64.0, rtol=1e-6)
