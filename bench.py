@@ -1,0 +1,454 @@
+#!/usr/bin/env python
+"""Benchmark of the fused rotate-and-quantize hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One STEP = one pass of the fused path over one batch of the headline workload: the 4096-token x
+d=4096 bf16 activation batch, quantized at b=3 and at b=4 (two launches of the fused kernel, as the
+workload names both bit-widths).  Inputs are synthetic, resident in HBM before the timed region; the
+launches rotate over NSETS distinct buffer sets whose footprint exceeds 4x the L2 so every launch
+reads from HBM.  The timed K steps are replayed from CUDA graphs, bracketed by a barrier and a
+device synchronise, timed with CUDA events on the launching stream, max over ranks.
+
+Prints ONE JSON line.  `value` is GB/s of algorithmic bytes (row in, packed codes + scales out).
+Extra keys: `roofline`, `cpu_baseline`, `e2e`, `clocks`, `gpu_launches`, and `also` (the d=3584
+workload and the other entry points, timed outside the K steps, for context).
+
+The path does not shard: with --gpus N every rank runs an independent replica on its own GPU.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "rotate+quantize GB/s and Mtokens/s at d=4096/3584, % of B200 HBM peak"
+HEADLINE = "llama4096"
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused kernel on the headline
+# workload, from the ncu capture summarised under profiles/ (None until a capture exists).
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+
+
+def algorithmic_bytes(n_rows: int, d: int, d_pad: int, bits: int, group: int, in_bytes: int) -> int:
+    """Bytes the method must move per launch: the row in, packed codes and scales out."""
+    spr = d_pad // group if group else 1
+    return n_rows * (d * in_bytes + d_pad * bits // 8 + 4 * spr)
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def aggregate(local_ms: float, local_units: float, dist_ok: bool, device=None):
+    """Whole-job figures: time = max over ranks, units = sum over ranks (replicas are independent)."""
+    if not dist_ok:
+        return local_ms, local_units
+    import torch.distributed as dist
+    t = torch.tensor([local_ms], dtype=torch.float64, device=device)
+    u = torch.tensor([local_units], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while the benchmark runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.timed = [], []
+        self.in_timed = False
+        self._stop_evt = threading.Event()
+        self.max_mhz = None
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+            phys = index
+            if vis:
+                ids = [v for v in vis.split(",") if v.strip() != ""]
+                if index < len(ids) and ids[index].strip().isdigit():
+                    phys = int(ids[index])
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(phys)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        while not self._stop_evt.is_set():
+            try:
+                mhz = nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)
+                reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                util = nv.nvmlDeviceGetUtilizationRates(self.h).gpu
+                rec = (mhz, int(reasons), util)
+                self.samples.append(rec)
+                if self.in_timed:
+                    self.timed.append(rec)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+
+    def summary(self):
+        if not self.ok or not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        nv = self.nv
+        pool = self.timed if len(self.timed) >= 3 else [s for s in self.samples if s[2] > 0] or self.samples
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        seen = [n for n, bit in names.items() if any(s[1] & bit for s in pool)]
+        return {"sm_mhz": statistics.median(s[0] for s in pool), "sm_max_mhz": self.max_mhz,
+                "reasons": seen, "samples": len(pool),
+                "window": "timed" if pool is self.timed else "under_load"}
+
+
+def time_oracle(x_host, w, bits_list, min_seconds: float, nthreads: int = 0):
+    """Time the float64 CPU oracle (as it stands) on whole-batch steps for about min_seconds."""
+    import oracle
+    from paper_2504_13989_b200 import synth
+    xa = synth.to_oracle_array(x_host)
+    steps, t0 = 0, time.perf_counter()
+    while True:
+        for b in bits_list:
+            oracle.rotate_quantize_rows(xa, w.d, w.d_pad, w.m, b, w.group, w.alpha, dense=False,
+                                        want_y=False, want_q=False, want_packed=True, nthreads=nthreads)
+        steps += 1
+        el = time.perf_counter() - t0
+        if el >= min_seconds:
+            return steps, el
+
+
+def run_reference(args, rank: int):
+    """Reference arm: the CPU oracle, as it stands, on the host cores (rank 0 only).
+
+    Each step is a bounded sample of the headline batch: the first `rows` token rows, quantized at
+    b=3 and b=4.  `rows` is sized from a short calibration so that K + W steps end within about two
+    minutes; the reported rate does not depend on it.
+    """
+    if rank != 0:
+        return
+    import oracle
+    from paper_2504_13989_b200 import synth
+    w = synth.WORKLOADS[HEADLINE]
+    cores = oracle.max_threads()
+    x_full = synth.make_host(HEADLINE, 1024)
+
+    def one_step(xa):
+        for b in w.bits:
+            oracle.rotate_quantize_rows(xa, w.d, w.d_pad, w.m, b, w.group, w.alpha,
+                                        dense=False, want_y=False, want_q=False, want_packed=True)
+    probe = synth.to_oracle_array(x_full[:128])
+    one_step(probe)
+    t0 = time.perf_counter()
+    one_step(probe)
+    per_row = (time.perf_counter() - t0) / 128
+    budget = 120.0
+    rows = int(budget / ((args.steps + args.warmup) * per_row))
+    rows = max(8, min(1024, rows))
+    xa = synth.to_oracle_array(x_full[:rows])
+    step_bytes = sum(algorithmic_bytes(rows, w.d, w.d_pad, b, w.group, 2) for b in w.bits)
+    for _ in range(args.warmup):
+        one_step(xa)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        one_step(xa)
+    el = time.perf_counter() - t0
+    ms = el * 1e3 / args.steps
+    gbs = step_bytes / (ms * 1e-3) / 1e9
+    sample = "first %d of %d rows of the batch per step, b=3 and b=4, butterfly rotation, OpenMP over rows" % (
+        rows, w.n_rows)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": "%s: %d of %d tokens x d=%d bf16, b=3 and b=4, per-token, alpha=%.2f" %
+                   (HEADLINE, rows, w.n_rows, w.d, w.alpha)},
+        "mtokens_per_s": len(w.bits) * rows / (ms * 1e-3) / 1e6,
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def build_sets(plan_list, x_base, nsets, device):
+    """NSETS distinct input/output buffer sets (inputs are row-rolled copies of the same batch)."""
+    sets = []
+    for i in range(nsets):
+        x = torch.roll(x_base, shifts=i * 17, dims=0).contiguous().to(device)
+        outs = [pl.alloc_outputs(x.shape[0], device) for pl in plan_list]
+        sets.append((x, outs))
+    return sets
+
+
+def run_step(plan_list, st):
+    x, outs = st
+    for pl, o in zip(plan_list, outs):
+        pl.rotate_quantize(x, out=o)
+
+
+def capture(plan_list, sets, idx_list, stream):
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=stream):
+        for i in idx_list:
+            run_step(plan_list, sets[i])
+    return g
+
+
+def timed_graph_loop(plan_list, sets, steps, warmup, stream, dist_ok, sampler=None):
+    """Time exactly `steps` steps replayed from CUDA graphs; returns local milliseconds."""
+    nsets = len(sets)
+    with torch.cuda.stream(stream):
+        for i in range(max(warmup, 3)):
+            run_step(plan_list, sets[i % nsets])
+    stream.synchronize()
+    g_all = capture(plan_list, sets, list(range(nsets)), stream)
+    rem = steps % nsets
+    g_rem = capture(plan_list, sets, list(range(rem)), stream) if rem else None
+    with torch.cuda.stream(stream):
+        g_all.replay()
+    stream.synchronize()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if dist_ok:
+        torch.distributed.barrier()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.in_timed = True
+    with torch.cuda.stream(stream):
+        start.record(stream)
+        for _ in range(steps // nsets):
+            g_all.replay()
+        if g_rem is not None:
+            g_rem.replay()
+        end.record(stream)
+    if dist_ok:
+        torch.distributed.barrier()
+    torch.cuda.synchronize()
+    if sampler:
+        sampler.in_timed = False
+    return start.elapsed_time(end)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--nsets", type=int, default=16)
+    ap.add_argument("--cpu-seconds", type=float, default=10.0)
+    ap.add_argument("--no-extras", action="store_true", help="skip the context legs under `also`")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the product path has no CPU fallback")
+    if args.gpus > 1 and world != args.gpus:
+        raise SystemExit("bench.py: --gpus %d must be launched with torch.distributed.run (WORLD_SIZE=%d)" %
+                         (args.gpus, world))
+    device = torch.device("cuda", local_rank)
+    torch.cuda.set_device(device)
+    dist_ok = world > 1
+    if dist_ok:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    from paper_2504_13989_b200 import Plan, synth
+    from paper_2504_13989_b200 import build as gbs_build
+    gbs_build.build()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+
+    w = synth.WORKLOADS[HEADLINE]
+    x_base = synth.make_host(HEADLINE)                       # seeded; every rank draws the same batch
+    plans = [Plan(w.d, w.d_pad, w.m, b, w.group, w.alpha) for b in w.bits]
+    sets = build_sets(plans, x_base, args.nsets, device)
+    stream = torch.cuda.Stream(device)
+    step_bytes = sum(algorithmic_bytes(w.n_rows, w.d, w.d_pad, b, w.group, 2) for b in w.bits)
+    step_tokens = len(w.bits) * w.n_rows
+    launches_per_step = len(w.bits)
+
+    local_ms = timed_graph_loop(plans, sets, args.steps, args.warmup, stream, dist_ok, sampler)
+    total_ms, total_bytes = aggregate(local_ms, step_bytes * args.steps, dist_ok, device)
+    _, total_tokens = aggregate(local_ms, step_tokens * args.steps, dist_ok, device)
+    ms_per_step = total_ms / args.steps
+    value = total_bytes / (total_ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+
+    # roofline of the fused kernel on this rank: algorithmic bytes per launch / mean launch duration
+    launch_ms = local_ms / (args.steps * launches_per_step)
+    achieved = (step_bytes / launches_per_step) / (launch_ms * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_kind": "of " + peak_kind,
+                "kernel": "fused rotate-quantize, mean of the b=3 and b=4 launches",
+                "frac_of_8000_nominal": achieved / 8000.0}
+
+    # ---- end to end through the public API with host buffers (copies inside the timed region)
+    x_pin = x_base.pin_memory()
+    host_outs = []
+    for pl in plans:
+        host_outs.append((torch.empty((w.n_rows, pl.info.code_bytes_per_row), dtype=torch.uint8).pin_memory(),
+                          torch.empty((w.n_rows, pl.info.scales_per_row), dtype=torch.float32).pin_memory()))
+    e2e_steps = max(3, min(args.steps, 20))
+
+    def e2e_step():
+        with torch.cuda.stream(stream):
+            xd = x_pin.to(device, non_blocking=True)
+            for pl, (ch, sh) in zip(plans, host_outs):
+                c, s, _ = pl.rotate_quantize(xd, stream=stream)
+                ch.copy_(c, non_blocking=True)
+                sh.copy_(s, non_blocking=True)
+    for _ in range(3):
+        e2e_step()
+    stream.synchronize()
+    if dist_ok:
+        torch.distributed.barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(e2e_steps):
+        e2e_step()
+    e1.record(stream)
+    stream.synchronize()
+    e2e_ms_local = e0.elapsed_time(e1)
+    e2e_ms, e2e_bytes = aggregate(e2e_ms_local, step_bytes * e2e_steps, dist_ok, device)
+    h2d = x_pin.numel() * x_pin.element_size()
+    d2h = sum(c.numel() + 4 * s.numel() for c, s in host_outs)
+    e2e = {"value": e2e_bytes / (e2e_ms * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+           "d2h_bytes_per_step": d2h, "steps": e2e_steps, "ms_per_step": e2e_ms / e2e_steps}
+
+    # ---- context legs (outside the K timed steps)
+    also = {}
+    if not args.no_extras and rank == 0:
+        also = extras(device, stream, args, peak)
+
+    sampler.stop()
+    clocks = sampler.summary()
+
+    # ---- the oracle timed beside it, rank 0 at N=1 only
+    cpu_baseline = None
+    if rank == 0 and world == 1 and args.cpu_seconds > 0:
+        import oracle
+        n_steps, el = time_oracle(x_base, w, w.bits, args.cpu_seconds)
+        cpu_baseline = {"value": step_bytes * n_steps / el / 1e9, "unit": "GB/s", "cores": oracle.max_threads(),
+                        "kind": "oracle", "mtokens_per_s": step_tokens * n_steps / el / 1e6,
+                        "sample": "%d whole-batch steps (4096 rows, b=3 and b=4) in %.1f s, butterfly rotation, "
+                                  "OpenMP over rows" % (n_steps, el)}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": "%s: %d tokens x d=%d bf16, H_%d, b=3 and b=4 (one launch each per step), "
+                                   "per-token scales, alpha=%.2f" % (HEADLINE, w.n_rows, w.d, w.d_pad, w.alpha),
+                       "replicas": world, "l2": "inputs rotate over %d buffer sets (%.0f MB > 4x L2)" %
+                       (args.nsets, args.nsets * (step_bytes + w.n_rows * w.d * 2) / 1e6),
+                       "launch": "CUDA graph replay", "levels": "D=2^(b-1)-1"},
+            "mtokens_per_s": total_tokens / (total_ms * 1e-3) / 1e6,
+            "hbm_frac_of_measured": value / world / peak, "hbm_frac_of_8000": value / world / 8000.0,
+            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "clocks": clocks,
+            "gpu_launches": args.steps * launches_per_step, "also": also,
+        }
+        print(json.dumps(line))
+    if dist_ok:
+        torch.distributed.barrier()
+        torch.distributed.destroy_process_group()
+
+
+def extras(device, stream, args, peak):
+    """Context figures for the other workloads / entry points (not part of the K timed steps)."""
+    from paper_2504_13989_b200 import Plan, synth
+    out = {}
+
+    def time_loop(fn, iters):
+        with torch.cuda.stream(stream):
+            for _ in range(3):
+                fn(0)
+        stream.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            a.record(stream)
+            for i in range(iters):
+                fn(i)
+            b.record(stream)
+        stream.synchronize()
+        return a.elapsed_time(b) / iters
+
+    # per-bit figures of the headline workload and the d=3584 workload (graph replay, rotating sets)
+    for name in ("llama4096", "qwen3584"):
+        w = synth.WORKLOADS[name]
+        xb = synth.make_host(name)
+        for b in w.bits:
+            pl = Plan(w.d, w.d_pad, w.m, b, w.group, w.alpha)
+            nbytes = algorithmic_bytes(w.n_rows, w.d, w.d_pad, b, w.group, 2)
+            nsets = max(4, int(4 * 126e6 / (nbytes + 1)) + 1)
+            sets = build_sets([pl], xb, nsets, device)
+            iters = 20 * nsets
+            ms = timed_graph_loop([pl], sets, iters, 3, stream, False) / iters
+            out["%s_b%d" % (name, b)] = {"us_per_launch": ms * 1e3, "gbs": nbytes / ms / 1e6,
+                                         "frac_of_measured": nbytes / ms / 1e6 / peak,
+                                         "frac_of_8000": nbytes / ms / 1e6 / 8000.0,
+                                         "mtokens_per_s": w.n_rows / ms / 1e3}
+            del sets, pl
+        del xb
+    torch.cuda.empty_cache()
+    # dequantize and clip-error on the headline workload
+    w = synth.WORKLOADS["llama4096"]
+    x = synth.make_host("llama4096").to(device)
+    pl = Plan(w.d, w.d_pad, w.m, 3, w.group, w.alpha)
+    codes, scales, _ = pl.rotate_quantize(x)
+    yhat = torch.empty((w.n_rows, w.d_pad), dtype=torch.bfloat16, device=device)
+    ms = time_loop(lambda i: pl.dequantize(codes, scales, out=yhat, stream=stream), 50)
+    dq_bytes = w.n_rows * (w.d_pad * 3 // 8 + 4 + w.d_pad * 2)
+    out["dequantize_b3_bf16"] = {"us_per_launch": ms * 1e3, "gbs": dq_bytes / ms / 1e6}
+    alphas = np.linspace(0.5, 1.0, 32)
+    err = torch.zeros(32, dtype=torch.float64, device=device)
+    ms = time_loop(lambda i: pl.clip_error(x, alphas, err_sum=err, stream=stream), 5)
+    evals = w.n_rows * w.d_pad * 32
+    out["clip_error_K32"] = {"us_per_launch": ms * 1e3, "gevals_per_s": evals / ms / 1e6,
+                             "mtokens_per_s": w.n_rows / ms / 1e3}
+    return out
+
+
+if __name__ == "__main__":
+    main()

@@ -177,13 +177,18 @@ def test_shape_sweep(d, d_pad, m, bits, group, alpha, rows, dtype):
     x = torch.from_numpy(xs.astype(np.float32)).to(dtype)
     ref = oracle.rotate_quantize_rows(synth.to_oracle_array(x), d, d_pad, m, bits, group, alpha,
                                       dense=(d_pad <= 2048))
+    # rows must start on 16-byte boundaries: place them in a buffer whose stride is a multiple of 8
+    stride = (d + 7) // 8 * 8
+    xd = torch.zeros((rows, stride), dtype=dtype, device=DEV)
+    xd[:, :d] = x.to(DEV)
+    xd = xd[:, :d]
     with Plan(d, d_pad, m, bits, group, alpha) as plan:
-        codes, scales, y = _run_rq(plan, x.to(DEV), rows)
+        codes, scales, y = _run_rq(plan, xd, rows)
         compare_rotate_quantize(x, ref, codes, scales, y, bits, group, d_pad)
         if rows > 2:
             assert int(codes[1].max()) == 0 and float(scales[1].abs().max()) == 0.0
         alphas = [1.0, 0.8, 0.45]
-        err = plan.clip_error(x.to(DEV), alphas)
+        err = plan.clip_error(xd, alphas)
         torch.cuda.synchronize()
         eref = oracle.clip_error_rows(synth.to_oracle_array(x), d, d_pad, m, bits, group, np.array(alphas))
         np.testing.assert_allclose(err.cpu().numpy(), eref, rtol=TOL_CLIP)
