@@ -69,7 +69,9 @@ typedef struct gbs_plan_info {
     int q_lo, q_hi;                /* -D, +D                                          */
     int64_t code_bytes_per_row;    /* d' * bits / 8                                   */
     int scales_per_row;            /* group ? d'/group : 1                            */
-    int variant;                   /* kernel family chosen for bf16 rows: 0 = generic */
+    int variant;                   /* kernel family chosen for bf16 rows: 0 = generic shared-memory path,
+                                      1 = tensor-core path for d' = 4096 (set GBS_FORCE_GENERIC=1 in the
+                                      environment before gbs_plan_create to force 0) */
 } gbs_plan_info_t;
 
 /*
@@ -92,6 +94,15 @@ int gbs_plan_destroy(gbs_plan_t* plan);
 
 /* Report the derived sizes of a plan. */
 int gbs_plan_info(const gbs_plan_t* plan, gbs_plan_info_t* out);
+
+/*
+ * Read and clear the plan's device-side status word.  The tensor-core kernels bound every wait on a
+ * barrier; if one ever expires the kernel records a non-zero code here, frees what it holds and
+ * returns instead of hanging (the results of that launch are then invalid).  0 = no such event.
+ * This call copies 4 bytes from the device and therefore WAITS for the device's pending work.
+ * (Not an operation of the paper: a diagnostic of this implementation.)
+ */
+int gbs_plan_device_status(const gbs_plan_t* plan, int* out);
 
 /*
  * Fused pad -> rotate -> per-token/group absmax -> scale -> round/clip -> pack

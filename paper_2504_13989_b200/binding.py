@@ -26,7 +26,7 @@ GBS_INVERSE_ROTATE = 1
 GBS_MAX_D_PAD = 32768
 GBS_MAX_CANDIDATES = 64
 
-EXPORTS = ("gbs_plan_create", "gbs_plan_destroy", "gbs_plan_info", "gbs_rotate_quantize",
+EXPORTS = ("gbs_plan_create", "gbs_plan_destroy", "gbs_plan_info", "gbs_plan_device_status", "gbs_rotate_quantize",
            "gbs_dequantize", "gbs_clip_error", "gbs_hadamard_m", "gbs_status_string")
 
 
@@ -62,6 +62,8 @@ def lib() -> ctypes.CDLL:
         L.gbs_plan_destroy.restype = i32
         L.gbs_plan_info.argtypes = [vp, ctypes.POINTER(PlanInfo)]
         L.gbs_plan_info.restype = i32
+        L.gbs_plan_device_status.argtypes = [vp, ctypes.POINTER(i32)]
+        L.gbs_plan_device_status.restype = i32
         L.gbs_rotate_quantize.argtypes = [vp, vp, i32, i64, i64, vp, vp, vp, vp]
         L.gbs_rotate_quantize.restype = i32
         L.gbs_dequantize.argtypes = [vp, vp, vp, i64, vp, i32, i32, vp]
@@ -138,6 +140,13 @@ def gbs_plan_info(plan: int) -> PlanInfo:
     return info
 
 
+def gbs_plan_device_status(plan: int) -> int:
+    """Read and clear the plan's device status word (0 = no bounded wait ever expired).  Synchronises."""
+    v = ctypes.c_int(0)
+    _check(lib().gbs_plan_device_status(ctypes.c_void_p(plan), ctypes.byref(v)), "gbs_plan_device_status")
+    return v.value
+
+
 def gbs_hadamard_m(m: int) -> torch.Tensor:
     """The m x m sign matrix H_m the plans use (host computation, int8)."""
     out = torch.zeros((m, m), dtype=torch.int8)
@@ -205,6 +214,9 @@ class Plan:
 
     def __exit__(self, *exc):
         self.close()
+
+    def device_status(self) -> int:
+        return gbs_plan_device_status(self.handle)
 
     def alloc_outputs(self, n_rows: int, device, want_y: bool = False):
         codes = torch.empty((n_rows, self.info.code_bytes_per_row), dtype=torch.uint8, device=device)

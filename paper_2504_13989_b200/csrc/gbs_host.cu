@@ -112,6 +112,12 @@ extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bi
 
     if (gbs_generic_smem_bytes(p, nullptr) > (size_t)p->smem_optin) { delete p; return GBS_ERR_UNSUPPORTED; }
 
+    e = cudaMalloc(&p->d_status, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(int));
+    if (e != cudaSuccess) { cudaGetLastError(); if (p->d_status) cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC; }
+    const char* force = getenv("GBS_FORCE_GENERIC");
+    if (!(force && force[0] == '1') && gbs_tc_pow2_supported(p)) p->variant = GBS_VARIANT_TC_POW2;
+
     if (m > 1) {
         float h[2 * 32 * 32];
         for (int i = 0; i < m; ++i)
@@ -120,9 +126,9 @@ extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bi
                 h[m * m + j * m + i] = (float)p->h_hm[i * m + j];     // transpose, for the inverse rotation
             }
         e = cudaMalloc(&p->d_hm, sizeof(float) * 2 * m * m);
-        if (e != cudaSuccess) { cudaGetLastError(); delete p; return GBS_ERR_ALLOC; }
+        if (e != cudaSuccess) { cudaGetLastError(); cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC; }
         e = cudaMemcpy(p->d_hm, h, sizeof(float) * 2 * m * m, cudaMemcpyHostToDevice);
-        if (e != cudaSuccess) { cudaGetLastError(); cudaFree(p->d_hm); delete p; return GBS_ERR_CUDA; }
+        if (e != cudaSuccess) { cudaGetLastError(); cudaFree(p->d_hm); cudaFree(p->d_status); delete p; return GBS_ERR_CUDA; }
     }
     *out = p;
     return GBS_OK;
@@ -132,11 +138,12 @@ extern "C" int gbs_plan_destroy(gbs_plan_t* plan)
 {
     if (!plan) return GBS_OK;
     int rc = GBS_OK;
-    if (plan->d_hm) {
+    {
         DeviceGuard g;
-        if (g.enter(plan->device) != cudaSuccess || cudaFree(plan->d_hm) != cudaSuccess) {
-            cudaGetLastError();
-            rc = GBS_ERR_CUDA;
+        if (g.enter(plan->device) != cudaSuccess) { cudaGetLastError(); rc = GBS_ERR_CUDA; }
+        else {
+            if (plan->d_hm && cudaFree(plan->d_hm) != cudaSuccess) { cudaGetLastError(); rc = GBS_ERR_CUDA; }
+            if (plan->d_status && cudaFree(plan->d_status) != cudaSuccess) { cudaGetLastError(); rc = GBS_ERR_CUDA; }
         }
     }
     delete plan;
@@ -155,6 +162,21 @@ extern "C" int gbs_plan_info(const gbs_plan_t* p, gbs_plan_info_t* out)
     return GBS_OK;
 }
 
+extern "C" int gbs_plan_device_status(const gbs_plan_t* p, int* out)
+{
+    if (!p || !out) return GBS_ERR_INVALID_ARG;
+    DeviceGuard g;
+    if (g.enter(p->device) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
+    int v = 0;
+    if (cudaMemcpy(&v, p->d_status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemset(p->d_status, 0, sizeof(int)) != cudaSuccess) {
+        cudaGetLastError();
+        return GBS_ERR_CUDA;
+    }
+    *out = v;
+    return GBS_OK;
+}
+
 extern "C" int gbs_rotate_quantize(const gbs_plan_t* p, const void* x, int x_dtype, int64_t n_rows,
                                    int64_t x_row_stride, void* codes, float* scales, float* y_opt,
                                    void* cuda_stream)
@@ -166,8 +188,13 @@ extern "C" int gbs_rotate_quantize(const gbs_plan_t* p, const void* x, int x_dty
         return GBS_ERR_ALIGNMENT;
     DeviceGuard g;
     if (g.enter(p->device) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
-    int e = gbs_generic_rotate_quantize(p, x, x_dtype, n_rows, x_row_stride, codes, scales, y_opt,
-                                        static_cast<cudaStream_t>(cuda_stream));
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    int e;
+    if (p->variant == GBS_VARIANT_TC_POW2 && x_dtype == GBS_DTYPE_BF16)
+        e = gbs_tc_pow2_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
+    else
+        e = gbs_generic_rotate_quantize(p, x, x_dtype, n_rows, x_row_stride, codes, scales, y_opt, stream);
+    if (e != 0) cudaGetLastError();
     return e == 0 ? GBS_OK : GBS_ERR_CUDA;
 }
 

@@ -1,0 +1,494 @@
+// Tensor-core family for power-of-two widths: d' = 4096 (m = 1, k = 12), bf16 rows, per-token scales.
+//
+// A row of 4096 values is viewed as a 128 x 32 matrix X[u][v] (flat index u*32 + v).  Because the
+// Sylvester matrix factors as H_4096 = H_128 (x) H_32 (Eq. (1) applied to the high and the low index
+// bits), the rotation is Y = H_128 * X * H_32:
+//
+//   * H_128 * X runs on the 5th-generation tensor cores (tcgen05.mma, kind::f16, bf16 inputs, fp32
+//     accumulation in TMEM).  The products (+-1) * bf16 are exact, so this half of the transform
+//     loses nothing beyond fp32 summation.  A = H_128 (K-major, 128B swizzle), B = the raw row tile
+//     exactly as TMA drops it into shared memory (N-major, 64B swizzle), four tokens per MMA (N = 128).
+//   * the accumulator row of TMEM lane u' holds the 32 values (H_128 X)[u'][0..31] of one token, i.e.
+//     one thread owns 32 CONSECUTIVE output coordinates: the remaining H_32 is five butterfly stages
+//     in registers with no shuffles and no shared-memory transposes.
+//   * per-token max|.| (Section 2.1) is a warp reduction plus a 4-warp exchange; Delta, rounding,
+//     clipping (Section 3.1) and the 3/4-bit packing are fused into the second sweep over TMEM, and
+//     each thread stores 12 or 16 contiguous bytes of codes.
+//
+// Warp roles (one persistent CTA per SM): warp 0 = TMA producer, warp 1 = MMA issuer / TMEM owner,
+// warps 2..9 = two epilogue groups of four warps (one TMEM lane quadrant each) that alternate stages.
+// Every mbarrier wait is bounded; on expiry the kernel records an error in the plan's status word,
+// all roles leave their loops, TMEM is freed and the kernel returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "gbs_internal.h"
+
+namespace {
+
+constexpr int U = 128;                 // tensor-core factor (high index bits)
+constexpr int V = 32;                  // in-register factor (low index bits)
+constexpr int TOK = 4;                 // tokens per pipeline stage (MMA N = TOK * V = 128)
+constexpr int STAGES = 4;
+constexpr int STAGE_BYTES = TOK * U * V * 2;      // 32 KB of bf16
+constexpr int A_BYTES = U * U * 2;                // 32 KB: H_128 as bf16
+constexpr int EPI_WARPS = 8;
+constexpr int THREADS = 32 * (2 + EPI_WARPS);
+constexpr int TMEM_COLS = 512;
+constexpr int STAGE_COLS = TOK * V;               // 128 fp32 columns per stage
+constexpr unsigned WAIT_LIMIT = 1u << 22;         // polls before a wait gives up
+
+struct __align__(1024) Smem {
+    unsigned char a[A_BYTES];
+    unsigned char b[STAGES][STAGE_BYTES];
+    unsigned long long full[STAGES], empty[STAGES], tfull[STAGES], tempty[STAGES];
+    unsigned long long gsync[2];           // per epilogue group: "all four warps have published their max"
+    float red[2][2][4][TOK];               // [group][iteration parity][warp][token]
+    unsigned tmem_base;
+    volatile int abort_flag;
+};
+
+struct TcParams {
+    long long n_rows;
+    int n_groups;                 // ceil(n_rows / TOK)
+    int code_row_bytes;           // 4096 * bits / 8
+    float c_scale;                // alpha / (D sqrt(d'))
+    float c_half;                 // 1 / (2 alpha):  y / (2 D Delta) = Y * c_half / max|Y|
+    float norm;                   // 1 / sqrt(d')
+    unsigned char* codes;
+    float* scales;
+    float* y_opt;
+    int* status;
+};
+
+// ---------------------------------------------------------------------------------------------
+// PTX wrappers
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(void* bar, unsigned count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(void* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(void* bar, unsigned bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(void* bar, unsigned parity)
+{
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+
+// Bounded wait.  Returns false if the wait expired (or, with watch_abort, once another role has
+// aborted).  The epilogue groups wait without watch_abort so that all threads of a group take the same
+// decision from the barrier state alone; no unbounded barrier is used between them.
+__device__ __forceinline__ bool mbar_wait(Smem* S, void* bar, unsigned parity, int* status, int code,
+                                          bool watch_abort = true)
+{
+    for (unsigned i = 0; i < WAIT_LIMIT; ++i) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (watch_abort && (i & 1023u) == 1023u && S->abort_flag) return false;
+    }
+    S->abort_flag = 1;
+    atomicCAS(status, 0, code);
+    return false;
+}
+
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, void* bar, int c0, int c1, int c2)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(unsigned* slot, unsigned cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(unsigned addr, unsigned cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_f16(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
+                                         unsigned idesc, unsigned accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(void* bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(unsigned taddr, float v[32])
+{
+    unsigned r[32];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+}
+
+__device__ __forceinline__ void tmem_st32(unsigned taddr, const float v[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+        ::"r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
+          "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
+          "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
+          "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
+          "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
+          "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
+          "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
+          "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31])),
+          "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// ---------------------------------------------------------------------------------------------
+// descriptors
+// ---------------------------------------------------------------------------------------------
+// Shared-memory matrix descriptor: start address, leading / stride byte offsets (all >> 4),
+// descriptor version 1, swizzle mode in the top three bits (2 = 128B, 4 = 64B).
+__device__ __forceinline__ unsigned long long smem_desc(unsigned addr, unsigned lbo_bytes, unsigned sbo_bytes,
+                                                        unsigned layout_type)
+{
+    unsigned long long d = 0;
+    d |= (unsigned long long)((addr >> 4) & 0x3fffu);
+    d |= (unsigned long long)((lbo_bytes >> 4) & 0x3fffu) << 16;
+    d |= (unsigned long long)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= 1ull << 46;
+    d |= (unsigned long long)layout_type << 61;
+    return d;
+}
+
+// Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, A K-major, B N-major, M x N.
+__host__ __device__ constexpr unsigned instr_desc(int M, int N)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((unsigned)(N >> 3) << 17) |
+           ((unsigned)(M >> 4) << 24);
+}
+
+// ---------------------------------------------------------------------------------------------
+// epilogue arithmetic
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ void fwht32(float v[32])
+{
+#pragma unroll
+    for (int h = 1; h < 32; h <<= 1)
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if ((i & h) == 0) {
+                float a = v[i], b = v[i + h];
+                v[i] = a + b;
+                v[i + h] = a - b;
+            }
+}
+
+// 32 consecutive codes -> packed little-endian bit stream (BITS * 4 bytes).
+//   w = sat(Y * a1 + 0.5) maps y/Delta in [-D, D] onto [0, 1] and clips outside (Section 3.1);
+//   s = w * 2D + (2^23 + 1) leaves rint(y/Delta) + D + 1 = q + 2^(BITS-1) in the low mantissa bits
+//   (round-half-even by the FMA's own rounding); fields are gathered with shift-adds, the constant
+//   contributed by the 2^23 exponent pattern falls outside the kept bits or is subtracted, and a
+//   final XOR with 2^(BITS-1) per field turns the offset code into the two's-complement field.
+template <int BITS>
+__device__ __forceinline__ void quantize_pack32(const float v[32], float a1, unsigned out[BITS])
+{
+    const float twoD = (float)(2 * ((1 << (BITS - 1)) - 1));
+    const float MAGIC = 8388609.f;                        // 2^23 + 1
+    unsigned acc[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        unsigned a = 0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            float w = __saturatef(fmaf(v[8 * g + e], a1, 0.5f));
+            float s = fmaf(w, twoD, MAGIC);
+            a += __float_as_uint(s) << (BITS * e);
+        }
+        acc[g] = a;
+    }
+    if (BITS == 4) {
+        // sum_e 0x4B000000 << 4e (mod 2^32) = 0x4B000000 + 0xB0000000
+        constexpr unsigned C = 0x4B000000u + 0xB0000000u;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) out[g] = (acc[g] - C) ^ 0x88888888u;
+    } else {
+        // the exponent pattern only touches bits >= 24, outside the 24 kept bits
+#pragma unroll
+        for (int g = 0; g < 4; ++g) acc[g] = (acc[g] & 0x00ffffffu) ^ 0x00924924u;
+        out[0] = acc[0] | (acc[1] << 24);
+        out[1] = (acc[1] >> 8) | (acc[2] << 16);
+        out[2] = (acc[2] >> 16) | (acc[3] << 8);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// kernel
+// ---------------------------------------------------------------------------------------------
+template <int BITS>
+__global__ void __launch_bounds__(THREADS, 1) k_tc_pow2_rq(const __grid_constant__ CUtensorMap tmap, TcParams P)
+{
+    extern __shared__ unsigned char smem_raw[];
+    Smem* S = reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    // ---- one-time setup: H_128 into shared memory (K-major rows of 64 bf16, 128B swizzle), barriers, TMEM
+    for (int i = threadIdx.x; i < U * U / 8; i += THREADS) {
+        // 16-byte chunk i: block kb (k / 64), row r, chunk c within the 128-byte row
+        const int kb = i / (U * 8), r = (i / 8) % U, c = i % 8;
+        unsigned w[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int k0 = kb * 64 + c * 8 + 2 * j;
+            const unsigned lo = (__popc(r & k0) & 1) ? 0xBF80u : 0x3F80u;
+            const unsigned hi = (__popc(r & (k0 + 1)) & 1) ? 0xBF80u : 0x3F80u;
+            w[j] = lo | (hi << 16);
+        }
+        const unsigned off = kb * (U * 128) + r * 128 + ((c ^ (r & 7)) << 4);
+        *reinterpret_cast<uint4*>(S->a + off) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&S->full[s], 1);
+            mbar_init(&S->empty[s], 1);
+            mbar_init(&S->tfull[s], 1);
+            mbar_init(&S->tempty[s], 4);
+        }
+        mbar_init(&S->gsync[0], 4);
+        mbar_init(&S->gsync[1], 4);
+        S->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes of A -> async proxy
+    if (warp == 1) tmem_alloc(&S->tmem_base, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const unsigned tmem_base = S->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer ------------------------------
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
+            int it = 0;
+            for (int g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it) {
+                const int s = it % STAGES;
+                const unsigned ph = (it / STAGES) & 1;
+                if (!mbar_wait(S, &S->empty[s], ph ^ 1, P.status, 1)) break;
+                mbar_arrive_expect_tx(&S->full[s], STAGE_BYTES);
+                tma_load_3d(S->b[s], &tmap, &S->full[s], 0, 0, g * TOK);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            constexpr unsigned IDESC = instr_desc(U, STAGE_COLS);
+            const unsigned a_base = smem_u32(S->a);
+            int it = 0;
+            for (int g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it) {
+                const int s = it % STAGES;
+                const unsigned ph = (it / STAGES) & 1;
+                if (!mbar_wait(S, &S->full[s], ph, P.status, 2)) break;
+                if (!mbar_wait(S, &S->tempty[s], ph ^ 1, P.status, 3)) break;
+                tc_fence_after();
+                const unsigned b_base = smem_u32(S->b[s]);
+#pragma unroll
+                for (int j = 0; j < U / 16; ++j) {
+                    // A: k-step j = 32 bytes inside the 128-byte swizzled row of block j/4; 8-row groups 1024 B apart
+                    const unsigned long long ad = smem_desc(a_base + (j >> 2) * (U * 128) + (j & 3) * 32, 16, 1024, 2);
+                    // B: 16 u-rows of 64 bytes per k-step; 8-row groups 512 B apart; next token (N atom) 8192 B away
+                    const unsigned long long bd = smem_desc(b_base + j * 1024, U * V * 2, 512, 4);
+                    umma_f16(tmem_base + s * STAGE_COLS, ad, bd, IDESC, j > 0 ? 1u : 0u);
+                }
+                umma_commit(&S->empty[s]);
+                umma_commit(&S->tfull[s]);
+            }
+        }
+    } else {
+        // ------------------------------ epilogue ------------------------------
+        const int e = (warp - 2) >> 2;            // epilogue group 0 / 1
+        const int q = warp & 3;                   // TMEM lane quadrant this warp may access
+        const int wi = (warp - 2) & 3;            // warp index inside the group
+        const int up = q * 32 + lane;             // u' : this thread owns outputs [up*32, up*32+32)
+        for (int it = e;; it += 2) {
+            const long long g = (long long)blockIdx.x + (long long)it * gridDim.x;
+            if (g >= P.n_groups) break;
+            const int s = it % STAGES;
+            const unsigned ph = (it / STAGES) & 1;
+            if (!mbar_wait(S, &S->tfull[s], ph, P.status, 4, false)) break;
+            tc_fence_after();
+            const int par = (it >> 1) & 1;
+            const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + s * STAGE_COLS;
+            float tmax[TOK];
+            // sweep 1: finish the transform (H_32 in registers), per-thread absmax, park the values in TMEM
+#pragma unroll
+            for (int t = 0; t < TOK; ++t) {
+                float v[32];
+                tmem_ld32(taddr + t * V, v);
+                fwht32(v);
+                float m0 = 0.f, m1 = 0.f;
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) {
+                    m0 = fmaxf(m0, fabsf(v[i]));
+                    m1 = fmaxf(m1, fabsf(v[i + 1]));
+                }
+                tmax[t] = fmaxf(m0, m1);
+                tmem_st32(taddr + t * V, v);
+            }
+#pragma unroll
+            for (int t = 0; t < TOK; ++t)
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) tmax[t] = fmaxf(tmax[t], __shfl_xor_sync(0xffffffffu, tmax[t], o));
+            if (lane == 0) {
+#pragma unroll
+                for (int t = 0; t < TOK; ++t) S->red[e][par][wi][t] = tmax[t];
+                mbar_arrive(&S->gsync[e]);
+            }
+            tmem_wait_st();
+            if (!mbar_wait(S, &S->gsync[e], (unsigned)par, P.status, 5, false)) break;
+            // sweep 2: Delta, round / clip, pack, store
+#pragma unroll
+            for (int t = 0; t < TOK; ++t) {
+                const long long row = g * TOK + t;
+                const float M = fmaxf(fmaxf(S->red[e][par][0][t], S->red[e][par][1][t]),
+                                      fmaxf(S->red[e][par][2][t], S->red[e][par][3][t]));
+                if (row < P.n_rows) {
+                    float v[32];
+                    tmem_ld32(taddr + t * V, v);
+                    const float a1 = (M > 0.f) ? (P.c_half / M) : 0.f;
+                    unsigned out[BITS];
+                    quantize_pack32<BITS>(v, a1, out);
+                    unsigned* dst = reinterpret_cast<unsigned*>(P.codes + row * P.code_row_bytes + up * (V * BITS / 8));
+                    if (BITS == 4) {
+                        *reinterpret_cast<uint4*>(dst) = make_uint4(out[0], out[1], out[2], out[3]);
+                    } else {
+                        dst[0] = out[0]; dst[1] = out[1]; dst[2] = out[2];
+                    }
+                    if (up == 0) P.scales[row] = P.c_scale * M;
+                    if (P.y_opt) {
+                        float4* yo = reinterpret_cast<float4*>(P.y_opt + row * (long long)(U * V) + up * V);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            yo[i] = make_float4(v[4 * i] * P.norm, v[4 * i + 1] * P.norm, v[4 * i + 2] * P.norm,
+                                                v[4 * i + 3] * P.norm);
+                    }
+                }
+            }
+            // red[e][par] is rewritten two iterations from now; no warp can get there before every warp of
+            // the group has passed the next iteration's gsync, i.e. finished reading it here.
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&S->tempty[s]);
+        }
+    }
+
+    // ---- teardown: every role leaves its loop (normally or through the abort flag), then TMEM is freed
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// host
+// ---------------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+}  // namespace
+
+bool gbs_tc_pow2_supported(const gbs_plan* p)
+{
+    return p->m == 1 && p->k == 12 && p->group == 0 && (p->d % V) == 0 && get_encode() != nullptr &&
+           p->smem_optin >= (int)(sizeof(Smem) + 1024);
+}
+
+int gbs_tc_pow2_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
+                                float* scales, float* y_opt, cudaStream_t stream)
+{
+    EncodeTiledFn encode = get_encode();
+    if (!encode) return (int)cudaErrorNotSupported;
+    CUtensorMap tmap;
+    const cuuint64_t gdim[3] = {(cuuint64_t)V, (cuuint64_t)(p->d / V), (cuuint64_t)n_rows};
+    const cuuint64_t gstr[2] = {(cuuint64_t)(V * 2), (cuuint64_t)(stride * 2)};
+    const cuuint32_t box[3] = {V, U, TOK};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), gdim, gstr, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return (int)cudaErrorInvalidValue;
+
+    TcParams P;
+    P.n_rows = n_rows;
+    P.n_groups = (int)((n_rows + TOK - 1) / TOK);
+    P.code_row_bytes = p->d_pad * p->bits / 8;
+    P.c_scale = p->c_scale;
+    P.c_half = (float)(1.0 / (2.0 * (double)p->alpha));
+    P.norm = p->norm;
+    P.codes = (unsigned char*)codes;
+    P.scales = scales;
+    P.y_opt = y_opt;
+    P.status = p->d_status;
+    const int smem = (int)sizeof(Smem) + 1024;
+    const int grid = P.n_groups < p->sm_count ? P.n_groups : p->sm_count;
+    // opt in to the large dynamic shared memory once per device (not a stream operation)
+    static bool attr_done[64] = {false};
+    cudaError_t e = cudaSuccess;
+    if (p->device < 0 || p->device >= 64 || !attr_done[p->device]) {
+        e = cudaFuncSetAttribute(k_tc_pow2_rq<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_pow2_rq<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return (int)e;
+        if (p->device >= 0 && p->device < 64) attr_done[p->device] = true;
+    }
+    if (p->bits == 3) k_tc_pow2_rq<3><<<grid, THREADS, smem, stream>>>(tmap, P);
+    else k_tc_pow2_rq<4><<<grid, THREADS, smem, stream>>>(tmap, P);
+    return (int)cudaGetLastError();
+}

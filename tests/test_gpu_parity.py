@@ -136,6 +136,49 @@ def test_workload_parity_reduced(name, rows, bits):
 
 
 # ------------------------------------------------------------------------------------------
+# the tensor-core family (d' = 4096, bf16, per-token): row counts around the 4-token tile, the
+# 148-CTA grid and the 4-stage pipeline; strides; zero padding; and the generic family forced
+# ------------------------------------------------------------------------------------------
+@pytest.mark.parametrize("rows", [1, 2, 3, 4, 5, 7, 148 * 4 - 1, 148 * 4 + 1, 148 * 4 * 4 + 3, 5003])
+@pytest.mark.parametrize("bits", [3, 4])
+def test_tensor_core_family_row_counts(rows, bits):
+    w = synth.WORKLOADS["llama4096"]
+    x = synth.make_host("llama4096", rows, seed=1000 + rows)
+    ref = oracle_rq(x, w, bits)
+    with Plan(w.d, w.d_pad, 1, bits, 0, w.alpha) as plan:
+        assert plan.info.variant == 1, "the tensor-core family must be the one that runs for this plan"
+        codes, scales, y = _run_rq(plan, x.to(DEV), rows)
+        assert plan.device_status() == 0
+        stats = compare_rotate_quantize(x, ref, codes, scales, y, bits, 0, w.d_pad)
+        print(rows, bits, stats)
+
+
+@pytest.mark.parametrize("d,stride", [(4096, 4096 + 64), (4000, 4000), (4064, 4096), (32, 32), (2048, 8192)])
+def test_tensor_core_family_padding_and_stride(d, stride):
+    rng = np.random.Generator(np.random.PCG64(d + stride))
+    rows = 37
+    xs = torch.from_numpy(rng.standard_t(3, size=(rows, stride)).astype(np.float32)).to(torch.bfloat16)
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(xs), d, 4096, 1, 3, 0, 0.9)
+    with Plan(d, 4096, 1, 3, 0, 0.9) as plan:
+        assert plan.info.variant == 1
+        xd = xs.to(DEV)[:, :d]
+        codes, scales, y = _run_rq(plan, xd, rows)
+        assert plan.device_status() == 0
+        compare_rotate_quantize(xs[:, :d], ref, codes, scales, y, 3, 0, 4096)
+
+
+def test_generic_family_forced_matches_too(monkeypatch):
+    monkeypatch.setenv("GBS_FORCE_GENERIC", "1")
+    w = synth.WORKLOADS["llama4096"]
+    x = synth.make_host("llama4096", 77)
+    ref = oracle_rq(x, w, 3)
+    with Plan(w.d, w.d_pad, 1, 3, 0, w.alpha) as plan:
+        assert plan.info.variant == 0
+        codes, scales, y = _run_rq(plan, x.to(DEV), 77)
+        compare_rotate_quantize(x, ref, codes, scales, y, 3, 0, w.d_pad)
+
+
+# ------------------------------------------------------------------------------------------
 # shapes: every supported m, small and large k, groups, padding, strides
 # ------------------------------------------------------------------------------------------
 SHAPES = [
