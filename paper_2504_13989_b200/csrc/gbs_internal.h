@@ -25,6 +25,7 @@ struct gbs_plan {
     int smem_optin;        // largest dynamic shared memory a block may opt in to
     int variant;
     float* d_hm;           // device: H_m as floats, m*m row-major, followed by H_m^T (m*m)
+    unsigned char* d_h128; // device: pre-swizzled bf16 image of H_128 for the tensor-core family (32 KB)
     int* d_status;         // device status word: 0, or the code of the first bounded wait that expired
     int8_t h_hm[32 * 32];  // host copy of H_m (m <= 32)
 };
@@ -45,5 +46,6 @@ size_t gbs_generic_smem_bytes(const gbs_plan* p, int* rows_per_cta);
 
 // gbs_tc_pow2.cu
 bool gbs_tc_pow2_supported(const gbs_plan* p);
+void gbs_tc_pow2_h128_image(unsigned char* img32k);
 int gbs_tc_pow2_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
                                 float* scales, float* y_opt, cudaStream_t stream);

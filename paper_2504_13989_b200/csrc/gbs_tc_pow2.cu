@@ -16,7 +16,8 @@
 //     each thread stores 12 or 16 contiguous bytes of codes.
 //
 // Warp roles (one persistent CTA per SM): warp 0 = TMA producer, warp 1 = MMA issuer / TMEM owner,
-// warps 2..9 = two epilogue groups of four warps (one TMEM lane quadrant each) that alternate stages.
+// warps 2..17 = four epilogue groups of four warps (one TMEM lane quadrant each); group e owns TMEM
+// stage e.  H_128 arrives as one bulk copy of a pre-swizzled 32 KB image owned by the plan.
 // Every mbarrier wait is bounded; on expiry the kernel records an error in the plan's status word,
 // all roles leave their loops, TMEM is freed and the kernel returns.
 #include <cuda.h>
@@ -29,10 +30,10 @@ namespace {
 constexpr int U = 128;                 // tensor-core factor (high index bits)
 constexpr int V = 32;                  // in-register factor (low index bits)
 constexpr int TOK = 4;                 // tokens per pipeline stage (MMA N = TOK * V = 128)
-constexpr int STAGES = 4;
+constexpr int STAGES = 4;              // shared-memory stages = TMEM stages = epilogue groups
 constexpr int STAGE_BYTES = TOK * U * V * 2;      // 32 KB of bf16
 constexpr int A_BYTES = U * U * 2;                // 32 KB: H_128 as bf16
-constexpr int EPI_WARPS = 8;
+constexpr int EPI_WARPS = 4 * STAGES;
 constexpr int THREADS = 32 * (2 + EPI_WARPS);
 constexpr int TMEM_COLS = 512;
 constexpr int STAGE_COLS = TOK * V;               // 128 fp32 columns per stage
@@ -42,8 +43,9 @@ struct __align__(1024) Smem {
     unsigned char a[A_BYTES];
     unsigned char b[STAGES][STAGE_BYTES];
     unsigned long long full[STAGES], empty[STAGES], tfull[STAGES], tempty[STAGES];
-    unsigned long long gsync[2];           // per epilogue group: "all four warps have published their max"
-    float red[2][2][4][TOK];               // [group][iteration parity][warp][token]
+    unsigned long long gsync[STAGES];      // per epilogue group: "all four warps have published their max"
+    unsigned long long abar;               // H_128 image has landed
+    float red[STAGES][2][4][TOK];          // [group][iteration parity][warp][token]
     unsigned tmem_base;
     volatile int abort_flag;
 };
@@ -55,6 +57,7 @@ struct TcParams {
     float c_scale;                // alpha / (D sqrt(d'))
     float c_half;                 // 1 / (2 alpha):  y / (2 D Delta) = Y * c_half / max|Y|
     float norm;                   // 1 / sqrt(d')
+    const unsigned char* h128;    // pre-swizzled shared-memory image of H_128 (bf16), 32 KB
     unsigned char* codes;
     float* scales;
     float* y_opt;
@@ -110,6 +113,12 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, v
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, void* bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
 
 __device__ __forceinline__ void tmem_alloc(unsigned* slot, unsigned cols)
 {
@@ -137,9 +146,12 @@ __device__ __forceinline__ void umma_commit(void* bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-__device__ __forceinline__ void tmem_ld32(unsigned taddr, float v[32])
+// 32 consecutive fp32 columns of this thread's TMEM lane -> 32 registers.  The load is asynchronous:
+// tmem_ld_wait() must be called (it names the registers so nothing is scheduled across it).
+#define R32(r) r[0], r[1], r[2], r[3], r[4], r[5], r[6], r[7], r[8], r[9], r[10], r[11], r[12], r[13], r[14], r[15], \
+               r[16], r[17], r[18], r[19], r[20], r[21], r[22], r[23], r[24], r[25], r[26], r[27], r[28], r[29], r[30], r[31]
+__device__ __forceinline__ void tmem_ld32_issue(unsigned taddr, unsigned r[32])
 {
-    unsigned r[32];
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -149,28 +161,66 @@ __device__ __forceinline__ void tmem_ld32(unsigned taddr, float v[32])
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
 }
-
-__device__ __forceinline__ void tmem_st32(unsigned taddr, const float v[32])
+__device__ __forceinline__ void tmem_ld_wait(unsigned r[32])
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+          "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+          "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+        :: "memory");
+}
+__device__ __forceinline__ void tmem_st32(unsigned taddr, const unsigned r[32])
 {
     asm volatile(
         "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
         "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
-        ::"r"(__float_as_uint(v[0])), "r"(__float_as_uint(v[1])), "r"(__float_as_uint(v[2])), "r"(__float_as_uint(v[3])),
-          "r"(__float_as_uint(v[4])), "r"(__float_as_uint(v[5])), "r"(__float_as_uint(v[6])), "r"(__float_as_uint(v[7])),
-          "r"(__float_as_uint(v[8])), "r"(__float_as_uint(v[9])), "r"(__float_as_uint(v[10])), "r"(__float_as_uint(v[11])),
-          "r"(__float_as_uint(v[12])), "r"(__float_as_uint(v[13])), "r"(__float_as_uint(v[14])), "r"(__float_as_uint(v[15])),
-          "r"(__float_as_uint(v[16])), "r"(__float_as_uint(v[17])), "r"(__float_as_uint(v[18])), "r"(__float_as_uint(v[19])),
-          "r"(__float_as_uint(v[20])), "r"(__float_as_uint(v[21])), "r"(__float_as_uint(v[22])), "r"(__float_as_uint(v[23])),
-          "r"(__float_as_uint(v[24])), "r"(__float_as_uint(v[25])), "r"(__float_as_uint(v[26])), "r"(__float_as_uint(v[27])),
-          "r"(__float_as_uint(v[28])), "r"(__float_as_uint(v[29])), "r"(__float_as_uint(v[30])), "r"(__float_as_uint(v[31])),
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
           "r"(taddr) : "memory");
 }
 __device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// packed fp32 pairs (sm_100 f32x2 arithmetic: two lanes per issue slot)
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pk(unsigned lo, unsigned hi)
+{
+    f32x2 d;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+    return d;
+}
+__device__ __forceinline__ void unpk(f32x2 v, unsigned& lo, unsigned& hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b)
+{
+    f32x2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b)
+{
+    f32x2 d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
+{
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 
 // ---------------------------------------------------------------------------------------------
 // descriptors
@@ -199,17 +249,32 @@ __host__ __device__ constexpr unsigned instr_desc(int M, int N)
 // ---------------------------------------------------------------------------------------------
 // epilogue arithmetic
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ void fwht32(float v[32])
+// H_32 on 32 registers (in place, natural order) and max|.| of the result.  The lowest stage pairs
+// neighbours (scalar add/sub); the other four stages run on packed pairs.
+__device__ __forceinline__ float fwht32_absmax(unsigned r[32])
 {
+    f32x2 p[16];
 #pragma unroll
-    for (int h = 1; h < 32; h <<= 1)
+    for (int i = 0; i < 16; ++i) {
+        const float a = __uint_as_float(r[2 * i]), b = __uint_as_float(r[2 * i + 1]);
+        p[i] = pk(__float_as_uint(a + b), __float_as_uint(a - b));
+    }
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
+    for (int h = 1; h < 16; h <<= 1)
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
             if ((i & h) == 0) {
-                float a = v[i], b = v[i + h];
-                v[i] = a + b;
-                v[i + h] = a - b;
+                const f32x2 a = p[i], b = p[i + h];
+                p[i] = add2(a, b);
+                p[i + h] = sub2(a, b);
             }
+    float m = 0.f;
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        unpk(p[i], r[2 * i], r[2 * i + 1]);
+        m = max3(fabsf(__uint_as_float(r[2 * i])), fabsf(__uint_as_float(r[2 * i + 1])), m);
+    }
+    return m;
 }
 
 // 32 consecutive codes -> packed little-endian bit stream (BITS * 4 bytes).
@@ -219,19 +284,24 @@ __device__ __forceinline__ void fwht32(float v[32])
 //   contributed by the 2^23 exponent pattern falls outside the kept bits or is subtracted, and a
 //   final XOR with 2^(BITS-1) per field turns the offset code into the two's-complement field.
 template <int BITS>
-__device__ __forceinline__ void quantize_pack32(const float v[32], float a1, unsigned out[BITS])
+__device__ __forceinline__ void quantize_pack32(const unsigned r[32], float a1, unsigned out[BITS])
 {
     const float twoD = (float)(2 * ((1 << (BITS - 1)) - 1));
     const float MAGIC = 8388609.f;                        // 2^23 + 1
+    const f32x2 twoD2 = pk(__float_as_uint(twoD), __float_as_uint(twoD));
+    const f32x2 magic2 = pk(__float_as_uint(MAGIC), __float_as_uint(MAGIC));
     unsigned acc[4];
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
         unsigned a = 0;
 #pragma unroll
-        for (int e = 0; e < 8; ++e) {
-            float w = __saturatef(fmaf(v[8 * g + e], a1, 0.5f));
-            float s = fmaf(w, twoD, MAGIC);
-            a += __float_as_uint(s) << (BITS * e);
+        for (int e = 0; e < 8; e += 2) {
+            const float w0 = __saturatef(fmaf(__uint_as_float(r[8 * g + e]), a1, 0.5f));
+            const float w1 = __saturatef(fmaf(__uint_as_float(r[8 * g + e + 1]), a1, 0.5f));
+            unsigned s0, s1;
+            unpk(fma2(pk(__float_as_uint(w0), __float_as_uint(w1)), twoD2, magic2), s0, s1);
+            a += s0 << (BITS * e);
+            a += s1 << (BITS * (e + 1));
         }
         acc[g] = a;
     }
@@ -260,34 +330,19 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_pow2_rq(const __grid_constant
     Smem* S = reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    // ---- one-time setup: H_128 into shared memory (K-major rows of 64 bf16, 128B swizzle), barriers, TMEM
-    for (int i = threadIdx.x; i < U * U / 8; i += THREADS) {
-        // 16-byte chunk i: block kb (k / 64), row r, chunk c within the 128-byte row
-        const int kb = i / (U * 8), r = (i / 8) % U, c = i % 8;
-        unsigned w[4];
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            const int k0 = kb * 64 + c * 8 + 2 * j;
-            const unsigned lo = (__popc(r & k0) & 1) ? 0xBF80u : 0x3F80u;
-            const unsigned hi = (__popc(r & (k0 + 1)) & 1) ? 0xBF80u : 0x3F80u;
-            w[j] = lo | (hi << 16);
-        }
-        const unsigned off = kb * (U * 128) + r * 128 + ((c ^ (r & 7)) << 4);
-        *reinterpret_cast<uint4*>(S->a + off) = make_uint4(w[0], w[1], w[2], w[3]);
-    }
+    // ---- one-time setup: barriers (thread 0) and TMEM (warp 1) in parallel, one block barrier
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&S->full[s], 1);
             mbar_init(&S->empty[s], 1);
             mbar_init(&S->tfull[s], 1);
             mbar_init(&S->tempty[s], 4);
+            mbar_init(&S->gsync[s], 4);
         }
-        mbar_init(&S->gsync[0], 4);
-        mbar_init(&S->gsync[1], 4);
+        mbar_init(&S->abar, 1);
         S->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes of A -> async proxy
     if (warp == 1) tmem_alloc(&S->tmem_base, TMEM_COLS);
     tc_fence_before();
     __syncthreads();
@@ -298,6 +353,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_pow2_rq(const __grid_constant
         // ------------------------------ TMA producer ------------------------------
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
+            mbar_arrive_expect_tx(&S->abar, A_BYTES);
+            bulk_load(S->a, P.h128, A_BYTES, &S->abar);
             int it = 0;
             for (int g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it) {
                 const int s = it % STAGES;
@@ -312,8 +369,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_pow2_rq(const __grid_constant
         if (lane == 0) {
             constexpr unsigned IDESC = instr_desc(U, STAGE_COLS);
             const unsigned a_base = smem_u32(S->a);
+            bool ok = mbar_wait(S, &S->abar, 0, P.status, 6);
             int it = 0;
-            for (int g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it) {
+            for (int g = blockIdx.x; ok && g < P.n_groups; g += gridDim.x, ++it) {
                 const int s = it % STAGES;
                 const unsigned ph = (it / STAGES) & 1;
                 if (!mbar_wait(S, &S->full[s], ph, P.status, 2)) break;
@@ -334,34 +392,31 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_pow2_rq(const __grid_constant
         }
     } else {
         // ------------------------------ epilogue ------------------------------
-        const int e = (warp - 2) >> 2;            // epilogue group 0 / 1
+        const int e = (warp - 2) >> 2;            // epilogue group = TMEM / shared-memory stage it serves
         const int q = warp & 3;                   // TMEM lane quadrant this warp may access
         const int wi = (warp - 2) & 3;            // warp index inside the group
         const int up = q * 32 + lane;             // u' : this thread owns outputs [up*32, up*32+32)
-        for (int it = e;; it += 2) {
+        const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + e * STAGE_COLS;
+        int n = 0;                                // iterations done by this group
+        for (int it = e;; it += STAGES, ++n) {
             const long long g = (long long)blockIdx.x + (long long)it * gridDim.x;
             if (g >= P.n_groups) break;
-            const int s = it % STAGES;
-            const unsigned ph = (it / STAGES) & 1;
-            if (!mbar_wait(S, &S->tfull[s], ph, P.status, 4, false)) break;
+            const unsigned ph = n & 1;
+            if (!mbar_wait(S, &S->tfull[e], ph, P.status, 4, false)) break;
             tc_fence_after();
-            const int par = (it >> 1) & 1;
-            const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + s * STAGE_COLS;
             float tmax[TOK];
-            // sweep 1: finish the transform (H_32 in registers), per-thread absmax, park the values in TMEM
+            unsigned ra[32], rb[32];
+            // sweep 1: finish the transform (H_32 in registers), per-thread absmax, park the values in TMEM;
+            // the load of token t+1 is in flight while token t is processed
+            tmem_ld32_issue(taddr, ra);
 #pragma unroll
             for (int t = 0; t < TOK; ++t) {
-                float v[32];
-                tmem_ld32(taddr + t * V, v);
-                fwht32(v);
-                float m0 = 0.f, m1 = 0.f;
-#pragma unroll
-                for (int i = 0; i < 32; i += 2) {
-                    m0 = fmaxf(m0, fabsf(v[i]));
-                    m1 = fmaxf(m1, fabsf(v[i + 1]));
-                }
-                tmax[t] = fmaxf(m0, m1);
-                tmem_st32(taddr + t * V, v);
+                unsigned* cur = (t & 1) ? rb : ra;
+                unsigned* nxt = (t & 1) ? ra : rb;
+                tmem_ld_wait(cur);
+                if (t + 1 < TOK) tmem_ld32_issue(taddr + (t + 1) * V, nxt);
+                tmax[t] = fwht32_absmax(cur);
+                tmem_st32(taddr + t * V, cur);
             }
 #pragma unroll
             for (int t = 0; t < TOK; ++t)
@@ -369,23 +424,26 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_pow2_rq(const __grid_constant
                 for (int o = 16; o > 0; o >>= 1) tmax[t] = fmaxf(tmax[t], __shfl_xor_sync(0xffffffffu, tmax[t], o));
             if (lane == 0) {
 #pragma unroll
-                for (int t = 0; t < TOK; ++t) S->red[e][par][wi][t] = tmax[t];
+                for (int t = 0; t < TOK; ++t) S->red[e][ph][wi][t] = tmax[t];
                 mbar_arrive(&S->gsync[e]);
             }
             tmem_wait_st();
-            if (!mbar_wait(S, &S->gsync[e], (unsigned)par, P.status, 5, false)) break;
+            tmem_ld32_issue(taddr, ra);
+            if (!mbar_wait(S, &S->gsync[e], ph, P.status, 5, false)) break;
             // sweep 2: Delta, round / clip, pack, store
 #pragma unroll
             for (int t = 0; t < TOK; ++t) {
+                unsigned* cur = (t & 1) ? rb : ra;
+                unsigned* nxt = (t & 1) ? ra : rb;
+                tmem_ld_wait(cur);
+                if (t + 1 < TOK) tmem_ld32_issue(taddr + (t + 1) * V, nxt);
                 const long long row = g * TOK + t;
-                const float M = fmaxf(fmaxf(S->red[e][par][0][t], S->red[e][par][1][t]),
-                                      fmaxf(S->red[e][par][2][t], S->red[e][par][3][t]));
+                const float M = fmaxf(fmaxf(S->red[e][ph][0][t], S->red[e][ph][1][t]),
+                                      fmaxf(S->red[e][ph][2][t], S->red[e][ph][3][t]));
                 if (row < P.n_rows) {
-                    float v[32];
-                    tmem_ld32(taddr + t * V, v);
                     const float a1 = (M > 0.f) ? (P.c_half / M) : 0.f;
                     unsigned out[BITS];
-                    quantize_pack32<BITS>(v, a1, out);
+                    quantize_pack32<BITS>(cur, a1, out);
                     unsigned* dst = reinterpret_cast<unsigned*>(P.codes + row * P.code_row_bytes + up * (V * BITS / 8));
                     if (BITS == 4) {
                         *reinterpret_cast<uint4*>(dst) = make_uint4(out[0], out[1], out[2], out[3]);
@@ -397,16 +455,16 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_pow2_rq(const __grid_constant
                         float4* yo = reinterpret_cast<float4*>(P.y_opt + row * (long long)(U * V) + up * V);
 #pragma unroll
                         for (int i = 0; i < 8; ++i)
-                            yo[i] = make_float4(v[4 * i] * P.norm, v[4 * i + 1] * P.norm, v[4 * i + 2] * P.norm,
-                                                v[4 * i + 3] * P.norm);
+                            yo[i] = make_float4(__uint_as_float(cur[4 * i]) * P.norm, __uint_as_float(cur[4 * i + 1]) * P.norm,
+                                                __uint_as_float(cur[4 * i + 2]) * P.norm, __uint_as_float(cur[4 * i + 3]) * P.norm);
                     }
                 }
             }
-            // red[e][par] is rewritten two iterations from now; no warp can get there before every warp of
+            // red[e][ph] is rewritten two iterations from now; no warp can get there before every warp of
             // the group has passed the next iteration's gsync, i.e. finished reading it here.
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&S->tempty[s]);
+            if (lane == 0) mbar_arrive(&S->tempty[e]);
         }
     }
 
@@ -445,6 +503,22 @@ EncodeTiledFn get_encode()
 
 }  // namespace
 
+// Shared-memory image of H_128 as bf16: two blocks of 64 k-columns, rows of 128 bytes, 16-byte chunks
+// XOR-swizzled with the row index (the 128B swizzle the MMA descriptor names).
+void gbs_tc_pow2_h128_image(unsigned char* img)
+{
+    unsigned short* h = reinterpret_cast<unsigned short*>(img);
+    for (int kb = 0; kb < 2; ++kb)
+        for (int r = 0; r < U; ++r)
+            for (int c = 0; c < 8; ++c)
+                for (int j = 0; j < 8; ++j) {
+                    const int k = kb * 64 + c * 8 + j;
+                    const bool neg = (__builtin_popcount((unsigned)(r & k)) & 1) != 0;
+                    const size_t off = (size_t)kb * (U * 128) + (size_t)r * 128 + (size_t)((c ^ (r & 7)) << 4) + j * 2;
+                    h[off / 2] = neg ? 0xBF80 : 0x3F80;
+                }
+}
+
 bool gbs_tc_pow2_supported(const gbs_plan* p)
 {
     return p->m == 1 && p->k == 12 && p->group == 0 && (p->d % V) == 0 && get_encode() != nullptr &&
@@ -473,6 +547,7 @@ int gbs_tc_pow2_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows
     P.c_scale = p->c_scale;
     P.c_half = (float)(1.0 / (2.0 * (double)p->alpha));
     P.norm = p->norm;
+    P.h128 = p->d_h128;
     P.codes = (unsigned char*)codes;
     P.scales = scales;
     P.y_opt = y_opt;
