@@ -70,8 +70,10 @@ typedef struct gbs_plan_info {
     int64_t code_bytes_per_row;    /* d' * bits / 8                                   */
     int scales_per_row;            /* group ? d'/group : 1                            */
     int variant;                   /* kernel family chosen for bf16 rows: 0 = generic shared-memory path,
-                                      1 = tensor-core path for d' = 4096 (set GBS_FORCE_GENERIC=1 in the
-                                      environment before gbs_plan_create to force 0) */
+                                      1 = tensor-core path for d' = 32 * U with U = m * 2^j <= 128, U % 16 == 0,
+                                      d % 32 == 0 and group in {0, 32 .. 1024} (set GBS_FORCE_GENERIC=1 in the
+                                      environment before gbs_plan_create to force 0; GBS_NO_PDL=1 launches it
+                                      without programmatic stream serialization) */
 } gbs_plan_info_t;
 
 /*

@@ -116,20 +116,9 @@ extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bi
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(int));
     if (e != cudaSuccess) { cudaGetLastError(); if (p->d_status) cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC; }
     const char* force = getenv("GBS_FORCE_GENERIC");
-    if (!(force && force[0] == '1') && gbs_tc_pow2_supported(p)) {
-        unsigned char* img = (unsigned char*)malloc(32768);
-        if (!img) { cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC; }
-        gbs_tc_pow2_h128_image(img);
-        e = cudaMalloc(&p->d_h128, 32768);
-        if (e == cudaSuccess) e = cudaMemcpy(p->d_h128, img, 32768, cudaMemcpyHostToDevice);
-        free(img);
-        if (e != cudaSuccess) {
-            cudaGetLastError();
-            if (p->d_h128) cudaFree(p->d_h128);
-            cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC;
-        }
-        p->variant = GBS_VARIANT_TC_POW2;
-    }
+    if (!(force && force[0] == '1') && gbs_tc_uv_supported(p)) p->variant = GBS_VARIANT_TC_UV;
+    const char* nopdl = getenv("GBS_NO_PDL");
+    p->pdl = (nopdl && nopdl[0] == '1') ? 0 : 1;
 
     if (m > 1) {
         float h[2 * 32 * 32];
@@ -139,9 +128,9 @@ extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bi
                 h[m * m + j * m + i] = (float)p->h_hm[i * m + j];     // transpose, for the inverse rotation
             }
         e = cudaMalloc(&p->d_hm, sizeof(float) * 2 * m * m);
-        if (e != cudaSuccess) { cudaGetLastError(); cudaFree(p->d_status); if (p->d_h128) cudaFree(p->d_h128); delete p; return GBS_ERR_ALLOC; }
+        if (e != cudaSuccess) { cudaGetLastError(); cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC; }
         e = cudaMemcpy(p->d_hm, h, sizeof(float) * 2 * m * m, cudaMemcpyHostToDevice);
-        if (e != cudaSuccess) { cudaGetLastError(); cudaFree(p->d_hm); cudaFree(p->d_status); if (p->d_h128) cudaFree(p->d_h128); delete p; return GBS_ERR_CUDA; }
+        if (e != cudaSuccess) { cudaGetLastError(); cudaFree(p->d_hm); cudaFree(p->d_status); delete p; return GBS_ERR_CUDA; }
     }
     *out = p;
     return GBS_OK;
@@ -157,7 +146,6 @@ extern "C" int gbs_plan_destroy(gbs_plan_t* plan)
         else {
             if (plan->d_hm && cudaFree(plan->d_hm) != cudaSuccess) { cudaGetLastError(); rc = GBS_ERR_CUDA; }
             if (plan->d_status && cudaFree(plan->d_status) != cudaSuccess) { cudaGetLastError(); rc = GBS_ERR_CUDA; }
-            if (plan->d_h128 && cudaFree(plan->d_h128) != cudaSuccess) { cudaGetLastError(); rc = GBS_ERR_CUDA; }
         }
     }
     delete plan;
@@ -204,8 +192,8 @@ extern "C" int gbs_rotate_quantize(const gbs_plan_t* p, const void* x, int x_dty
     if (g.enter(p->device) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     int e;
-    if (p->variant == GBS_VARIANT_TC_POW2 && x_dtype == GBS_DTYPE_BF16)
-        e = gbs_tc_pow2_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
+    if (p->variant == GBS_VARIANT_TC_UV && x_dtype == GBS_DTYPE_BF16)
+        e = gbs_tc_uv_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
     else
         e = gbs_generic_rotate_quantize(p, x, x_dtype, n_rows, x_row_stride, codes, scales, y_opt, stream);
     if (e != 0) cudaGetLastError();

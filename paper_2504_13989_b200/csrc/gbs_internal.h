@@ -9,7 +9,8 @@
 // Kernel families a plan can select for bf16 rows.
 enum gbs_variant {
     GBS_VARIANT_GENERIC = 0,   // shared-memory FWHT on the plain ALUs; any supported (m, k), any dtype
-    GBS_VARIANT_TC_POW2 = 1,   // d' = 4096: H_128 on tcgen05 tensor cores + H_32 in registers (bf16 rows)
+    GBS_VARIANT_TC_UV = 1,     // d' = U*32, U = m*2^j <= 128: (H_m (x) H_{2^j}) on tcgen05 tensor cores + H_32 in
+                               // registers (bf16 rows)
 };
 
 struct gbs_plan {
@@ -25,7 +26,7 @@ struct gbs_plan {
     int smem_optin;        // largest dynamic shared memory a block may opt in to
     int variant;
     float* d_hm;           // device: H_m as floats, m*m row-major, followed by H_m^T (m*m)
-    unsigned char* d_h128; // device: pre-swizzled bf16 image of H_128 for the tensor-core family (32 KB)
+    int pdl;               // tensor-core families launch with programmatic stream serialization
     int* d_status;         // device status word: 0, or the code of the first bounded wait that expired
     int8_t h_hm[32 * 32];  // host copy of H_m (m <= 32)
 };
@@ -44,8 +45,7 @@ int gbs_generic_dequantize(const gbs_plan* p, const void* codes, const float* sc
                            void* out, int out_dtype, int inverse, cudaStream_t stream);
 size_t gbs_generic_smem_bytes(const gbs_plan* p, int* rows_per_cta);
 
-// gbs_tc_pow2.cu
-bool gbs_tc_pow2_supported(const gbs_plan* p);
-void gbs_tc_pow2_h128_image(unsigned char* img32k);
-int gbs_tc_pow2_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
-                                float* scales, float* y_opt, cudaStream_t stream);
+// gbs_tc_uv.cu
+bool gbs_tc_uv_supported(const gbs_plan* p);
+int gbs_tc_uv_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
+                              float* scales, float* y_opt, cudaStream_t stream);

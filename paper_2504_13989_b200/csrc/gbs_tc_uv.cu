@@ -1,25 +1,29 @@
-// Tensor-core family for power-of-two widths: d' = 4096 (m = 1, k = 12), bf16 rows, per-token scales.
+// Tensor-core family "UV": bf16 rows of padded width d' = U * 32 with U = m * 2^j <= 128.
 //
-// A row of 4096 values is viewed as a 128 x 32 matrix X[u][v] (flat index u*32 + v).  Because the
-// Sylvester matrix factors as H_4096 = H_128 (x) H_32 (Eq. (1) applied to the high and the low index
-// bits), the rotation is Y = H_128 * X * H_32:
+// A padded row is viewed as a U x 32 matrix X[u][v] (flat index u*32 + v, u = a*2^j + c_hi, v = c_lo).
+// With 2^k = 2^j * 32 the rotation H_m (x) H_{2^k} factors as (H_m (x) H_{2^j}) (x) H_32 (Eq. (1) applied
+// to the high and the low bits of the Sylvester index; Algorithm 2 for H_m), so
 //
-//   * H_128 * X runs on the 5th-generation tensor cores (tcgen05.mma, kind::f16, bf16 inputs, fp32
-//     accumulation in TMEM).  The products (+-1) * bf16 are exact, so this half of the transform
-//     loses nothing beyond fp32 summation.  A = H_128 (K-major, 128B swizzle), B = the raw row tile
-//     exactly as TMA drops it into shared memory (N-major, 64B swizzle), four tokens per MMA (N = 128).
-//   * the accumulator row of TMEM lane u' holds the 32 values (H_128 X)[u'][0..31] of one token, i.e.
-//     one thread owns 32 CONSECUTIVE output coordinates: the remaining H_32 is five butterfly stages
-//     in registers with no shuffles and no shared-memory transposes.
-//   * per-token max|.| (Section 2.1) is a warp reduction plus a 4-warp exchange; Delta, rounding,
-//     clipping (Section 3.1) and the 3/4-bit packing are fused into the second sweep over TMEM, and
-//     each thread stores 12 or 16 contiguous bytes of codes.
+//        Y = A * X * H_32,      A = H_m (x) H_{2^j}   (U x U, entries +-1).
 //
-// Warp roles (one persistent CTA per SM): warp 0 = TMA producer, warp 1 = MMA issuer / TMEM owner,
-// warps 2..17 = four epilogue groups of four warps (one TMEM lane quadrant each); group e owns TMEM
-// stage e.  H_128 arrives as one bulk copy of a pre-swizzled 32 KB image owned by the plan.
-// Every mbarrier wait is bounded; on expiry the kernel records an error in the plan's status word,
-// all roles leave their loops, TMEM is freed and the kernel returns.
+//   * A * X runs on the 5th-generation tensor cores (tcgen05.mma, kind::f16, bf16 operands, fp32
+//     accumulators in TMEM).  Products (+-1) * bf16 are exact, so this half of the transform loses
+//     nothing beyond fp32 summation.  A is generated in shared memory by the CTA itself (K-major,
+//     128-byte swizzle); B is the raw row tile exactly as TMA drops it (N-major, 64-byte swizzle),
+//     four tokens per MMA (N = 128).  Rows of A beyond U are zero; columns of X beyond d are filled
+//     with zeros by TMA, which is the zero-pad expansion of Section 4.2.
+//   * TMEM lane u' then holds (A X)[u'][0..31] of a token: one thread owns 32 CONSECUTIVE output
+//     coordinates, and the remaining H_32 is five butterfly stages in its registers.
+//   * max|.| (Section 2.1): per token = warp shuffle + a 4-warp exchange; per group of 32*g
+//     coordinates (g <= 32 lanes) = warp shuffle only.  Delta, rounding, clipping (Section 3.1) and
+//     the 3/4-bit packing follow from registers; each thread stores 12 or 16 contiguous bytes.
+//
+// One persistent CTA per SM.  Warp 0 = TMA producer, warp 1 = MMA issuer / TMEM owner, warps 2..17 =
+// epilogue: warp (q, t) serves TMEM lane quadrant q and token t of EVERY stage, so all sixteen work on
+// each 4-token tile and a tile's accumulators are released as soon as they are in registers.
+// The first loads are issued before the rest of the set-up.  Every mbarrier wait is bounded; on expiry
+// the kernel records a code in the plan's status word, all roles leave their loops, TMEM is freed and
+// the kernel returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -27,13 +31,13 @@
 
 namespace {
 
-constexpr int U = 128;                 // tensor-core factor (high index bits)
 constexpr int V = 32;                  // in-register factor (low index bits)
 constexpr int TOK = 4;                 // tokens per pipeline stage (MMA N = TOK * V = 128)
-constexpr int STAGES = 4;              // shared-memory stages = TMEM stages = epilogue groups
-constexpr int STAGE_BYTES = TOK * U * V * 2;      // 32 KB of bf16
-constexpr int A_BYTES = U * U * 2;                // 32 KB: H_128 as bf16
-constexpr int EPI_WARPS = 4 * STAGES;
+constexpr int STAGES = 4;              // shared-memory stages = TMEM stages
+constexpr int UMAX = 128;              // largest tensor-core factor
+constexpr int STAGE_BYTES_MAX = TOK * UMAX * V * 2;   // 32 KB of bf16
+constexpr int A_BYTES = UMAX * UMAX * 2;              // 32 KB: A as bf16, two K blocks of 64
+constexpr int EPI_WARPS = 4 * TOK;
 constexpr int THREADS = 32 * (2 + EPI_WARPS);
 constexpr int TMEM_COLS = 512;
 constexpr int STAGE_COLS = TOK * V;               // 128 fp32 columns per stage
@@ -41,23 +45,28 @@ constexpr unsigned WAIT_LIMIT = 1u << 22;         // polls before a wait gives u
 
 struct __align__(1024) Smem {
     unsigned char a[A_BYTES];
-    unsigned char b[STAGES][STAGE_BYTES];
+    unsigned char b[STAGES][STAGE_BYTES_MAX];
     unsigned long long full[STAGES], empty[STAGES], tfull[STAGES], tempty[STAGES];
-    unsigned long long gsync[STAGES];      // per epilogue group: "all four warps have published their max"
-    unsigned long long abar;               // H_128 image has landed
-    float red[STAGES][2][4][TOK];          // [group][iteration parity][warp][token]
+    unsigned long long gsync[TOK];         // per token slot: "all four quadrant warps have published their max"
+    __align__(16) float red[TOK][2][4];    // [token slot][iteration parity][quadrant]
     unsigned tmem_base;
     volatile int abort_flag;
 };
 
-struct TcParams {
+struct UvParams {
     long long n_rows;
     int n_groups;                 // ceil(n_rows / TOK)
-    int code_row_bytes;           // 4096 * bits / 8
+    int U;                        // m * 2^j, multiple of 16, <= 128
+    int j;                        // log2 of the Sylvester part of A
+    int ksteps;                   // U / 16
+    int code_row_bytes;           // d' * bits / 8
+    int d_pad;
+    int glog;                     // lane-group mode: log2(lanes per quantization group)
+    int spr;                      // scales per row
     float c_scale;                // alpha / (D sqrt(d'))
     float c_half;                 // 1 / (2 alpha):  y / (2 D Delta) = Y * c_half / max|Y|
     float norm;                   // 1 / sqrt(d')
-    const unsigned char* h128;    // pre-swizzled shared-memory image of H_128 (bf16), 32 KB
+    unsigned hm_neg[32];          // bit a of word a': H_m[a'][a] == -1
     unsigned char* codes;
     float* scales;
     float* y_opt;
@@ -93,8 +102,8 @@ __device__ __forceinline__ bool mbar_try_wait(void* bar, unsigned parity)
 }
 
 // Bounded wait.  Returns false if the wait expired (or, with watch_abort, once another role has
-// aborted).  The epilogue groups wait without watch_abort so that all threads of a group take the same
-// decision from the barrier state alone; no unbounded barrier is used between them.
+// aborted).  The epilogue warps wait without watch_abort so that the warps sharing a barrier take the
+// same decision from the barrier state alone; no unbounded barrier is used between them.
 __device__ __forceinline__ bool mbar_wait(Smem* S, void* bar, unsigned parity, int* status, int code,
                                           bool watch_abort = true)
 {
@@ -112,12 +121,6 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, v
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, void* bar)
-{
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
 __device__ __forceinline__ void tmem_alloc(unsigned* slot, unsigned cols)
@@ -148,8 +151,6 @@ __device__ __forceinline__ void umma_commit(void* bar)
 
 // 32 consecutive fp32 columns of this thread's TMEM lane -> 32 registers.  The load is asynchronous:
 // tmem_ld_wait() must be called (it names the registers so nothing is scheduled across it).
-#define R32(r) r[0], r[1], r[2], r[3], r[4], r[5], r[6], r[7], r[8], r[9], r[10], r[11], r[12], r[13], r[14], r[15], \
-               r[16], r[17], r[18], r[19], r[20], r[21], r[22], r[23], r[24], r[25], r[26], r[27], r[28], r[29], r[30], r[31]
 __device__ __forceinline__ void tmem_ld32_issue(unsigned taddr, unsigned r[32])
 {
     asm volatile(
@@ -171,19 +172,6 @@ __device__ __forceinline__ void tmem_ld_wait(unsigned r[32])
           "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
         :: "memory");
 }
-__device__ __forceinline__ void tmem_st32(unsigned taddr, const unsigned r[32])
-{
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
-        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
-          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
-          "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 // packed fp32 pairs (sm_100 f32x2 arithmetic: two lanes per issue slot)
 typedef unsigned long long f32x2;
@@ -249,16 +237,14 @@ __host__ __device__ constexpr unsigned instr_desc(int M, int N)
 // ---------------------------------------------------------------------------------------------
 // epilogue arithmetic
 // ---------------------------------------------------------------------------------------------
-// H_32 on 32 registers (in place, natural order) and max|.| of the result.  The lowest stage pairs
-// neighbours (scalar add/sub); the other four stages run on packed pairs.
+// H_32 on 32 registers (in place, natural order) and max|.| of the result.  The four upper stages act on
+// register pairs as they come out of TMEM (packed add/sub); the lowest stage pairs the two halves of a
+// pair and is scalar, which leaves the results as the scalars the quantizer consumes.
 __device__ __forceinline__ float fwht32_absmax(unsigned r[32])
 {
     f32x2 p[16];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        const float a = __uint_as_float(r[2 * i]), b = __uint_as_float(r[2 * i + 1]);
-        p[i] = pk(__float_as_uint(a + b), __float_as_uint(a - b));
-    }
+    for (int i = 0; i < 16; ++i) p[i] = pk(r[2 * i], r[2 * i + 1]);
 #pragma unroll
     for (int h = 1; h < 16; h <<= 1)
 #pragma unroll
@@ -271,8 +257,13 @@ __device__ __forceinline__ float fwht32_absmax(unsigned r[32])
     float m = 0.f;
 #pragma unroll
     for (int i = 0; i < 16; ++i) {
-        unpk(p[i], r[2 * i], r[2 * i + 1]);
-        m = max3(fabsf(__uint_as_float(r[2 * i])), fabsf(__uint_as_float(r[2 * i + 1])), m);
+        unsigned ua, ub;
+        unpk(p[i], ua, ub);
+        const float a = __uint_as_float(ua), b = __uint_as_float(ub);
+        const float y0 = a + b, y1 = a - b;
+        r[2 * i] = __float_as_uint(y0);
+        r[2 * i + 1] = __float_as_uint(y1);
+        m = max3(fabsf(y0), fabsf(y1), m);
     }
     return m;
 }
@@ -320,71 +311,111 @@ __device__ __forceinline__ void quantize_pack32(const unsigned r[32], float a1, 
     }
 }
 
+// A = H_m (x) H_{2^j} as bf16 (+-1, zero outside U x U) in the K-major 128-byte-swizzled layout the MMA
+// descriptor names: two blocks of 64 k-columns, rows of 128 bytes, 16-byte chunks XOR-swizzled with the
+// row index.  Written by the epilogue warps while the first tiles are in flight.
+__device__ __forceinline__ void generate_a(const UvParams& P, unsigned char* a_smem, int tid, int nthreads)
+{
+    const unsigned jm = (1u << P.j) - 1u;
+    for (int c = tid; c < 2 * UMAX * 8; c += nthreads) {
+        const int kb = c >> 10, r = (c >> 3) & (UMAX - 1), ch = c & 7;
+        const int k0 = kb * 64 + ch * 8;
+        unsigned w[4];
+        const unsigned rowbits = (r < P.U) ? P.hm_neg[r >> P.j] : 0u;
+#pragma unroll
+        for (int e = 0; e < 8; e += 2) {
+            unsigned h2 = 0;
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                const int k = k0 + e + t;
+                const unsigned neg = ((rowbits >> (k >> P.j)) ^ (unsigned)__popc((unsigned)r & (unsigned)k & jm)) & 1u;
+                const unsigned h = (r < P.U && k < P.U) ? (neg ? 0xBF80u : 0x3F80u) : 0u;
+                h2 |= h << (16 * t);
+            }
+            w[e >> 1] = h2;
+        }
+        *reinterpret_cast<uint4*>(a_smem + (size_t)kb * (UMAX * 128) + (size_t)r * 128 + (size_t)((ch ^ (r & 7)) << 4)) =
+            make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // kernel
 // ---------------------------------------------------------------------------------------------
-template <int BITS>
-__global__ void __launch_bounds__(THREADS, 1) k_tc_pow2_rq(const __grid_constant__ CUtensorMap tmap, TcParams P)
+// GROUPED = false: one scale per token.  GROUPED = true: one scale per 2^glog adjacent lanes (32 * 2^glog
+// consecutive coordinates), 2^glog <= 32.
+template <int BITS, bool GROUPED>
+__global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__ CUtensorMap tmap,
+                                                         const __grid_constant__ UvParams P)
 {
     extern __shared__ unsigned char smem_raw[];
     Smem* S = reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const unsigned stage_bytes = (unsigned)(TOK * P.U * V * 2);
 
-    // ---- one-time setup: barriers (thread 0) and TMEM (warp 1) in parallel, one block barrier
+    // ---- set-up.  Thread 0 arms the barriers and starts the first loads at once; warp 1 allocates
+    // TMEM; the epilogue warps write A.  One block barrier joins the three.
+    int it_p = 0;                                  // producer iterations already issued
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             mbar_init(&S->full[s], 1);
             mbar_init(&S->empty[s], 1);
             mbar_init(&S->tfull[s], 1);
-            mbar_init(&S->tempty[s], 4);
-            mbar_init(&S->gsync[s], 4);
+            mbar_init(&S->tempty[s], EPI_WARPS);
         }
-        mbar_init(&S->abar, 1);
+        for (int t = 0; t < TOK; ++t) mbar_init(&S->gsync[t], 4);
         S->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        // programmatic dependent launch: nothing of the caller's memory is touched before this point
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        for (int g = blockIdx.x; it_p < STAGES && g < P.n_groups; g += gridDim.x, ++it_p) {
+            mbar_arrive_expect_tx(&S->full[it_p], stage_bytes);
+            tma_load_3d(S->b[it_p], &tmap, &S->full[it_p], 0, 0, g * TOK);
+        }
     }
     if (warp == 1) tmem_alloc(&S->tmem_base, TMEM_COLS);
+    if (warp >= 2) {
+        generate_a(P, S->a, threadIdx.x - 64, THREADS - 64);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const unsigned tmem_base = S->tmem_base;
 
     if (warp == 0) {
         // ------------------------------ TMA producer ------------------------------
         if (lane == 0) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&tmap) : "memory");
-            mbar_arrive_expect_tx(&S->abar, A_BYTES);
-            bulk_load(S->a, P.h128, A_BYTES, &S->abar);
-            int it = 0;
-            for (int g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it) {
+            int it = it_p;
+            for (int g = blockIdx.x + it * (int)gridDim.x; g < P.n_groups; g += gridDim.x, ++it) {
                 const int s = it % STAGES;
                 const unsigned ph = (it / STAGES) & 1;
                 if (!mbar_wait(S, &S->empty[s], ph ^ 1, P.status, 1)) break;
-                mbar_arrive_expect_tx(&S->full[s], STAGE_BYTES);
+                mbar_arrive_expect_tx(&S->full[s], stage_bytes);
                 tma_load_3d(S->b[s], &tmap, &S->full[s], 0, 0, g * TOK);
             }
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
-            constexpr unsigned IDESC = instr_desc(U, STAGE_COLS);
+            constexpr unsigned IDESC = instr_desc(UMAX, STAGE_COLS);
             const unsigned a_base = smem_u32(S->a);
-            bool ok = mbar_wait(S, &S->abar, 0, P.status, 6);
+            const unsigned tok_bytes = (unsigned)(P.U * V * 2);
             int it = 0;
-            for (int g = blockIdx.x; ok && g < P.n_groups; g += gridDim.x, ++it) {
+            for (int g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it) {
                 const int s = it % STAGES;
                 const unsigned ph = (it / STAGES) & 1;
                 if (!mbar_wait(S, &S->full[s], ph, P.status, 2)) break;
                 if (!mbar_wait(S, &S->tempty[s], ph ^ 1, P.status, 3)) break;
                 tc_fence_after();
                 const unsigned b_base = smem_u32(S->b[s]);
-#pragma unroll
-                for (int j = 0; j < U / 16; ++j) {
-                    // A: k-step j = 32 bytes inside the 128-byte swizzled row of block j/4; 8-row groups 1024 B apart
-                    const unsigned long long ad = smem_desc(a_base + (j >> 2) * (U * 128) + (j & 3) * 32, 16, 1024, 2);
-                    // B: 16 u-rows of 64 bytes per k-step; 8-row groups 512 B apart; next token (N atom) 8192 B away
-                    const unsigned long long bd = smem_desc(b_base + j * 1024, U * V * 2, 512, 4);
-                    umma_f16(tmem_base + s * STAGE_COLS, ad, bd, IDESC, j > 0 ? 1u : 0u);
+                for (int ks = 0; ks < P.ksteps; ++ks) {
+                    // A: k-step ks = 32 bytes inside the 128-byte swizzled row of block ks/4; 8-row groups 1024 B apart
+                    const unsigned long long ad = smem_desc(a_base + (ks >> 2) * (UMAX * 128) + (ks & 3) * 32, 16, 1024, 2);
+                    // B: 16 u-rows of 64 bytes per k-step; 8-row groups 512 B apart; next token (N atom) U*64 B away
+                    const unsigned long long bd = smem_desc(b_base + ks * 1024, tok_bytes, 512, 4);
+                    umma_f16(tmem_base + s * STAGE_COLS, ad, bd, IDESC, ks > 0 ? 1u : 0u);
                 }
                 umma_commit(&S->empty[s]);
                 umma_commit(&S->tfull[s]);
@@ -392,79 +423,63 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_pow2_rq(const __grid_constant
         }
     } else {
         // ------------------------------ epilogue ------------------------------
-        const int e = (warp - 2) >> 2;            // epilogue group = TMEM / shared-memory stage it serves
+        const int t = (warp - 2) >> 2;            // token slot inside every stage
         const int q = warp & 3;                   // TMEM lane quadrant this warp may access
-        const int wi = (warp - 2) & 3;            // warp index inside the group
         const int up = q * 32 + lane;             // u' : this thread owns outputs [up*32, up*32+32)
-        const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + e * STAGE_COLS;
-        int n = 0;                                // iterations done by this group
-        for (int it = e;; it += STAGES, ++n) {
-            const long long g = (long long)blockIdx.x + (long long)it * gridDim.x;
-            if (g >= P.n_groups) break;
-            const unsigned ph = n & 1;
-            if (!mbar_wait(S, &S->tfull[e], ph, P.status, 4, false)) break;
+        const unsigned taddr0 = tmem_base + ((unsigned)(q * 32) << 16) + t * V;
+        int it = 0;
+        for (long long g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it) {
+            const int s = it % STAGES;
+            const unsigned ph = (it / STAGES) & 1;
+            if (!mbar_wait(S, &S->tfull[s], ph, P.status, 4, false)) break;
             tc_fence_after();
-            float tmax[TOK];
-            unsigned ra[32], rb[32];
-            // sweep 1: finish the transform (H_32 in registers), per-thread absmax, park the values in TMEM;
-            // the load of token t+1 is in flight while token t is processed
-            tmem_ld32_issue(taddr, ra);
-#pragma unroll
-            for (int t = 0; t < TOK; ++t) {
-                unsigned* cur = (t & 1) ? rb : ra;
-                unsigned* nxt = (t & 1) ? ra : rb;
-                tmem_ld_wait(cur);
-                if (t + 1 < TOK) tmem_ld32_issue(taddr + (t + 1) * V, nxt);
-                tmax[t] = fwht32_absmax(cur);
-                tmem_st32(taddr + t * V, cur);
-            }
-#pragma unroll
-            for (int t = 0; t < TOK; ++t)
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) tmax[t] = fmaxf(tmax[t], __shfl_xor_sync(0xffffffffu, tmax[t], o));
-            if (lane == 0) {
-#pragma unroll
-                for (int t = 0; t < TOK; ++t) S->red[e][ph][wi][t] = tmax[t];
-                mbar_arrive(&S->gsync[e]);
-            }
-            tmem_wait_st();
-            tmem_ld32_issue(taddr, ra);
-            if (!mbar_wait(S, &S->gsync[e], ph, P.status, 5, false)) break;
-            // sweep 2: Delta, round / clip, pack, store
-#pragma unroll
-            for (int t = 0; t < TOK; ++t) {
-                unsigned* cur = (t & 1) ? rb : ra;
-                unsigned* nxt = (t & 1) ? ra : rb;
-                tmem_ld_wait(cur);
-                if (t + 1 < TOK) tmem_ld32_issue(taddr + (t + 1) * V, nxt);
-                const long long row = g * TOK + t;
-                const float M = fmaxf(fmaxf(S->red[e][ph][0][t], S->red[e][ph][1][t]),
-                                      fmaxf(S->red[e][ph][2][t], S->red[e][ph][3][t]));
-                if (row < P.n_rows) {
-                    const float a1 = (M > 0.f) ? (P.c_half / M) : 0.f;
-                    unsigned out[BITS];
-                    quantize_pack32<BITS>(cur, a1, out);
-                    unsigned* dst = reinterpret_cast<unsigned*>(P.codes + row * P.code_row_bytes + up * (V * BITS / 8));
-                    if (BITS == 4) {
-                        *reinterpret_cast<uint4*>(dst) = make_uint4(out[0], out[1], out[2], out[3]);
-                    } else {
-                        dst[0] = out[0]; dst[1] = out[1]; dst[2] = out[2];
-                    }
-                    if (up == 0) P.scales[row] = P.c_scale * M;
-                    if (P.y_opt) {
-                        float4* yo = reinterpret_cast<float4*>(P.y_opt + row * (long long)(U * V) + up * V);
-#pragma unroll
-                        for (int i = 0; i < 8; ++i)
-                            yo[i] = make_float4(__uint_as_float(cur[4 * i]) * P.norm, __uint_as_float(cur[4 * i + 1]) * P.norm,
-                                                __uint_as_float(cur[4 * i + 2]) * P.norm, __uint_as_float(cur[4 * i + 3]) * P.norm);
-                    }
-                }
-            }
-            // red[e][ph] is rewritten two iterations from now; no warp can get there before every warp of
-            // the group has passed the next iteration's gsync, i.e. finished reading it here.
+            unsigned r[32];
+            tmem_ld32_issue(taddr0 + s * STAGE_COLS, r);
+            tmem_ld_wait(r);
+            // the accumulators are in registers: hand the TMEM stage back to the MMA issuer
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(&S->tempty[e]);
+            if (lane == 0) mbar_arrive(&S->tempty[s]);
+
+            float M = fwht32_absmax(r);
+            const long long row = g * TOK + t;
+            if (GROUPED) {
+                for (int o = (1 << P.glog) >> 1; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+            } else {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+                const unsigned gp = it & 1;
+                if (lane == 0) {
+                    S->red[t][gp][q] = M;
+                    mbar_arrive(&S->gsync[t]);
+                }
+                if (!mbar_wait(S, &S->gsync[t], gp, P.status, 5, false)) break;
+                const float4 m4 = *reinterpret_cast<const float4*>(&S->red[t][gp][0]);
+                M = fmaxf(fmaxf(m4.x, m4.y), fmaxf(m4.z, m4.w));
+            }
+            if (row < P.n_rows && up < P.U) {
+                const float a1 = (M > 0.f) ? (P.c_half / M) : 0.f;
+                unsigned out[BITS];
+                quantize_pack32<BITS>(r, a1, out);
+                unsigned* dst = reinterpret_cast<unsigned*>(P.codes + row * P.code_row_bytes + up * (V * BITS / 8));
+                if (BITS == 4) {
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(out[0], out[1], out[2], out[3]);
+                } else {
+                    dst[0] = out[0]; dst[1] = out[1]; dst[2] = out[2];
+                }
+                if (GROUPED) {
+                    if ((lane & ((1 << P.glog) - 1)) == 0) P.scales[row * P.spr + (up >> P.glog)] = P.c_scale * M;
+                } else {
+                    if (up == 0) P.scales[row] = P.c_scale * M;
+                }
+                if (P.y_opt) {
+                    float4* yo = reinterpret_cast<float4*>(P.y_opt + row * (long long)P.d_pad + up * V);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        yo[i] = make_float4(__uint_as_float(r[4 * i]) * P.norm, __uint_as_float(r[4 * i + 1]) * P.norm,
+                                            __uint_as_float(r[4 * i + 2]) * P.norm, __uint_as_float(r[4 * i + 3]) * P.norm);
+                }
+            }
         }
     }
 
@@ -501,53 +516,77 @@ EncodeTiledFn get_encode()
     return fn;
 }
 
+int ilog2(int v)
+{
+    int l = 0;
+    while ((1 << l) < v) ++l;
+    return l;
+}
+
+template <typename KernelT>
+cudaError_t launch(KernelT kernel, int grid, int smem, cudaStream_t stream, bool pdl, const CUtensorMap& tmap,
+                   const UvParams& P)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, tmap, P);
+}
+
 }  // namespace
 
-// Shared-memory image of H_128 as bf16: two blocks of 64 k-columns, rows of 128 bytes, 16-byte chunks
-// XOR-swizzled with the row index (the 128B swizzle the MMA descriptor names).
-void gbs_tc_pow2_h128_image(unsigned char* img)
+bool gbs_tc_uv_supported(const gbs_plan* p)
 {
-    unsigned short* h = reinterpret_cast<unsigned short*>(img);
-    for (int kb = 0; kb < 2; ++kb)
-        for (int r = 0; r < U; ++r)
-            for (int c = 0; c < 8; ++c)
-                for (int j = 0; j < 8; ++j) {
-                    const int k = kb * 64 + c * 8 + j;
-                    const bool neg = (__builtin_popcount((unsigned)(r & k)) & 1) != 0;
-                    const size_t off = (size_t)kb * (U * 128) + (size_t)r * 128 + (size_t)((c ^ (r & 7)) << 4) + j * 2;
-                    h[off / 2] = neg ? 0xBF80 : 0x3F80;
-                }
+    if (p->d_pad % V != 0 || p->d % V != 0 || p->k < 5) return false;
+    const int U = p->d_pad / V;
+    if (U > UMAX || U % 16 != 0) return false;
+    if (p->group != 0 && (p->group < V || p->group / V > 32)) return false;
+    return get_encode() != nullptr && p->smem_optin >= (int)(sizeof(Smem) + 1024);
 }
 
-bool gbs_tc_pow2_supported(const gbs_plan* p)
-{
-    return p->m == 1 && p->k == 12 && p->group == 0 && (p->d % V) == 0 && get_encode() != nullptr &&
-           p->smem_optin >= (int)(sizeof(Smem) + 1024);
-}
-
-int gbs_tc_pow2_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
-                                float* scales, float* y_opt, cudaStream_t stream)
+int gbs_tc_uv_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
+                              float* scales, float* y_opt, cudaStream_t stream)
 {
     EncodeTiledFn encode = get_encode();
     if (!encode) return (int)cudaErrorNotSupported;
+    const int U = p->d_pad / V;
     CUtensorMap tmap;
     const cuuint64_t gdim[3] = {(cuuint64_t)V, (cuuint64_t)(p->d / V), (cuuint64_t)n_rows};
     const cuuint64_t gstr[2] = {(cuuint64_t)(V * 2), (cuuint64_t)(stride * 2)};
-    const cuuint32_t box[3] = {V, U, TOK};
+    const cuuint32_t box[3] = {V, (cuuint32_t)U, TOK};
     const cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), gdim, gstr, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return (int)cudaErrorInvalidValue;
 
-    TcParams P;
+    UvParams P;
     P.n_rows = n_rows;
     P.n_groups = (int)((n_rows + TOK - 1) / TOK);
+    P.U = U;
+    P.j = p->k - 5;
+    P.ksteps = U / 16;
     P.code_row_bytes = p->d_pad * p->bits / 8;
+    P.d_pad = p->d_pad;
+    P.glog = p->group ? ilog2(p->group / V) : 0;
+    P.spr = p->group ? p->d_pad / p->group : 1;
     P.c_scale = p->c_scale;
     P.c_half = (float)(1.0 / (2.0 * (double)p->alpha));
     P.norm = p->norm;
-    P.h128 = p->d_h128;
+    for (int a = 0; a < 32; ++a) {
+        unsigned bits = 0;
+        if (a < p->m)
+            for (int b = 0; b < p->m; ++b)
+                if (p->h_hm[a * p->m + b] < 0) bits |= 1u << b;
+        P.hm_neg[a] = bits;
+    }
     P.codes = (unsigned char*)codes;
     P.scales = scales;
     P.y_opt = y_opt;
@@ -558,12 +597,20 @@ int gbs_tc_pow2_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows
     static bool attr_done[64] = {false};
     cudaError_t e = cudaSuccess;
     if (p->device < 0 || p->device >= 64 || !attr_done[p->device]) {
-        e = cudaFuncSetAttribute(k_tc_pow2_rq<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_pow2_rq<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        e = cudaFuncSetAttribute(k_tc_uv_rq<3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return (int)e;
         if (p->device >= 0 && p->device < 64) attr_done[p->device] = true;
     }
-    if (p->bits == 3) k_tc_pow2_rq<3><<<grid, THREADS, smem, stream>>>(tmap, P);
-    else k_tc_pow2_rq<4><<<grid, THREADS, smem, stream>>>(tmap, P);
-    return (int)cudaGetLastError();
+    const bool pdl = p->pdl != 0;
+    if (p->group) {
+        if (p->bits == 3) e = launch(k_tc_uv_rq<3, true>, grid, smem, stream, pdl, tmap, P);
+        else e = launch(k_tc_uv_rq<4, true>, grid, smem, stream, pdl, tmap, P);
+    } else {
+        if (p->bits == 3) e = launch(k_tc_uv_rq<3, false>, grid, smem, stream, pdl, tmap, P);
+        else e = launch(k_tc_uv_rq<4, false>, grid, smem, stream, pdl, tmap, P);
+    }
+    return (int)e;
 }

@@ -136,8 +136,9 @@ def test_workload_parity_reduced(name, rows, bits):
 
 
 # ------------------------------------------------------------------------------------------
-# the tensor-core family (d' = 4096, bf16, per-token): row counts around the 4-token tile, the
-# 148-CTA grid and the 4-stage pipeline; strides; zero padding; and the generic family forced
+# the tensor-core family (bf16, d' = U*32 with U = m*2^j <= 128): row counts around the 4-token
+# tile, the 148-CTA grid and the 4-stage pipeline; strides; zero padding; every m; per-token and
+# per-group scales; and the generic family forced
 # ------------------------------------------------------------------------------------------
 @pytest.mark.parametrize("rows", [1, 2, 3, 4, 5, 7, 148 * 4 - 1, 148 * 4 + 1, 148 * 4 * 4 + 3, 5003])
 @pytest.mark.parametrize("bits", [3, 4])
@@ -176,6 +177,74 @@ def test_generic_family_forced_matches_too(monkeypatch):
         assert plan.info.variant == 0
         codes, scales, y = _run_rq(plan, x.to(DEV), 77)
         compare_rotate_quantize(x, ref, codes, scales, y, 3, 0, w.d_pad)
+
+
+UV_SHAPES = [
+    # d, d_pad, m, bits, group, alpha, rows
+    (512, 512, 1, 4, 0, 0.9, 41),
+    (512, 512, 1, 3, 32, 0.9, 41),
+    (1024, 1024, 1, 3, 1024, 0.8, 150),
+    (1000 // 32 * 32, 1024, 1, 4, 64, 1.0, 33),
+    (2048, 2048, 1, 3, 0, 0.9, 599),
+    (2048, 2048, 1, 4, 256, 0.7, 64),
+    (1536, 1536, 12, 3, 128, 0.9, 77),
+    (1536, 1536, 24, 4, 64, 0.9, 77),
+    (1536, 1536, 24, 3, 0, 0.9, 5),
+    (2560, 2560, 20, 3, 0, 0.95, 90),
+    (2560, 2560, 20, 4, 32, 0.95, 90),
+    (2400, 2560, 20, 4, 128, 0.85, 19),
+    (3584, 3584, 28, 3, 128, 0.85, 601),
+    (3584, 3584, 28, 4, 0, 0.85, 148 * 4 + 2),
+    (3584, 3584, 28, 3, 64, 0.5, 9),
+    (3520, 3584, 28, 3, 32, 1.0, 21),
+    (4096, 4096, 1, 3, 1024, 0.9, 50),
+    (4096, 4096, 1, 4, 128, 0.9, 50),
+]
+
+
+@pytest.mark.parametrize("d,d_pad,m,bits,group,alpha,rows", UV_SHAPES)
+def test_tensor_core_family_shapes(d, d_pad, m, bits, group, alpha, rows):
+    rng = np.random.Generator(np.random.PCG64(d * 11 + m * 5 + bits + group))
+    xs = rng.standard_t(3, size=(rows, d))
+    xs[:, rng.integers(0, d, 3)] *= 40
+    if rows > 2:
+        xs[2, :] = 0.0
+    x = torch.from_numpy(xs.astype(np.float32)).to(torch.bfloat16)
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(x), d, d_pad, m, bits, group, alpha,
+                                      dense=(d_pad <= 2048))
+    with Plan(d, d_pad, m, bits, group, alpha) as plan:
+        assert plan.info.variant == 1, "the tensor-core family must be the one that runs for this plan"
+        codes, scales, y = _run_rq(plan, x.to(DEV), rows)
+        assert plan.device_status() == 0
+        stats = compare_rotate_quantize(x, ref, codes, scales, y, bits, group, d_pad)
+        print(stats)
+        if rows > 2:
+            assert int(codes[2].max()) == 0 and float(scales[2].abs().max()) == 0.0
+        codes2, scales2, _ = _run_rq(plan, x.to(DEV), rows, want_y=False)
+        assert torch.equal(codes, codes2) and torch.equal(scales, scales2)
+
+
+def test_back_to_back_launches_on_one_stream():
+    """Consecutive launches overlap their set-up with the predecessor's tail (programmatic dependent
+    launch); a launch that reads what the previous one on the stream wrote must still see it."""
+    w = synth.WORKLOADS["llama4096"]
+    rows = 600
+    x = synth.make_host("llama4096", rows).to(DEV)
+    ref = oracle_rq(x.cpu(), w, 3)
+    with Plan(w.d, w.d_pad, 1, 3, 0, w.alpha) as plan:
+        buf = torch.zeros_like(x)
+        outs = [plan.alloc_outputs(rows, DEV) for _ in range(6)]
+        for i in range(6):
+            buf.copy_(x if i % 2 == 0 else torch.flip(x, dims=(0,)))      # a writer between the launches
+            plan.rotate_quantize(buf, out=outs[i])
+        for i in range(3):                                                # launches chained directly
+            plan.rotate_quantize(x, out=outs[i])
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+        for i in (0, 1, 2):
+            compare_rotate_quantize(x.cpu(), ref, outs[i][0], outs[i][1], None, 3, 0, w.d_pad)
+        assert torch.equal(outs[3][0], torch.flip(outs[0][0], dims=(0,)))
+        assert torch.equal(outs[4][0], outs[0][0])
 
 
 # ------------------------------------------------------------------------------------------
