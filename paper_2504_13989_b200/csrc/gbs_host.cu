@@ -116,7 +116,20 @@ extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bi
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(int));
     if (e != cudaSuccess) { cudaGetLastError(); if (p->d_status) cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC; }
     const char* force = getenv("GBS_FORCE_GENERIC");
-    if (!(force && force[0] == '1') && gbs_tc_uv_supported(p)) p->variant = GBS_VARIANT_TC_UV;
+    if (!(force && force[0] == '1') && gbs_tc_uv_supported(p)) {
+        unsigned char* img = (unsigned char*)malloc(32768);
+        if (!img) { cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC; }
+        gbs_tc_uv_a_image(p, img);
+        e = cudaMalloc(&p->d_aimg, 32768);
+        if (e == cudaSuccess) e = cudaMemcpy(p->d_aimg, img, 32768, cudaMemcpyHostToDevice);
+        free(img);
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            if (p->d_aimg) cudaFree(p->d_aimg);
+            cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC;
+        }
+        p->variant = GBS_VARIANT_TC_UV;
+    }
     const char* nopdl = getenv("GBS_NO_PDL");
     p->pdl = (nopdl && nopdl[0] == '1') ? 0 : 1;
 
@@ -128,9 +141,9 @@ extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bi
                 h[m * m + j * m + i] = (float)p->h_hm[i * m + j];     // transpose, for the inverse rotation
             }
         e = cudaMalloc(&p->d_hm, sizeof(float) * 2 * m * m);
-        if (e != cudaSuccess) { cudaGetLastError(); cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC; }
+        if (e != cudaSuccess) { cudaGetLastError(); cudaFree(p->d_status); if (p->d_aimg) cudaFree(p->d_aimg); delete p; return GBS_ERR_ALLOC; }
         e = cudaMemcpy(p->d_hm, h, sizeof(float) * 2 * m * m, cudaMemcpyHostToDevice);
-        if (e != cudaSuccess) { cudaGetLastError(); cudaFree(p->d_hm); cudaFree(p->d_status); delete p; return GBS_ERR_CUDA; }
+        if (e != cudaSuccess) { cudaGetLastError(); cudaFree(p->d_hm); cudaFree(p->d_status); if (p->d_aimg) cudaFree(p->d_aimg); delete p; return GBS_ERR_CUDA; }
     }
     *out = p;
     return GBS_OK;
@@ -146,6 +159,7 @@ extern "C" int gbs_plan_destroy(gbs_plan_t* plan)
         else {
             if (plan->d_hm && cudaFree(plan->d_hm) != cudaSuccess) { cudaGetLastError(); rc = GBS_ERR_CUDA; }
             if (plan->d_status && cudaFree(plan->d_status) != cudaSuccess) { cudaGetLastError(); rc = GBS_ERR_CUDA; }
+            if (plan->d_aimg && cudaFree(plan->d_aimg) != cudaSuccess) { cudaGetLastError(); rc = GBS_ERR_CUDA; }
         }
     }
     delete plan;

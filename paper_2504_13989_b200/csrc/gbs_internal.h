@@ -27,6 +27,7 @@ struct gbs_plan {
     int variant;
     float* d_hm;           // device: H_m as floats, m*m row-major, followed by H_m^T (m*m)
     int pdl;               // tensor-core families launch with programmatic stream serialization
+    unsigned char* d_aimg; // device: pre-swizzled bf16 image of H_m (x) H_{2^j} for the tensor-core family (32 KB)
     int* d_status;         // device status word: 0, or the code of the first bounded wait that expired
     int8_t h_hm[32 * 32];  // host copy of H_m (m <= 32)
 };
@@ -47,5 +48,6 @@ size_t gbs_generic_smem_bytes(const gbs_plan* p, int* rows_per_cta);
 
 // gbs_tc_uv.cu
 bool gbs_tc_uv_supported(const gbs_plan* p);
+void gbs_tc_uv_a_image(const gbs_plan* p, unsigned char* img32k);
 int gbs_tc_uv_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
                               float* scales, float* y_opt, cudaStream_t stream);

@@ -8,8 +8,9 @@
 //
 //   * A * X runs on the 5th-generation tensor cores (tcgen05.mma, kind::f16, bf16 operands, fp32
 //     accumulators in TMEM).  Products (+-1) * bf16 are exact, so this half of the transform loses
-//     nothing beyond fp32 summation.  A is generated in shared memory by the CTA itself (K-major,
-//     128-byte swizzle); B is the raw row tile exactly as TMA drops it (N-major, 64-byte swizzle),
+//     nothing beyond fp32 summation.  A arrives as one bulk copy of a plan-owned, pre-swizzled 32 KB
+//     image (K-major, 128-byte swizzle); B is the raw row tile exactly as TMA drops it (N-major,
+//     64-byte swizzle),
 //     four tokens per MMA (N = 128).  Rows of A beyond U are zero; columns of X beyond d are filled
 //     with zeros by TMA, which is the zero-pad expansion of Section 4.2.
 //   * TMEM lane u' then holds (A X)[u'][0..31] of a token: one thread owns 32 CONSECUTIVE output
@@ -21,7 +22,8 @@
 // One persistent CTA per SM.  Warp 0 = TMA producer, warp 1 = MMA issuer / TMEM owner, warps 2..17 =
 // epilogue: warp (q, t) serves TMEM lane quadrant q and token t of EVERY stage, so all sixteen work on
 // each 4-token tile and a tile's accumulators are released as soon as they are in registers.
-// The first loads are issued before the rest of the set-up.  Every mbarrier wait is bounded; on expiry
+// The first loads are issued before the rest of the set-up.  Waiting threads sleep in the barrier
+// hardware (try_wait with a suspend-time hint) instead of spinning.  Every wait is bounded; on expiry
 // the kernel records a code in the plan's status word, all roles leave their loops, TMEM is freed and
 // the kernel returns.
 #include <cuda.h>
@@ -41,13 +43,15 @@ constexpr int EPI_WARPS = 4 * TOK;
 constexpr int THREADS = 32 * (2 + EPI_WARPS);
 constexpr int TMEM_COLS = 512;
 constexpr int STAGE_COLS = TOK * V;               // 128 fp32 columns per stage
-constexpr unsigned WAIT_LIMIT = 1u << 22;         // polls before a wait gives up
+constexpr unsigned WAIT_HINT_NS = 20000;          // a waiting thread may sleep this long per poll
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after two seconds
 
 struct __align__(1024) Smem {
     unsigned char a[A_BYTES];
     unsigned char b[STAGES][STAGE_BYTES_MAX];
     unsigned long long full[STAGES], empty[STAGES], tfull[STAGES], tempty[STAGES];
-    unsigned long long gsync[TOK];         // per token slot: "all four quadrant warps have published their max"
+    unsigned long long abar;               // the image of A has landed
+    int gabort[TOK][2];                    // [token slot][iteration parity]: a warp of the slot gave up waiting
     __align__(16) float red[TOK][2][4];    // [token slot][iteration parity][quadrant]
     unsigned tmem_base;
     volatile int abort_flag;
@@ -66,7 +70,7 @@ struct UvParams {
     float c_scale;                // alpha / (D sqrt(d'))
     float c_half;                 // 1 / (2 alpha):  y / (2 D Delta) = Y * c_half / max|Y|
     float norm;                   // 1 / sqrt(d')
-    unsigned hm_neg[32];          // bit a of word a': H_m[a'][a] == -1
+    const unsigned char* a_img;   // pre-swizzled shared-memory image of A (bf16), 32 KB, plan-owned
     unsigned char* codes;
     float* scales;
     float* y_opt;
@@ -95,25 +99,42 @@ __device__ __forceinline__ bool mbar_try_wait(void* bar, unsigned parity)
     unsigned ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(WAIT_HINT_NS) : "memory");
     return ok != 0;
 }
 
-// Bounded wait.  Returns false if the wait expired (or, with watch_abort, once another role has
-// aborted).  The epilogue warps wait without watch_abort so that the warps sharing a barrier take the
-// same decision from the barrier state alone; no unbounded barrier is used between them.
-__device__ __forceinline__ bool mbar_wait(Smem* S, void* bar, unsigned parity, int* status, int code,
-                                          bool watch_abort = true)
+__device__ __forceinline__ unsigned long long global_ns()
 {
-    for (unsigned i = 0; i < WAIT_LIMIT; ++i) {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait: gives up WAIT_LIMIT_NS after its first unsuccessful poll.  Returns false if the wait
+// expired (or, with watch_abort, once another role has aborted).  The epilogue warps wait without
+// watch_abort: they leave only on their own expiry, and the four warps of a token slot leave together.
+__device__ __noinline__ bool mbar_wait_slow(Smem* S, void* bar, unsigned parity, int* status, int code,
+                                            bool watch_abort)
+{
+    const unsigned long long t0 = global_ns();
+    for (unsigned i = 1;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
-        if (watch_abort && (i & 1023u) == 1023u && S->abort_flag) return false;
+        if ((i & 15u) == 0) {
+            if (watch_abort && S->abort_flag) return false;
+            if (global_ns() - t0 > WAIT_LIMIT_NS) break;
+        }
     }
     S->abort_flag = 1;
     atomicCAS(status, 0, code);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(Smem* S, void* bar, unsigned parity, int* status, int code,
+                                          bool watch_abort = true)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(S, bar, parity, status, code, watch_abort);
 }
 
 __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, void* bar, int c0, int c1, int c2)
@@ -121,6 +142,13 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, v
     asm volatile(
         "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, void* bar)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
 __device__ __forceinline__ void tmem_alloc(unsigned* slot, unsigned cols)
@@ -311,34 +339,6 @@ __device__ __forceinline__ void quantize_pack32(const unsigned r[32], float a1, 
     }
 }
 
-// A = H_m (x) H_{2^j} as bf16 (+-1, zero outside U x U) in the K-major 128-byte-swizzled layout the MMA
-// descriptor names: two blocks of 64 k-columns, rows of 128 bytes, 16-byte chunks XOR-swizzled with the
-// row index.  Written by the epilogue warps while the first tiles are in flight.
-__device__ __forceinline__ void generate_a(const UvParams& P, unsigned char* a_smem, int tid, int nthreads)
-{
-    const unsigned jm = (1u << P.j) - 1u;
-    for (int c = tid; c < 2 * UMAX * 8; c += nthreads) {
-        const int kb = c >> 10, r = (c >> 3) & (UMAX - 1), ch = c & 7;
-        const int k0 = kb * 64 + ch * 8;
-        unsigned w[4];
-        const unsigned rowbits = (r < P.U) ? P.hm_neg[r >> P.j] : 0u;
-#pragma unroll
-        for (int e = 0; e < 8; e += 2) {
-            unsigned h2 = 0;
-#pragma unroll
-            for (int t = 0; t < 2; ++t) {
-                const int k = k0 + e + t;
-                const unsigned neg = ((rowbits >> (k >> P.j)) ^ (unsigned)__popc((unsigned)r & (unsigned)k & jm)) & 1u;
-                const unsigned h = (r < P.U && k < P.U) ? (neg ? 0xBF80u : 0x3F80u) : 0u;
-                h2 |= h << (16 * t);
-            }
-            w[e >> 1] = h2;
-        }
-        *reinterpret_cast<uint4*>(a_smem + (size_t)kb * (UMAX * 128) + (size_t)r * 128 + (size_t)((ch ^ (r & 7)) << 4)) =
-            make_uint4(w[0], w[1], w[2], w[3]);
-    }
-}
-
 // ---------------------------------------------------------------------------------------------
 // kernel
 // ---------------------------------------------------------------------------------------------
@@ -353,19 +353,15 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const unsigned stage_bytes = (unsigned)(TOK * P.U * V * 2);
 
-    // ---- set-up.  Thread 0 arms the barriers and starts the first loads at once; warp 1 allocates
-    // TMEM; the epilogue warps write A.  One block barrier joins the three.
+    // ---- set-up.  Thread 0 arms the load barriers and starts the first loads at once; one thread of
+    // warp 2 arms the remaining barriers; warp 1 allocates TMEM.  One block barrier joins the three.
     int it_p = 0;                                  // producer iterations already issued
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(&S->full[s], 1);
-            mbar_init(&S->empty[s], 1);
-            mbar_init(&S->tfull[s], 1);
-            mbar_init(&S->tempty[s], EPI_WARPS);
-        }
-        for (int t = 0; t < TOK; ++t) mbar_init(&S->gsync[t], 4);
-        S->abort_flag = 0;
+        for (int s = 0; s < STAGES; ++s) mbar_init(&S->full[s], 1);
+        mbar_init(&S->abar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_arrive_expect_tx(&S->abar, A_BYTES);
+        bulk_load(S->a, P.a_img, A_BYTES, &S->abar);          // plan-owned, immutable: needs no ordering
         // programmatic dependent launch: nothing of the caller's memory is touched before this point
         asm volatile("griddepcontrol.wait;" ::: "memory");
         for (int g = blockIdx.x; it_p < STAGES && g < P.n_groups; g += gridDim.x, ++it_p) {
@@ -373,11 +369,17 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
             tma_load_3d(S->b[it_p], &tmap, &S->full[it_p], 0, 0, g * TOK);
         }
     }
-    if (warp == 1) tmem_alloc(&S->tmem_base, TMEM_COLS);
-    if (warp >= 2) {
-        generate_a(P, S->a, threadIdx.x - 64, THREADS - 64);
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    if (threadIdx.x == 64) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(&S->empty[s], 1);
+            mbar_init(&S->tfull[s], 1);
+            mbar_init(&S->tempty[s], EPI_WARPS);
+        }
+        for (int t = 0; t < TOK; ++t) S->gabort[t][0] = S->gabort[t][1] = 0;
+        S->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (warp == 1) tmem_alloc(&S->tmem_base, TMEM_COLS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -402,8 +404,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
             constexpr unsigned IDESC = instr_desc(UMAX, STAGE_COLS);
             const unsigned a_base = smem_u32(S->a);
             const unsigned tok_bytes = (unsigned)(P.U * V * 2);
+            bool ok = mbar_wait(S, &S->abar, 0, P.status, 6);
             int it = 0;
-            for (int g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it) {
+            for (int g = blockIdx.x; ok && g < P.n_groups; g += gridDim.x, ++it) {
                 const int s = it % STAGES;
                 const unsigned ph = (it / STAGES) & 1;
                 if (!mbar_wait(S, &S->full[s], ph, P.status, 2)) break;
@@ -431,31 +434,37 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
         for (long long g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it) {
             const int s = it % STAGES;
             const unsigned ph = (it / STAGES) & 1;
-            if (!mbar_wait(S, &S->tfull[s], ph, P.status, 4, false)) break;
-            tc_fence_after();
+            const bool ok = mbar_wait(S, &S->tfull[s], ph, P.status, 4, false);
+            if (GROUPED && !ok) break;
             unsigned r[32];
-            tmem_ld32_issue(taddr0 + s * STAGE_COLS, r);
-            tmem_ld_wait(r);
-            // the accumulators are in registers: hand the TMEM stage back to the MMA issuer
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(&S->tempty[s]);
-
-            float M = fwht32_absmax(r);
+            float M = 0.f;
+            if (ok) {
+                tc_fence_after();
+                tmem_ld32_issue(taddr0 + s * STAGE_COLS, r);
+                tmem_ld_wait(r);
+                // the accumulators are in registers: hand the TMEM stage back to the MMA issuer
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&S->tempty[s]);
+                M = fwht32_absmax(r);
+            }
             const long long row = g * TOK + t;
             if (GROUPED) {
                 for (int o = (1 << P.glog) >> 1; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
             } else {
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+                // per-token max: one warp-wide integer max (the values are non-negative floats), then the four
+                // quadrant warps of the token meet at a 128-thread named barrier.  A warp whose wait expired
+                // still comes to the barrier and raises the slot's flag first, so the four leave together.
                 const unsigned gp = it & 1;
+                const unsigned mw = __reduce_max_sync(0xffffffffu, __float_as_uint(M));
                 if (lane == 0) {
-                    S->red[t][gp][q] = M;
-                    mbar_arrive(&S->gsync[t]);
+                    S->red[t][gp][q] = __uint_as_float(mw);
+                    if (!ok) S->gabort[t][gp] = 1;
                 }
-                if (!mbar_wait(S, &S->gsync[t], gp, P.status, 5, false)) break;
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
                 const float4 m4 = *reinterpret_cast<const float4*>(&S->red[t][gp][0]);
                 M = fmaxf(fmaxf(m4.x, m4.y), fmaxf(m4.z, m4.w));
+                if (S->gabort[t][gp]) break;
             }
             if (row < P.n_rows && up < P.U) {
                 const float a1 = (M > 0.f) ? (P.c_half / M) : 0.f;
@@ -542,6 +551,29 @@ cudaError_t launch(KernelT kernel, int grid, int smem, cudaStream_t stream, bool
 
 }  // namespace
 
+// Shared-memory image of A = H_m (x) H_{2^j} as bf16 (+-1; zero outside U x U): two blocks of 64
+// k-columns, 128 rows of 128 bytes each, 16-byte chunks XOR-swizzled with the row index (the 128-byte
+// swizzle the MMA descriptor names).  Row = output index u', column = input index u (y = H x).
+void gbs_tc_uv_a_image(const gbs_plan* p, unsigned char* img)
+{
+    const int U = p->d_pad / V, j = p->k - 5, jm = (1 << j) - 1;
+    unsigned short* h = reinterpret_cast<unsigned short*>(img);
+    for (int kb = 0; kb < 2; ++kb)
+        for (int r = 0; r < UMAX; ++r)
+            for (int c = 0; c < 8; ++c)
+                for (int e = 0; e < 8; ++e) {
+                    const int k = kb * 64 + c * 8 + e;
+                    unsigned short v = 0;
+                    if (r < U && k < U) {
+                        int sign = p->h_hm[(r >> j) * p->m + (k >> j)];
+                        if (__builtin_popcount((unsigned)(r & k & jm)) & 1) sign = -sign;
+                        v = sign < 0 ? 0xBF80 : 0x3F80;
+                    }
+                    const size_t off = (size_t)kb * (UMAX * 128) + (size_t)r * 128 + (size_t)((c ^ (r & 7)) << 4) + e * 2;
+                    h[off / 2] = v;
+                }
+}
+
 bool gbs_tc_uv_supported(const gbs_plan* p)
 {
     if (p->d_pad % V != 0 || p->d % V != 0 || p->k < 5) return false;
@@ -580,13 +612,7 @@ int gbs_tc_uv_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, 
     P.c_scale = p->c_scale;
     P.c_half = (float)(1.0 / (2.0 * (double)p->alpha));
     P.norm = p->norm;
-    for (int a = 0; a < 32; ++a) {
-        unsigned bits = 0;
-        if (a < p->m)
-            for (int b = 0; b < p->m; ++b)
-                if (p->h_hm[a * p->m + b] < 0) bits |= 1u << b;
-        P.hm_neg[a] = bits;
-    }
+    P.a_img = p->d_aimg;
     P.codes = (unsigned char*)codes;
     P.scales = scales;
     P.y_opt = y_opt;
