@@ -58,6 +58,8 @@ extern "C" {
 /* largest padded width and largest number of clip-ratio candidates per call */
 #define GBS_MAX_D_PAD 32768
 #define GBS_MAX_CANDIDATES 64
+/* largest padded width gbs_rotate_quantize_static serves from its fixed device array */
+#define GBS_STATIC_MAX_D_PAD 4096
 
 typedef struct gbs_plan gbs_plan_t;
 
@@ -121,6 +123,41 @@ int gbs_plan_device_status(const gbs_plan_t* plan, int* out);
 int gbs_rotate_quantize(const gbs_plan_t* plan, const void* x, int x_dtype, int64_t n_rows,
                         int64_t x_row_stride, void* codes, float* scales, float* y_opt,
                         void* cuda_stream);
+
+/*
+ * gbs_rotate_quantize for callers that must not allocate device memory.  (The paper has no counterpart
+ * of this call; it exists for the deployment reasons below.)
+ *
+ * A plan owns a little device memory that gbs_plan_create obtains from cudaMalloc: the tensor-core
+ * kernel reads a 32 KB table (the +-1 matrix H_m (x) H_{2^j} laid out for the MMA unit) and has a
+ * status word.  Some callers cannot go through that: a serving process whose memory pool has already
+ * claimed all of the GPU, so that a later cudaMalloc fails; a real-time loop that may not take the
+ * device-wide synchronisation cudaMalloc and cudaFree imply; code that is handed a device it may use
+ * but not grow on.  For them this call takes the plan's parameters directly and keeps the table and
+ * the status word in one fixed array inside the library's device image (about 32 KB on every GPU
+ * that loads the library, held until the process exits).  It calls no cudaMalloc, cudaFree or other
+ * allocating routine, and the caller still passes the input and both outputs.
+ *
+ *   d, d_pad, m, bits, group, alpha   as for gbs_plan_create, with these extra limits: bf16 rows only;
+ *                d_pad <= GBS_STATIC_MAX_D_PAD; d_pad and d multiples of 32; d_pad / 32 a multiple of
+ *                16; group 0 or 32 .. 1024.  Anything else in gbs_plan_create's range returns
+ *                GBS_ERR_UNSUPPORTED ("larger than the fixed array serves, or outside its kernel"):
+ *                use a plan for those.
+ *   x, n_rows, x_row_stride, codes, scales, cuda_stream   as for gbs_rotate_quantize with
+ *                x_dtype = GBS_DTYPE_BF16; results are identical to the plan-based call.
+ *
+ * The array is shared by every call on a device and keeps what the last call left in it:
+ *   - The first call on a device looks up the array's device address (with that device current) and
+ *     clears the status word.  Make that first call before any stream capture begins.
+ *   - A call whose (d_pad, m) differs from the previous call's on that device first rewrites the
+ *     table, with a small kernel on `cuda_stream`; calls with the same (d_pad, m) reuse it.
+ *   - Calls that can overlap on the GPU (different streams, or different host threads without
+ *     ordering between their streams) race on the array unless they all use the same (d_pad, m).
+ *     Serialise them, or give the concurrent users plans.
+ */
+int gbs_rotate_quantize_static(int d, int d_pad, int m, int bits, int group, float alpha, const void* x,
+                               int64_t n_rows, int64_t x_row_stride, void* codes, float* scales,
+                               void* cuda_stream);
 
 /*
  * Inverse of the quantizer: yhat = q * Delta (Section 2.1) in the rotated domain, width d';

@@ -27,7 +27,8 @@ GBS_MAX_D_PAD = 32768
 GBS_MAX_CANDIDATES = 64
 
 EXPORTS = ("gbs_plan_create", "gbs_plan_destroy", "gbs_plan_info", "gbs_plan_device_status", "gbs_rotate_quantize",
-           "gbs_dequantize", "gbs_clip_error", "gbs_hadamard_m", "gbs_status_string")
+           "gbs_rotate_quantize_static", "gbs_dequantize", "gbs_clip_error", "gbs_hadamard_m", "gbs_status_string")
+GBS_STATIC_MAX_D_PAD = 4096
 
 
 class GbsError(RuntimeError):
@@ -66,6 +67,8 @@ def lib() -> ctypes.CDLL:
         L.gbs_plan_device_status.restype = i32
         L.gbs_rotate_quantize.argtypes = [vp, vp, i32, i64, i64, vp, vp, vp, vp]
         L.gbs_rotate_quantize.restype = i32
+        L.gbs_rotate_quantize_static.argtypes = [i32, i32, i32, i32, i32, ctypes.c_float, vp, i64, i64, vp, vp, vp]
+        L.gbs_rotate_quantize_static.restype = i32
         L.gbs_dequantize.argtypes = [vp, vp, vp, i64, vp, i32, i32, vp]
         L.gbs_dequantize.restype = i32
         L.gbs_clip_error.argtypes = [vp, vp, i32, i64, i64, ctypes.POINTER(ctypes.c_float), i32, vp, vp, vp]
@@ -162,6 +165,20 @@ def gbs_rotate_quantize(plan: int, x: torch.Tensor, codes: torch.Tensor, scales:
                                      codes.data_ptr(), scales.data_ptr(),
                                      y_opt.data_ptr() if y_opt is not None else None, _stream_ptr(stream)),
            "gbs_rotate_quantize")
+
+
+def gbs_rotate_quantize_static(d: int, d_pad: int, m: int, bits: int, group: int, alpha: float, x: torch.Tensor,
+                               codes: torch.Tensor, scales: torch.Tensor, stream=None) -> None:
+    """gbs_rotate_quantize without a plan and without any device allocation inside the library: for
+    processes that may not call cudaMalloc (all memory already claimed by a pool, or no tolerance for
+    the device-wide synchronisation an allocation implies).  bf16 rows, d_pad <= GBS_STATIC_MAX_D_PAD;
+    see include/gbs.h for the limits and for how calls share the library's fixed device array."""
+    xv, n_rows, stride = _rows_view(x, d)
+    if xv.dtype != torch.bfloat16:
+        raise TypeError("gbs_rotate_quantize_static: x must be bfloat16")
+    _check(lib().gbs_rotate_quantize_static(d, d_pad, m, bits, group, alpha, xv.data_ptr(), n_rows, stride,
+                                            codes.data_ptr(), scales.data_ptr(), _stream_ptr(stream)),
+           "gbs_rotate_quantize_static")
 
 
 def gbs_dequantize(plan: int, codes: torch.Tensor, scales: torch.Tensor, n_rows: int, out: torch.Tensor,

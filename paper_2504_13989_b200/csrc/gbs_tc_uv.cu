@@ -28,6 +28,10 @@
 // the kernel returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <math.h>
+#include <string.h>
+
+#include <mutex>
 
 #include "gbs_internal.h"
 
@@ -639,4 +643,145 @@ int gbs_tc_uv_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, 
         else e = launch(k_tc_uv_rq<4, false>, grid, smem, stream, pdl, tmap, P);
     }
     return (int)e;
+}
+
+// ---------------------------------------------------------------------------------------------
+// gbs_rotate_quantize_static: the same fused kernel for callers that cannot allocate device memory
+// ---------------------------------------------------------------------------------------------
+// The kernel above needs 32 KB of device memory besides its inputs and outputs (the image of A) and
+// a status word.  A plan gets them from cudaMalloc; here they live in a file-scope device array that
+// every GPU loading this library carries until the process exits.
+namespace {
+
+constexpr int STATIC_IMAGE_BYTES = A_BYTES;
+constexpr int STATIC_SCRATCH_BYTES = STATIC_IMAGE_BYTES + 256;        // image, then the status word
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+
+// Fills the image of A = H_m (x) H_{2^j} (same layout as gbs_tc_uv_a_image) straight into the array.
+struct StaticFillParams {
+    int U, j;
+    unsigned hm_neg[32];          // bit a of word a': H_m[a'][a] == -1
+};
+__global__ void __launch_bounds__(256) k_static_fill_a(const __grid_constant__ StaticFillParams F)
+{
+    const unsigned jm = (1u << F.j) - 1u;
+    for (int c = blockIdx.x * blockDim.x + threadIdx.x; c < 2 * UMAX * 8; c += gridDim.x * blockDim.x) {
+        const int kb = c >> 10, r = (c >> 3) & (UMAX - 1), ch = c & 7;
+        const unsigned rowbits = (r < F.U) ? F.hm_neg[r >> F.j] : 0u;
+        unsigned w[4];
+#pragma unroll
+        for (int e = 0; e < 8; e += 2) {
+            unsigned h2 = 0;
+#pragma unroll
+            for (int t = 0; t < 2; ++t) {
+                const int k = kb * 64 + ch * 8 + e + t;
+                const unsigned neg = ((rowbits >> (k >> F.j)) ^ (unsigned)__popc((unsigned)r & (unsigned)k & jm)) & 1u;
+                const unsigned h = (r < F.U && k < F.U) ? (neg ? 0xBF80u : 0x3F80u) : 0u;
+                h2 |= h << (16 * t);
+            }
+            w[e >> 1] = h2;
+        }
+        *reinterpret_cast<uint4*>(g_static_scratch + (size_t)kb * (UMAX * 128) + (size_t)r * 128 +
+                                  (size_t)((ch ^ (r & 7)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+}
+
+struct StaticDeviceState {
+    unsigned char* scratch = nullptr;   // device address of g_static_scratch on this device
+    int sm_count = 0, smem_optin = 0;
+    int image_m = 0, image_k = 0;       // which A the array holds now (0 = none yet)
+};
+StaticDeviceState g_static_state[64];
+std::mutex g_static_mutex;
+
+}  // namespace
+
+extern "C" int gbs_rotate_quantize_static(int d, int d_pad, int m, int bits, int group, float alpha, const void* x,
+                                          int64_t n_rows, int64_t x_row_stride, void* codes, float* scales,
+                                          void* cuda_stream)
+{
+    // ---- arguments: the ranges of gbs_plan_create and gbs_rotate_quantize, then this entry point's own limits
+    if (d < 1 || d_pad < d || m < 1) return GBS_ERR_INVALID_ARG;
+    if (bits != 3 && bits != 4) return GBS_ERR_INVALID_ARG;
+    if (!(alpha > 0.f) || !(alpha <= 1.f)) return GBS_ERR_INVALID_ARG;
+    if (d_pad % m != 0) return GBS_ERR_INVALID_ARG;
+    int k = -1;
+    for (int l = 0; l < 31; ++l)
+        if ((d_pad / m) == (1 << l)) k = l;
+    if (k < 3) return GBS_ERR_INVALID_ARG;
+    if (group != 0 && (group < 8 || (group & (group - 1)) != 0 || (1 << k) % group != 0)) return GBS_ERR_INVALID_ARG;
+    if (n_rows < 0) return GBS_ERR_INVALID_ARG;
+    if (d_pad > GBS_STATIC_MAX_D_PAD) return GBS_ERR_UNSUPPORTED;          // beyond what the fixed array serves
+    if (!(m == 1 || m == 12 || m == 20 || m == 24 || m == 28)) return GBS_ERR_UNSUPPORTED;   // orders a plan accepts
+    gbs_plan p;
+    memset(&p, 0, sizeof(p));
+    if (gbs_build_hadamard_m(m, p.h_hm) != GBS_OK) return GBS_ERR_UNSUPPORTED;
+    p.d = d; p.d_pad = d_pad; p.m = m; p.k = k; p.bits = bits; p.group = group; p.alpha = alpha;
+    {
+        const int U = d_pad / V;
+        if (d_pad % V != 0 || d % V != 0 || k < 5 || U % 16 != 0 || (group != 0 && (group < V || group / V > 32)))
+            return GBS_ERR_UNSUPPORTED;                                      // outside this kernel family
+    }
+    if (n_rows == 0) return GBS_OK;
+    if (!x || !codes || !scales || x_row_stride < d) return GBS_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(x) & 15u) || ((x_row_stride * 2) & 15) || (reinterpret_cast<uintptr_t>(codes) & 15u) ||
+        (reinterpret_cast<uintptr_t>(scales) & 3u))
+        return GBS_ERR_ALIGNMENT;
+
+    p.levels = (1 << (bits - 1)) - 1;
+    const double rootn = sqrt((double)d_pad);
+    p.norm = (float)(1.0 / rootn);
+    p.c_scale = (float)((double)alpha / ((double)p.levels * rootn));
+    p.c_inv = (float)((double)p.levels / (double)alpha);
+    p.variant = GBS_VARIANT_TC_UV;
+    p.pdl = 0;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return GBS_ERR_CUDA; }
+    p.device = dev;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticDeviceState& st = g_static_state[dev];
+    if (!st.scratch) {
+        // set-up, once per device, with that device current: the array's name is only a host-side handle,
+        // the kernels need its device address
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) { cudaGetLastError(); return GBS_ERR_CUDA; }
+        if (cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&st.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
+            cudaGetLastError();
+            return GBS_ERR_CUDA;
+        }
+        if (st.smem_optin < (int)(sizeof(Smem) + 1024) || get_encode() == nullptr) return GBS_ERR_UNSUPPORTED;
+        // the status word must start at zero; the image is written below
+        if (cudaMemsetAsync(static_cast<unsigned char*>(ptr) + STATIC_IMAGE_BYTES, 0, 256, stream) != cudaSuccess) {
+            cudaGetLastError();
+            return GBS_ERR_CUDA;
+        }
+        st.scratch = static_cast<unsigned char*>(ptr);
+    }
+    p.sm_count = st.sm_count;
+    p.smem_optin = st.smem_optin;
+    p.d_aimg = st.scratch;
+    p.d_status = reinterpret_cast<int*>(st.scratch + STATIC_IMAGE_BYTES);
+    if (st.image_m != m || st.image_k != k) {
+        // the array still holds the previous call's A: rewrite it, on the caller's stream, before the kernel
+        StaticFillParams F;
+        F.U = d_pad / V;
+        F.j = k - 5;
+        for (int a = 0; a < 32; ++a) {
+            unsigned neg = 0;
+            if (a < m)
+                for (int b = 0; b < m; ++b)
+                    if (p.h_hm[a * m + b] < 0) neg |= 1u << b;
+            F.hm_neg[a] = neg;
+        }
+        k_static_fill_a<<<8, 256, 0, stream>>>(F);
+        if (cudaGetLastError() != cudaSuccess) return GBS_ERR_CUDA;
+        st.image_m = m;
+        st.image_k = k;
+    }
+    const int e = gbs_tc_uv_rotate_quantize(&p, x, n_rows, x_row_stride, codes, scales, nullptr, stream);
+    if (e != 0) cudaGetLastError();
+    return e == 0 ? GBS_OK : GBS_ERR_CUDA;
 }
