@@ -116,10 +116,14 @@ extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bi
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(int));
     if (e != cudaSuccess) { cudaGetLastError(); if (p->d_status) cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC; }
     const char* force = getenv("GBS_FORCE_GENERIC");
-    if (!(force && force[0] == '1') && gbs_tc_uv_supported(p)) {
+    const bool want_tc = !(force && force[0] == '1');
+    const bool tc_uv = want_tc && gbs_tc_uv_supported(p);
+    const bool tc_row = want_tc && !tc_uv && gbs_tc_row_supported(p);
+    if (tc_uv || tc_row) {
         unsigned char* img = (unsigned char*)malloc(32768);
         if (!img) { cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC; }
-        gbs_tc_uv_a_image(p, img);
+        if (tc_uv) gbs_tc_uv_a_image(p, img);
+        else gbs_tc_sign_image(p->h_hm, 1, 7, 128, img);                 // H_128 itself
         e = cudaMalloc(&p->d_aimg, 32768);
         if (e == cudaSuccess) e = cudaMemcpy(p->d_aimg, img, 32768, cudaMemcpyHostToDevice);
         free(img);
@@ -128,7 +132,7 @@ extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bi
             if (p->d_aimg) cudaFree(p->d_aimg);
             cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC;
         }
-        p->variant = GBS_VARIANT_TC_UV;
+        p->variant = tc_uv ? GBS_VARIANT_TC_UV : GBS_VARIANT_TC_ROW;
     }
     const char* nopdl = getenv("GBS_NO_PDL");
     p->pdl = (nopdl && nopdl[0] == '1') ? 0 : 1;
@@ -208,6 +212,8 @@ extern "C" int gbs_rotate_quantize(const gbs_plan_t* p, const void* x, int x_dty
     int e;
     if (p->variant == GBS_VARIANT_TC_UV && x_dtype == GBS_DTYPE_BF16)
         e = gbs_tc_uv_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
+    else if (p->variant == GBS_VARIANT_TC_ROW && x_dtype == GBS_DTYPE_BF16)
+        e = gbs_tc_row_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
     else
         e = gbs_generic_rotate_quantize(p, x, x_dtype, n_rows, x_row_stride, codes, scales, y_opt, stream);
     if (e != 0) cudaGetLastError();

@@ -9,6 +9,7 @@
 // Kernel families a plan can select for bf16 rows.
 enum gbs_variant {
     GBS_VARIANT_GENERIC = 0,   // shared-memory FWHT on the plain ALUs; any supported (m, k), any dtype
+    GBS_VARIANT_TC_ROW = 2,    // d' = 128 (KV rows): X * H_128 on tcgen05 tensor cores, one thread owns one row
     GBS_VARIANT_TC_UV = 1,     // d' = U*32, U = m*2^j <= 128: (H_m (x) H_{2^j}) on tcgen05 tensor cores + H_32 in
                                // registers (bf16 rows)
 };
@@ -49,5 +50,12 @@ size_t gbs_generic_smem_bytes(const gbs_plan* p, int* rows_per_cta);
 // gbs_tc_uv.cu
 bool gbs_tc_uv_supported(const gbs_plan* p);
 void gbs_tc_uv_a_image(const gbs_plan* p, unsigned char* img32k);
+// image of H_m (x) H_{2^j} (U x U inside 128 x 128, bf16 +-1, K-major, 128-byte swizzle)
+void gbs_tc_sign_image(const int8_t* hm, int m, int j, int U, unsigned char* img32k);
+
+// gbs_tc_row.cu
+bool gbs_tc_row_supported(const gbs_plan* p);
+int gbs_tc_row_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
+                               float* scales, float* y_opt, cudaStream_t stream);
 int gbs_tc_uv_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
                               float* scales, float* y_opt, cudaStream_t stream);

@@ -26,14 +26,13 @@
 // hardware (try_wait with a suspend-time hint) instead of spinning.  Every wait is bounded; on expiry
 // the kernel records a code in the plan's status word, all roles leave their loops, TMEM is freed and
 // the kernel returns.
-#include <cuda.h>
-#include <cuda_bf16.h>
 #include <math.h>
 #include <string.h>
 
 #include <mutex>
 
 #include "gbs_internal.h"
+#include "gbs_tc_common.cuh"
 
 namespace {
 
@@ -47,8 +46,6 @@ constexpr int EPI_WARPS = 4 * TOK;
 constexpr int THREADS = 32 * (2 + EPI_WARPS);
 constexpr int TMEM_COLS = 512;
 constexpr int STAGE_COLS = TOK * V;               // 128 fp32 columns per stage
-constexpr unsigned WAIT_HINT_NS = 20000;          // a waiting thread may sleep this long per poll
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // a wait gives up after two seconds
 
 struct __align__(1024) Smem {
     unsigned char a[A_BYTES];
@@ -80,268 +77,6 @@ struct UvParams {
     float* y_opt;
     int* status;
 };
-
-// ---------------------------------------------------------------------------------------------
-// PTX wrappers
-// ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ unsigned smem_u32(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(void* bar, unsigned count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(void* bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(void* bar, unsigned bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(void* bar, unsigned parity)
-{
-    unsigned ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity), "r"(WAIT_HINT_NS) : "memory");
-    return ok != 0;
-}
-
-__device__ __forceinline__ unsigned long long global_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Bounded wait: gives up WAIT_LIMIT_NS after its first unsuccessful poll.  Returns false if the wait
-// expired (or, with watch_abort, once another role has aborted).  The epilogue warps wait without
-// watch_abort: they leave only on their own expiry, and the four warps of a token slot leave together.
-__device__ __noinline__ bool mbar_wait_slow(Smem* S, void* bar, unsigned parity, int* status, int code,
-                                            bool watch_abort)
-{
-    const unsigned long long t0 = global_ns();
-    for (unsigned i = 1;; ++i) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((i & 15u) == 0) {
-            if (watch_abort && S->abort_flag) return false;
-            if (global_ns() - t0 > WAIT_LIMIT_NS) break;
-        }
-    }
-    S->abort_flag = 1;
-    atomicCAS(status, 0, code);
-    return false;
-}
-__device__ __forceinline__ bool mbar_wait(Smem* S, void* bar, unsigned parity, int* status, int code,
-                                          bool watch_abort = true)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(S, bar, parity, status, code, watch_abort);
-}
-
-__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, void* bar, int c0, int c1, int c2)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
-}
-
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, void* bar)
-{
-    asm volatile(
-        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-        ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
-
-__device__ __forceinline__ void tmem_alloc(unsigned* slot, unsigned cols)
-{
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(unsigned addr, unsigned cols)
-{
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void umma_f16(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
-                                         unsigned idesc, unsigned accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_commit(void* bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-
-// 32 consecutive fp32 columns of this thread's TMEM lane -> 32 registers.  The load is asynchronous:
-// tmem_ld_wait() must be called (it names the registers so nothing is scheduled across it).
-__device__ __forceinline__ void tmem_ld32_issue(unsigned taddr, unsigned r[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait(unsigned r[32])
-{
-    asm volatile("tcgen05.wait::ld.sync.aligned;"
-        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
-          "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
-          "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-        :: "memory");
-}
-
-// packed fp32 pairs (sm_100 f32x2 arithmetic: two lanes per issue slot)
-typedef unsigned long long f32x2;
-__device__ __forceinline__ f32x2 pk(unsigned lo, unsigned hi)
-{
-    f32x2 d;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
-    return d;
-}
-__device__ __forceinline__ void unpk(f32x2 v, unsigned& lo, unsigned& hi)
-{
-    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
-}
-__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b)
-{
-    f32x2 d;
-    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ f32x2 sub2(f32x2 a, f32x2 b)
-{
-    f32x2 d;
-    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
-__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
-{
-    f32x2 d;
-    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-    return d;
-}
-__device__ __forceinline__ float max3(float a, float b, float c)
-{
-    float d;
-    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-    return d;
-}
-
-// ---------------------------------------------------------------------------------------------
-// descriptors
-// ---------------------------------------------------------------------------------------------
-// Shared-memory matrix descriptor: start address, leading / stride byte offsets (all >> 4),
-// descriptor version 1, swizzle mode in the top three bits (2 = 128B, 4 = 64B).
-__device__ __forceinline__ unsigned long long smem_desc(unsigned addr, unsigned lbo_bytes, unsigned sbo_bytes,
-                                                        unsigned layout_type)
-{
-    unsigned long long d = 0;
-    d |= (unsigned long long)((addr >> 4) & 0x3fffu);
-    d |= (unsigned long long)((lbo_bytes >> 4) & 0x3fffu) << 16;
-    d |= (unsigned long long)((sbo_bytes >> 4) & 0x3fffu) << 32;
-    d |= 1ull << 46;
-    d |= (unsigned long long)layout_type << 61;
-    return d;
-}
-
-// Instruction descriptor, kind::f16: fp32 accumulate, bf16 A and B, A K-major, B N-major, M x N.
-__host__ __device__ constexpr unsigned instr_desc(int M, int N)
-{
-    return (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((unsigned)(N >> 3) << 17) |
-           ((unsigned)(M >> 4) << 24);
-}
-
-// ---------------------------------------------------------------------------------------------
-// epilogue arithmetic
-// ---------------------------------------------------------------------------------------------
-// H_32 on 32 registers (in place, natural order) and max|.| of the result.  The four upper stages act on
-// register pairs as they come out of TMEM (packed add/sub); the lowest stage pairs the two halves of a
-// pair and is scalar, which leaves the results as the scalars the quantizer consumes.
-__device__ __forceinline__ float fwht32_absmax(unsigned r[32])
-{
-    f32x2 p[16];
-#pragma unroll
-    for (int i = 0; i < 16; ++i) p[i] = pk(r[2 * i], r[2 * i + 1]);
-#pragma unroll
-    for (int h = 1; h < 16; h <<= 1)
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-            if ((i & h) == 0) {
-                const f32x2 a = p[i], b = p[i + h];
-                p[i] = add2(a, b);
-                p[i + h] = sub2(a, b);
-            }
-    float m = 0.f;
-#pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        unsigned ua, ub;
-        unpk(p[i], ua, ub);
-        const float a = __uint_as_float(ua), b = __uint_as_float(ub);
-        const float y0 = a + b, y1 = a - b;
-        r[2 * i] = __float_as_uint(y0);
-        r[2 * i + 1] = __float_as_uint(y1);
-        m = max3(fabsf(y0), fabsf(y1), m);
-    }
-    return m;
-}
-
-// 32 consecutive codes -> packed little-endian bit stream (BITS * 4 bytes).
-//   w = sat(Y * a1 + 0.5) maps y/Delta in [-D, D] onto [0, 1] and clips outside (Section 3.1);
-//   s = w * 2D + (2^23 + 1) leaves rint(y/Delta) + D + 1 = q + 2^(BITS-1) in the low mantissa bits
-//   (round-half-even by the FMA's own rounding); fields are gathered with shift-adds, the constant
-//   contributed by the 2^23 exponent pattern falls outside the kept bits or is subtracted, and a
-//   final XOR with 2^(BITS-1) per field turns the offset code into the two's-complement field.
-template <int BITS>
-__device__ __forceinline__ void quantize_pack32(const unsigned r[32], float a1, unsigned out[BITS])
-{
-    const float twoD = (float)(2 * ((1 << (BITS - 1)) - 1));
-    const float MAGIC = 8388609.f;                        // 2^23 + 1
-    const f32x2 twoD2 = pk(__float_as_uint(twoD), __float_as_uint(twoD));
-    const f32x2 magic2 = pk(__float_as_uint(MAGIC), __float_as_uint(MAGIC));
-    unsigned acc[4];
-#pragma unroll
-    for (int g = 0; g < 4; ++g) {
-        unsigned a = 0;
-#pragma unroll
-        for (int e = 0; e < 8; e += 2) {
-            const float w0 = __saturatef(fmaf(__uint_as_float(r[8 * g + e]), a1, 0.5f));
-            const float w1 = __saturatef(fmaf(__uint_as_float(r[8 * g + e + 1]), a1, 0.5f));
-            unsigned s0, s1;
-            unpk(fma2(pk(__float_as_uint(w0), __float_as_uint(w1)), twoD2, magic2), s0, s1);
-            a += s0 << (BITS * e);
-            a += s1 << (BITS * (e + 1));
-        }
-        acc[g] = a;
-    }
-    if (BITS == 4) {
-        // sum_e 0x4B000000 << 4e (mod 2^32) = 0x4B000000 + 0xB0000000
-        constexpr unsigned C = 0x4B000000u + 0xB0000000u;
-#pragma unroll
-        for (int g = 0; g < 4; ++g) out[g] = (acc[g] - C) ^ 0x88888888u;
-    } else {
-        // the exponent pattern only touches bits >= 24, outside the 24 kept bits
-#pragma unroll
-        for (int g = 0; g < 4; ++g) acc[g] = (acc[g] & 0x00ffffffu) ^ 0x00924924u;
-        out[0] = acc[0] | (acc[1] << 24);
-        out[1] = (acc[1] >> 8) | (acc[2] << 16);
-        out[2] = (acc[2] >> 16) | (acc[3] << 8);
-    }
-}
 
 // ---------------------------------------------------------------------------------------------
 // kernel
@@ -397,7 +132,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
             for (int g = blockIdx.x + it * (int)gridDim.x; g < P.n_groups; g += gridDim.x, ++it) {
                 const int s = it % STAGES;
                 const unsigned ph = (it / STAGES) & 1;
-                if (!mbar_wait(S, &S->empty[s], ph ^ 1, P.status, 1)) break;
+                if (!mbar_wait(&S->abort_flag, &S->empty[s], ph ^ 1, P.status, 1)) break;
                 mbar_arrive_expect_tx(&S->full[s], stage_bytes);
                 tma_load_3d(S->b[s], &tmap, &S->full[s], 0, 0, g * TOK);
             }
@@ -408,13 +143,13 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
             constexpr unsigned IDESC = instr_desc(UMAX, STAGE_COLS);
             const unsigned a_base = smem_u32(S->a);
             const unsigned tok_bytes = (unsigned)(P.U * V * 2);
-            bool ok = mbar_wait(S, &S->abar, 0, P.status, 6);
+            bool ok = mbar_wait(&S->abort_flag, &S->abar, 0, P.status, 6);
             int it = 0;
             for (int g = blockIdx.x; ok && g < P.n_groups; g += gridDim.x, ++it) {
                 const int s = it % STAGES;
                 const unsigned ph = (it / STAGES) & 1;
-                if (!mbar_wait(S, &S->full[s], ph, P.status, 2)) break;
-                if (!mbar_wait(S, &S->tempty[s], ph ^ 1, P.status, 3)) break;
+                if (!mbar_wait(&S->abort_flag, &S->full[s], ph, P.status, 2)) break;
+                if (!mbar_wait(&S->abort_flag, &S->tempty[s], ph ^ 1, P.status, 3)) break;
                 tc_fence_after();
                 const unsigned b_base = smem_u32(S->b[s]);
                 for (int ks = 0; ks < P.ksteps; ++ks) {
@@ -438,7 +173,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
         for (long long g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it) {
             const int s = it % STAGES;
             const unsigned ph = (it / STAGES) & 1;
-            const bool ok = mbar_wait(S, &S->tfull[s], ph, P.status, 4, false);
+            const bool ok = mbar_wait(&S->abort_flag, &S->tfull[s], ph, P.status, 4, false);
             if (GROUPED && !ok) break;
             unsigned r[32];
             float M = 0.f;
@@ -508,27 +243,6 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
 // ---------------------------------------------------------------------------------------------
 // host
 // ---------------------------------------------------------------------------------------------
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode()
-{
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* p = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(p);
-        else
-            cudaGetLastError();
-    }
-    return fn;
-}
-
 int ilog2(int v)
 {
     int l = 0;
@@ -558,9 +272,9 @@ cudaError_t launch(KernelT kernel, int grid, int smem, cudaStream_t stream, bool
 // Shared-memory image of A = H_m (x) H_{2^j} as bf16 (+-1; zero outside U x U): two blocks of 64
 // k-columns, 128 rows of 128 bytes each, 16-byte chunks XOR-swizzled with the row index (the 128-byte
 // swizzle the MMA descriptor names).  Row = output index u', column = input index u (y = H x).
-void gbs_tc_uv_a_image(const gbs_plan* p, unsigned char* img)
+void gbs_tc_sign_image(const int8_t* hm, int m, int j, int U, unsigned char* img)
 {
-    const int U = p->d_pad / V, j = p->k - 5, jm = (1 << j) - 1;
+    const int jm = (1 << j) - 1;
     unsigned short* h = reinterpret_cast<unsigned short*>(img);
     for (int kb = 0; kb < 2; ++kb)
         for (int r = 0; r < UMAX; ++r)
@@ -569,13 +283,18 @@ void gbs_tc_uv_a_image(const gbs_plan* p, unsigned char* img)
                     const int k = kb * 64 + c * 8 + e;
                     unsigned short v = 0;
                     if (r < U && k < U) {
-                        int sign = p->h_hm[(r >> j) * p->m + (k >> j)];
+                        int sign = hm[(r >> j) * m + (k >> j)];
                         if (__builtin_popcount((unsigned)(r & k & jm)) & 1) sign = -sign;
                         v = sign < 0 ? 0xBF80 : 0x3F80;
                     }
                     const size_t off = (size_t)kb * (UMAX * 128) + (size_t)r * 128 + (size_t)((c ^ (r & 7)) << 4) + e * 2;
                     h[off / 2] = v;
                 }
+}
+
+void gbs_tc_uv_a_image(const gbs_plan* p, unsigned char* img)
+{
+    gbs_tc_sign_image(p->h_hm, p->m, p->k - 5, p->d_pad / V, img);
 }
 
 bool gbs_tc_uv_supported(const gbs_plan* p)

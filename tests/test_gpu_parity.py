@@ -224,6 +224,45 @@ def test_tensor_core_family_shapes(d, d_pad, m, bits, group, alpha, rows):
         assert torch.equal(codes, codes2) and torch.equal(scales, scales2)
 
 
+ROW_SHAPES = [
+    # d, bits, group, alpha, rows, stride
+    (128, 3, 0, 1.0, 1, 128),
+    (128, 4, 0, 0.9, 127, 128),
+    (128, 3, 0, 1.0, 129, 128),
+    (128, 3, 32, 0.8, 148 * 128 + 5, 128),
+    (128, 4, 64, 0.9, 1000, 256),
+    (128, 3, 128, 0.7, 70001, 128),
+    (96, 4, 0, 0.9, 300, 96),
+    (64, 3, 32, 1.0, 300, 72),
+    (40, 3, 0, 0.9, 515, 40),
+    (8, 4, 64, 0.9, 33, 8),
+]
+
+
+@pytest.mark.parametrize("d,bits,group,alpha,rows,stride", ROW_SHAPES)
+def test_row_family_shapes(d, bits, group, alpha, rows, stride):
+    """d' = 128 rows (KV entries): one tensor-core contraction per 128-row tile, one thread per row."""
+    rng = np.random.Generator(np.random.PCG64(d * 13 + bits + group + rows))
+    xs = rng.standard_t(3, size=(rows, stride))
+    xs[:, rng.integers(0, d, 2)] *= 40
+    if rows > 2:
+        xs[2, :] = 0.0
+    xb = torch.from_numpy(xs.astype(np.float32)).to(torch.bfloat16)
+    x = xb[:, :d]
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(x.contiguous()), d, 128, 1, bits, group, alpha, dense=True)
+    with Plan(d, 128, 1, bits, group, alpha) as plan:
+        assert plan.info.variant == 2, "the row tensor-core family must be the one that runs for this plan"
+        xd = xb.to(DEV)[:, :d]
+        codes, scales, y = _run_rq(plan, xd, rows)
+        assert plan.device_status() == 0
+        stats = compare_rotate_quantize(x, ref, codes, scales, y, bits, group, 128)
+        print(stats)
+        if rows > 2:
+            assert int(codes[2].max()) == 0 and float(scales[2].abs().max()) == 0.0
+        codes2, scales2, _ = _run_rq(plan, xd, rows, want_y=False)
+        assert torch.equal(codes, codes2) and torch.equal(scales, scales2)
+
+
 def test_back_to_back_launches_on_one_stream():
     """Consecutive launches overlap their set-up with the predecessor's tail (programmatic dependent
     launch); a launch that reads what the previous one on the stream wrote must still see it."""
