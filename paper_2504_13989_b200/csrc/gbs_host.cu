@@ -259,7 +259,13 @@ extern "C" int gbs_clip_error(const gbs_plan_t* p, const void* x, int x_dtype, i
         return GBS_ERR_ALIGNMENT;
     DeviceGuard g;
     if (g.enter(p->device) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
-    int e = gbs_generic_clip_error(p, x, x_dtype, n_rows, x_row_stride, c_scale, c_inv, K, err_sum, err_rows_opt,
+    int e;
+    if (p->variant == GBS_VARIANT_TC_UV && x_dtype == GBS_DTYPE_BF16)
+        e = gbs_tc_uv_clip_error(p, x, n_rows, x_row_stride, alphas_host, K, err_sum, err_rows_opt,
+                                 static_cast<cudaStream_t>(cuda_stream));
+    else
+        e = gbs_generic_clip_error(p, x, x_dtype, n_rows, x_row_stride, c_scale, c_inv, K, err_sum, err_rows_opt,
                                    static_cast<cudaStream_t>(cuda_stream));
+    if (e != 0) cudaGetLastError();
     return e == 0 ? GBS_OK : GBS_ERR_CUDA;
 }

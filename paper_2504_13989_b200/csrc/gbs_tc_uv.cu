@@ -54,6 +54,7 @@ struct __align__(1024) Smem {
     unsigned long long abar;               // the image of A has landed
     int gabort[TOK][2];                    // [token slot][iteration parity]: a warp of the slot gave up waiting
     __align__(16) float red[TOK][2][4];    // [token slot][iteration parity][quadrant]
+    float part[TOK][2][4][GBS_MAX_CANDIDATES];   // clip scoring: per-quadrant error sums of a token
     unsigned tmem_base;
     volatile int abort_flag;
 };
@@ -76,14 +77,86 @@ struct UvParams {
     float* scales;
     float* y_opt;
     int* status;
+    // clip-ratio scoring (the CLIP instantiation only)
+    int K;                        // candidates
+    int levels;                   // D
+    float norm2;                  // 1 / d'
+    float clip_half[GBS_MAX_CANDIDATES];    // 1 / (2 alpha_k), zero beyond K
+    float clip_scale[GBS_MAX_CANDIDATES];   // alpha_k / D,     zero beyond K
+    double* err_sum;
+    float* err_rows;
 };
+
+// Squared quantization error of this thread's 32 rotated values under every candidate clip ratio
+// (Sections 2.1, 3.1), in units of the unnormalised rotation; the sums over the warp's 32 lanes are left in
+// part_q[0 .. K).  Per value and candidate: clamp to the clipped range (fma.sat), round half-even (magic
+// add), residual, square-accumulate: five fp32 operations.  Candidates go eight at a time so the 32
+// values stay in registers; the eight partial sums are folded across the warp by a halving exchange.
+__device__ __forceinline__ void clip_score32(const unsigned r[32], float M, const UvParams& P, float* part_q, int lane)
+{
+    const float rM = (M > 0.f) ? (1.f / M) : 0.f;
+    const float twoD = (float)(2 * P.levels);
+    const float MAGIC = 8388608.f;                       // 2^23: w * 2D + MAGIC has rint(w * 2D) in its low bits
+    const float mD = MAGIC + (float)P.levels;
+    for (int k0 = 0; k0 < P.K; k0 += 8) {
+        float a1[8], dl[8], acc[8];
+#pragma unroll
+        for (int kk = 0; kk < 8; ++kk) {
+            a1[kk] = P.clip_half[k0 + kk] * rM;
+            dl[kk] = -P.clip_scale[k0 + kk] * M;         // -Delta_k
+            acc[kk] = 0.f;
+        }
+#pragma unroll
+        for (int e = 0; e < 32; ++e) {
+            const float y = __uint_as_float(r[e]);
+#pragma unroll
+            for (int kk = 0; kk < 8; ++kk) {
+                const float w = __saturatef(fmaf(y, a1[kk], 0.5f));
+                const float qv = fmaf(w, twoD, MAGIC) - mD;            // the code, as a float
+                const float err = fmaf(qv, dl[kk], y);
+                acc[kk] = fmaf(err, err, acc[kk]);
+            }
+        }
+        // fold 8 sums x 32 lanes: after three halving exchanges lane l holds candidate ((l>>4)&1)*4 +
+        // ((l>>3)&1)*2 + ((l>>2)&1) summed over 8 lanes; two more exchanges finish the warp sum
+        float h4[4], h2[2], h1;
+        {
+            const bool up = (lane & 16) != 0;
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float send = up ? acc[i] : acc[i + 4];
+                const float keep = up ? acc[i + 4] : acc[i];
+                h4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+            }
+        }
+        {
+            const bool up = (lane & 8) != 0;
+#pragma unroll
+            for (int i = 0; i < 2; ++i) {
+                const float send = up ? h4[i] : h4[i + 2];
+                const float keep = up ? h4[i + 2] : h4[i];
+                h2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+            }
+        }
+        {
+            const bool up = (lane & 4) != 0;
+            const float send = up ? h2[0] : h2[1];
+            const float keep = up ? h2[1] : h2[0];
+            h1 = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+        }
+        h1 += __shfl_xor_sync(0xffffffffu, h1, 2);
+        h1 += __shfl_xor_sync(0xffffffffu, h1, 1);
+        const int kk = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
+        if ((lane & 3) == 0 && k0 + kk < P.K) part_q[k0 + kk] = h1;
+    }
+}
 
 // ---------------------------------------------------------------------------------------------
 // kernel
 // ---------------------------------------------------------------------------------------------
 // GROUPED = false: one scale per token.  GROUPED = true: one scale per 2^glog adjacent lanes (32 * 2^glog
-// consecutive coordinates), 2^glog <= 32.
-template <int BITS, bool GROUPED>
+// consecutive coordinates), 2^glog <= 32.  CLIP = true: instead of quantizing, score K clip ratios.
+template <int BITS, bool GROUPED, bool CLIP>
 __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__ CUtensorMap tmap,
                                                          const __grid_constant__ UvParams P)
 {
@@ -169,12 +242,13 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
         const int q = warp & 3;                   // TMEM lane quadrant this warp may access
         const int up = q * 32 + lane;             // u' : this thread owns outputs [up*32, up*32+32)
         const unsigned taddr0 = tmem_base + ((unsigned)(q * 32) << 16) + t * V;
+        double dacc0 = 0.0, dacc1 = 0.0;          // CLIP, quadrant-0 warps: totals of candidates lane, lane + 32
         int it = 0;
         for (long long g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it) {
             const int s = it % STAGES;
             const unsigned ph = (it / STAGES) & 1;
             const bool ok = mbar_wait(&S->abort_flag, &S->tfull[s], ph, P.status, 4, false);
-            if (GROUPED && !ok) break;
+            if (!CLIP && GROUPED && !ok) break;
             unsigned r[32];
             float M = 0.f;
             if (ok) {
@@ -188,13 +262,13 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
                 M = fwht32_absmax(r);
             }
             const long long row = g * TOK + t;
+            const unsigned gp = it & 1;
             if (GROUPED) {
                 for (int o = (1 << P.glog) >> 1; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
             } else {
                 // per-token max: one warp-wide integer max (the values are non-negative floats), then the four
                 // quadrant warps of the token meet at a 128-thread named barrier.  A warp whose wait expired
                 // still comes to the barrier and raises the slot's flag first, so the four leave together.
-                const unsigned gp = it & 1;
                 const unsigned mw = __reduce_max_sync(0xffffffffu, __float_as_uint(M));
                 if (lane == 0) {
                     S->red[t][gp][q] = __uint_as_float(mw);
@@ -203,7 +277,25 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
                 asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
                 const float4 m4 = *reinterpret_cast<const float4*>(&S->red[t][gp][0]);
                 M = fmaxf(fmaxf(m4.x, m4.y), fmaxf(m4.z, m4.w));
+                if (!CLIP && S->gabort[t][gp]) break;
+            }
+            if (CLIP) {
+                // each quadrant warp leaves its 32-lane sums in shared memory; the four meet at the token's
+                // named barrier (a warp whose wait expired comes too, flag raised), then the quadrant-0 warp
+                // adds the four parts in a fixed order: per-row output and fp64 running totals
+                if (GROUPED && !ok && lane == 0) S->gabort[t][gp] = 1;
+                if (ok) clip_score32(r, M, P, S->part[t][gp][q], lane);
+                asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
                 if (S->gabort[t][gp]) break;
+                if (q == 0) {
+                    for (int k = lane; k < P.K; k += 32) {
+                        const float rk = (S->part[t][gp][0][k] + S->part[t][gp][1][k]) +
+                                         (S->part[t][gp][2][k] + S->part[t][gp][3][k]);
+                        if (P.err_rows && row < P.n_rows) P.err_rows[row * P.K + k] = rk * P.norm2;
+                        if (k < 32) dacc0 += (double)rk; else dacc1 += (double)rk;
+                    }
+                }
+                continue;
             }
             if (row < P.n_rows && up < P.U) {
                 const float a1 = (M > 0.f) ? (P.c_half / M) : 0.f;
@@ -228,6 +320,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
                                             __uint_as_float(r[4 * i + 2]) * P.norm, __uint_as_float(r[4 * i + 3]) * P.norm);
                 }
             }
+        }
+        if (CLIP && q == 0) {
+            if (lane < P.K) atomicAdd(&P.err_sum[lane], dacc0 * (double)P.norm2);
+            if (lane + 32 < P.K) atomicAdd(&P.err_sum[lane + 32], dacc1 * (double)P.norm2);
         }
     }
 
@@ -306,61 +402,108 @@ bool gbs_tc_uv_supported(const gbs_plan* p)
     return get_encode() != nullptr && p->smem_optin >= (int)(sizeof(Smem) + 1024);
 }
 
-int gbs_tc_uv_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
-                              float* scales, float* y_opt, cudaStream_t stream)
+namespace {
+
+// Tensor map of the rows and the parameters common to both uses of the kernel.
+int uv_prepare(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, CUtensorMap* tmap, UvParams* P)
 {
     EncodeTiledFn encode = get_encode();
     if (!encode) return (int)cudaErrorNotSupported;
+    if (n_rows > (int64_t)0x7fffffff - TOK) return (int)cudaErrorInvalidValue;      // TMA coordinates are 32-bit
     const int U = p->d_pad / V;
-    CUtensorMap tmap;
     const cuuint64_t gdim[3] = {(cuuint64_t)V, (cuuint64_t)(p->d / V), (cuuint64_t)n_rows};
     const cuuint64_t gstr[2] = {(cuuint64_t)(V * 2), (cuuint64_t)(stride * 2)};
     const cuuint32_t box[3] = {V, (cuuint32_t)U, TOK};
     const cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), gdim, gstr, box, estr,
+    CUresult r = encode(tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), gdim, gstr, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return (int)cudaErrorInvalidValue;
+    memset(P, 0, sizeof(*P));
+    P->n_rows = n_rows;
+    P->n_groups = (int)((n_rows + TOK - 1) / TOK);
+    P->U = U;
+    P->j = p->k - 5;
+    P->ksteps = U / 16;
+    P->code_row_bytes = p->d_pad * p->bits / 8;
+    P->d_pad = p->d_pad;
+    P->glog = p->group ? ilog2(p->group / V) : 0;
+    P->spr = p->group ? p->d_pad / p->group : 1;
+    P->c_scale = p->c_scale;
+    P->c_half = (float)(1.0 / (2.0 * (double)p->alpha));
+    P->norm = p->norm;
+    P->a_img = p->d_aimg;
+    P->status = p->d_status;
+    P->levels = p->levels;
+    P->norm2 = (float)(1.0 / (double)p->d_pad);
+    return 0;
+}
 
+// opt in to the large dynamic shared memory once per device (not a stream operation)
+cudaError_t uv_opt_in(const gbs_plan* p, int smem)
+{
+    static bool attr_done[64] = {false};
+    if (p->device >= 0 && p->device < 64 && attr_done[p->device]) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(k_tc_uv_rq<3, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<4, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<3, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<4, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<4, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<4, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess && p->device >= 0 && p->device < 64) attr_done[p->device] = true;
+    return e;
+}
+
+}  // namespace
+
+int gbs_tc_uv_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
+                              float* scales, float* y_opt, cudaStream_t stream)
+{
+    CUtensorMap tmap;
     UvParams P;
-    P.n_rows = n_rows;
-    P.n_groups = (int)((n_rows + TOK - 1) / TOK);
-    P.U = U;
-    P.j = p->k - 5;
-    P.ksteps = U / 16;
-    P.code_row_bytes = p->d_pad * p->bits / 8;
-    P.d_pad = p->d_pad;
-    P.glog = p->group ? ilog2(p->group / V) : 0;
-    P.spr = p->group ? p->d_pad / p->group : 1;
-    P.c_scale = p->c_scale;
-    P.c_half = (float)(1.0 / (2.0 * (double)p->alpha));
-    P.norm = p->norm;
-    P.a_img = p->d_aimg;
+    int rc = uv_prepare(p, x, n_rows, stride, &tmap, &P);
+    if (rc != 0) return rc;
     P.codes = (unsigned char*)codes;
     P.scales = scales;
     P.y_opt = y_opt;
-    P.status = p->d_status;
     const int smem = (int)sizeof(Smem) + 1024;
     const int grid = P.n_groups < p->sm_count ? P.n_groups : p->sm_count;
-    // opt in to the large dynamic shared memory once per device (not a stream operation)
-    static bool attr_done[64] = {false};
-    cudaError_t e = cudaSuccess;
-    if (p->device < 0 || p->device >= 64 || !attr_done[p->device]) {
-        e = cudaFuncSetAttribute(k_tc_uv_rq<3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return (int)e;
-        if (p->device >= 0 && p->device < 64) attr_done[p->device] = true;
-    }
+    cudaError_t e = uv_opt_in(p, smem);
+    if (e != cudaSuccess) return (int)e;
     const bool pdl = p->pdl != 0;
     if (p->group) {
-        if (p->bits == 3) e = launch(k_tc_uv_rq<3, true>, grid, smem, stream, pdl, tmap, P);
-        else e = launch(k_tc_uv_rq<4, true>, grid, smem, stream, pdl, tmap, P);
+        if (p->bits == 3) e = launch(k_tc_uv_rq<3, true, false>, grid, smem, stream, pdl, tmap, P);
+        else e = launch(k_tc_uv_rq<4, true, false>, grid, smem, stream, pdl, tmap, P);
     } else {
-        if (p->bits == 3) e = launch(k_tc_uv_rq<3, false>, grid, smem, stream, pdl, tmap, P);
-        else e = launch(k_tc_uv_rq<4, false>, grid, smem, stream, pdl, tmap, P);
+        if (p->bits == 3) e = launch(k_tc_uv_rq<3, false, false>, grid, smem, stream, pdl, tmap, P);
+        else e = launch(k_tc_uv_rq<4, false, false>, grid, smem, stream, pdl, tmap, P);
     }
+    return (int)e;
+}
+
+// Clip-ratio scoring on the same front end: rotate on the tensor cores, keep the rotated values in
+// registers, score all K candidates from there.
+int gbs_tc_uv_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, const float* alphas, int K,
+                         double* err_sum, float* err_rows, cudaStream_t stream)
+{
+    CUtensorMap tmap;
+    UvParams P;
+    int rc = uv_prepare(p, x, n_rows, stride, &tmap, &P);
+    if (rc != 0) return rc;
+    P.K = K;
+    for (int i = 0; i < K; ++i) {
+        P.clip_half[i] = (float)(1.0 / (2.0 * (double)alphas[i]));
+        P.clip_scale[i] = (float)((double)alphas[i] / (double)p->levels);
+    }
+    P.err_sum = err_sum;
+    P.err_rows = err_rows;
+    const int smem = (int)sizeof(Smem) + 1024;
+    const int grid = P.n_groups < p->sm_count ? P.n_groups : p->sm_count;
+    cudaError_t e = uv_opt_in(p, smem);
+    if (e != cudaSuccess) return (int)e;
+    const bool pdl = p->pdl != 0;
+    if (p->group) e = launch(k_tc_uv_rq<4, true, true>, grid, smem, stream, pdl, tmap, P);
+    else e = launch(k_tc_uv_rq<4, false, true>, grid, smem, stream, pdl, tmap, P);
     return (int)e;
 }
 
