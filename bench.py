@@ -38,7 +38,7 @@ HEADLINE = "llama4096"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused kernel on the headline
 # workload, from the ncu capture summarised under profiles/ (None until a capture exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 33_610_240   # reads 33.61 MB; the codes are still in L2 when the kernel ends
 
 
 def algorithmic_bytes(n_rows: int, d: int, d_pad: int, bits: int, group: int, in_bytes: int) -> int:
@@ -268,6 +268,9 @@ def main():
     ap.add_argument("--nsets", type=int, default=16)
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-extras", action="store_true", help="skip the context legs under `also`")
+    ap.add_argument("--profile", default=None, metavar="WORKLOAD[:ROWS]",
+                    help="launch one workload's kernel a few times and exit (for ncu captures), e.g. kv128:262144, "
+                         "clip:8192")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
@@ -295,6 +298,10 @@ def main():
     from paper_2504_13989_b200 import Plan, synth
     from paper_2504_13989_b200 import build as gbs_build
     gbs_build.build()
+
+    if args.profile:
+        run_profile(args.profile, device)
+        return
 
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -395,6 +402,27 @@ def main():
         torch.distributed.destroy_process_group()
 
 
+def run_profile(spec, device):
+    """A few launches of one kernel on a small case, for an ncu capture (prints nothing a result line would)."""
+    from paper_2504_13989_b200 import Plan, synth
+    name, _, rows = spec.partition(":")
+    clip = name == "clip"
+    w = synth.WORKLOADS["calib4096" if clip else name]
+    n = int(rows) if rows else min(w.n_rows, 8192)
+    bits = w.bits[0]
+    x = synth.make_device(w.name, n, device=str(device))
+    pl = Plan(w.d, w.d_pad, w.m, bits, w.group, w.alpha)
+    outs = pl.alloc_outputs(n, device)
+    err = torch.zeros(32, dtype=torch.float64, device=device)
+    for _ in range(6):
+        if clip:
+            pl.clip_error(x, np.linspace(0.5, 1.0, 32), err_sum=err)
+        else:
+            pl.rotate_quantize(x, out=outs)
+    torch.cuda.synchronize()
+    print(json.dumps({"profile": spec, "rows": n, "kernel_family": pl.info.variant, "status": pl.device_status()}))
+
+
 def extras(device, stream, args, peak):
     """Context figures for the other workloads / entry points (not part of the K timed steps)."""
     from paper_2504_13989_b200 import Plan, synth
@@ -414,23 +442,34 @@ def extras(device, stream, args, peak):
         stream.synchronize()
         return a.elapsed_time(b) / iters
 
-    # per-bit figures of the headline workload and the d=3584 workload (graph replay, rotating sets)
-    for name in ("llama4096", "qwen3584"):
+    # per-bit figures of every rotate-quantize workload (graph replay, rotating buffer sets > 4x L2)
+    for name in ("llama4096", "qwen3584", "mlp18944", "kv128"):
         w = synth.WORKLOADS[name]
-        xb = synth.make_host(name)
+        xb = synth.make_host(name) if name != "kv128" else synth.make_device(name, device=str(device))
         for b in w.bits:
             pl = Plan(w.d, w.d_pad, w.m, b, w.group, w.alpha)
             nbytes = algorithmic_bytes(w.n_rows, w.d, w.d_pad, b, w.group, 2)
-            nsets = max(4, int(4 * 126e6 / (nbytes + 1)) + 1)
+            nsets = max(2, min(16, int(4 * 126e6 / (nbytes + 1)) + 1))
             sets = build_sets([pl], xb, nsets, device)
-            iters = 20 * nsets
+            iters = max(2 * nsets, min(20 * nsets, int(20e-3 / (nbytes / 5e12)) // nsets * nsets))
             ms = timed_graph_loop([pl], sets, iters, 3, stream, False) / iters
             out["%s_b%d" % (name, b)] = {"us_per_launch": ms * 1e3, "gbs": nbytes / ms / 1e6,
                                          "frac_of_measured": nbytes / ms / 1e6 / peak,
                                          "frac_of_8000": nbytes / ms / 1e6 / 8000.0,
-                                         "mtokens_per_s": w.n_rows / ms / 1e3}
+                                         "mrows_per_s": w.n_rows / ms / 1e3, "kernel_family": pl.info.variant}
             del sets, pl
         del xb
+        torch.cuda.empty_cache()
+    # steady state of the d=4096 kernel: 65536 tokens per launch (the batch tiled 16 times)
+    w = synth.WORKLOADS["llama4096"]
+    xb = synth.make_host("llama4096").repeat(16, 1)
+    pl = Plan(w.d, w.d_pad, w.m, 3, w.group, w.alpha)
+    nbytes = algorithmic_bytes(xb.shape[0], w.d, w.d_pad, 3, w.group, 2)
+    sets = build_sets([pl], xb, 2, device)
+    ms = timed_graph_loop([pl], sets, 20, 3, stream, False) / 20
+    out["llama4096_b3_65536rows"] = {"us_per_launch": ms * 1e3, "gbs": nbytes / ms / 1e6,
+                                     "frac_of_measured": nbytes / ms / 1e6 / peak}
+    del sets, pl, xb
     torch.cuda.empty_cache()
     # dequantize and clip-error on the headline workload
     w = synth.WORKLOADS["llama4096"]
@@ -441,12 +480,22 @@ def extras(device, stream, args, peak):
     ms = time_loop(lambda i: pl.dequantize(codes, scales, out=yhat, stream=stream), 50)
     dq_bytes = w.n_rows * (w.d_pad * 3 // 8 + 4 + w.d_pad * 2)
     out["dequantize_b3_bf16"] = {"us_per_launch": ms * 1e3, "gbs": dq_bytes / ms / 1e6}
+    # clip-ratio scoring, K = 32, on a 32768-token sample of one calibration layer (262144 tokens x 4096)
+    del x, codes, scales, yhat
+    wc = synth.WORKLOADS["calib4096"]
+    xc = synth.make_device("calib4096", 32768, device=str(device))
     alphas = np.linspace(0.5, 1.0, 32)
     err = torch.zeros(32, dtype=torch.float64, device=device)
-    ms = time_loop(lambda i: pl.clip_error(x, alphas, err_sum=err, stream=stream), 5)
-    evals = w.n_rows * w.d_pad * 32
+    ms = time_loop(lambda i: pl.clip_error(xc, alphas, err_sum=err, stream=stream), 5)
+    evals = 32768 * wc.d_pad * 32
+    sm_clock_hz = 1.965e9
+    alu_peak = 148 * 128 * sm_clock_hz                  # fp32 lanes x clock: lane-operations per second
     out["clip_error_K32"] = {"us_per_launch": ms * 1e3, "gevals_per_s": evals / ms / 1e6,
-                             "mtokens_per_s": w.n_rows / ms / 1e3}
+                             "ms_per_layer_262144_tokens": ms * 8, "mtokens_per_s": 32768 / ms / 1e3,
+                             "roofline": {"bound": "alu", "unit": "Glane-op/s", "achieved": 5 * evals / ms / 1e6,
+                                          "peak": alu_peak / 1e9, "frac": 5 * evals / ms / 1e6 / (alu_peak / 1e9),
+                                          "note": "5 fp32 operations per value and candidate; peak = 148 SMs x 128 "
+                                                  "lanes x 1.965 GHz"}}
     return out
 
 
