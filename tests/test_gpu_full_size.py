@@ -1,0 +1,81 @@
+"""GPU parity at the full workload sizes, in the launch configuration the benchmark times (the plans the
+benchmark builds, whole batches, no optional rotated output): every row where the oracle finishes in
+seconds, sampled rows where the tensor is too large, plus properties that hold at any size."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2504_13989_b200 import Plan, synth
+from paper_2504_13989_b200 import build as gbs_build
+from parity_util import TOL_CLIP, TOL_SCALE, compare_rotate_quantize, oracle_rq, unpack_codes
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    gbs_build.build()
+
+
+@pytest.mark.parametrize("name", ["llama4096", "qwen3584", "mlp18944"])
+def test_full_batch_every_row(name):
+    w = synth.WORKLOADS[name]
+    x = synth.make_host(name)
+    xd = x.to(DEV)
+    for bits in w.bits:
+        ref = oracle_rq(x, w, bits)
+        with Plan(w.d, w.d_pad, w.m, bits, w.group, w.alpha) as plan:
+            codes, scales, _ = plan.rotate_quantize(xd)
+            torch.cuda.synchronize()
+            assert plan.device_status() == 0
+            stats = compare_rotate_quantize(x, ref, codes, scales, None, bits, w.group, w.d_pad)
+            print(name, bits, stats)
+
+
+def test_kv_tensor_sampled_rows_and_code_range():
+    """Both KV tensors' worth of rows (2 097 152 x 128) in one launch; the oracle checks the first and
+    last tiles and every 257th row; every code of every row must lie in [-D, D]."""
+    w = synth.WORKLOADS["kv128"]
+    x = synth.make_device("kv128", device=DEV)
+    n = x.shape[0]
+    with Plan(w.d, w.d_pad, w.m, 3, w.group, w.alpha) as plan:
+        assert plan.info.variant == 2
+        codes, scales, _ = plan.rotate_quantize(x)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+        idx = torch.unique(torch.cat([torch.arange(0, 256), torch.arange(n - 300, n), torch.arange(0, n, 257)]))
+        xs = x[idx.to(DEV)].cpu()
+        ref = oracle_rq(xs, w, 3)
+        compare_rotate_quantize(xs, ref, codes[idx.to(DEV)], scales[idx.to(DEV)], None, 3, w.group, w.d_pad)
+        # any size: 3-bit fields never hold the pattern 100 (= -4), i.e. codes stay in [-3, 3]
+        c = codes.view(-1, 3).to(torch.int32)
+        word = c[:, 0] | (c[:, 1] << 8) | (c[:, 2] << 16)
+        bad = torch.zeros((), dtype=torch.bool, device=DEV)
+        for e in range(8):
+            bad |= (((word >> (3 * e)) & 7) == 4).any()
+        assert not bool(bad)
+        # alpha = 1: each row's largest code magnitude is D wherever the row is not all zero
+        assert bool((scales >= 0).all())
+
+
+def test_calibration_layer_clip_error_sampled_rows():
+    """One calibration layer's scoring call at K = 32 on 65 536 tokens of the layer; per-row errors of
+    sampled rows against the oracle, and the fp64 totals against the sum of the kernel's own rows."""
+    w = synth.WORKLOADS["calib4096"]
+    n = 65536
+    x = synth.make_device("calib4096", n, device=DEV)
+    alphas = np.linspace(0.5, 1.0, 32)
+    with Plan(w.d, w.d_pad, w.m, 3, w.group, w.alpha) as plan:
+        err, rows = plan.clip_error(x, alphas, want_rows=True)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+        idx = torch.arange(0, n, 331)
+        xs = x[idx.to(DEV)].cpu()
+        eref, rref = oracle.clip_error_rows(synth.to_oracle_array(xs), w.d, w.d_pad, w.m, 3, w.group, alphas,
+                                            want_rows=True)
+        np.testing.assert_allclose(rows[idx.to(DEV)].cpu().double().numpy(), rref, rtol=1e-4, atol=1e-12)
+        np.testing.assert_allclose(err.cpu().numpy(), rows.double().sum(dim=0).cpu().numpy(), rtol=TOL_CLIP)
+        # the sampled rows' totals agree with the oracle's totals to the tolerance of the sums
+        np.testing.assert_allclose(rows[idx.to(DEV)].double().sum(dim=0).cpu().numpy(), eref, rtol=TOL_CLIP)
