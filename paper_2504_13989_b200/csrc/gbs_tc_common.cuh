@@ -258,20 +258,18 @@ __device__ __forceinline__ void quantize_pack32(const unsigned r[32], float a1, 
 {
     const float twoD = (float)(2 * ((1 << (BITS - 1)) - 1));
     const float MAGIC = 8388609.f;                        // 2^23 + 1
-    const f32x2 twoD2 = pk(__float_as_uint(twoD), __float_as_uint(twoD));
-    const f32x2 magic2 = pk(__float_as_uint(MAGIC), __float_as_uint(MAGIC));
     unsigned acc[4];
 #pragma unroll
     for (int g = 0; g < 4; ++g) {
         unsigned a = 0;
 #pragma unroll
-        for (int e = 0; e < 8; e += 2) {
-            const float w0 = __saturatef(fmaf(__uint_as_float(r[8 * g + e]), a1, 0.5f));
-            const float w1 = __saturatef(fmaf(__uint_as_float(r[8 * g + e + 1]), a1, 0.5f));
-            unsigned s0, s1;
-            unpk(fma2(pk(__float_as_uint(w0), __float_as_uint(w1)), twoD2, magic2), s0, s1);
-            a += s0 << (BITS * e);
-            a += s1 << (BITS * (e + 1));
+        for (int e = 0; e < 8; ++e) {
+            const float w = __saturatef(fmaf(__uint_as_float(r[8 * g + e]), a1, 0.5f));
+            const unsigned s = __float_as_uint(fmaf(w, twoD, MAGIC));
+            // shift on the integer pipe (funnel shift), so that the FP32 pipe only sees the two FMAs
+            unsigned t;
+            asm("shf.l.clamp.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(0u), "r"(s), "r"((unsigned)(BITS * e)));
+            a += t;
         }
         acc[g] = a;
     }

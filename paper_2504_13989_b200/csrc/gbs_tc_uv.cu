@@ -243,8 +243,17 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
         const int up = q * 32 + lane;             // u' : this thread owns outputs [up*32, up*32+32)
         const unsigned taddr0 = tmem_base + ((unsigned)(q * 32) << 16) + t * V;
         double dacc0 = 0.0, dacc1 = 0.0;          // CLIP, quadrant-0 warps: totals of candidates lane, lane + 32
+        // output cursors of this thread, advanced by one grid stride of token groups per iteration
+        const bool lane_live = up < P.U;
+        const long long row_step = (long long)gridDim.x * TOK;
+        long long row = (long long)blockIdx.x * TOK + t;
+        unsigned char* cptr = P.codes + row * P.code_row_bytes + up * (V * BITS / 8);
+        const long long cstep = row_step * P.code_row_bytes;
+        float* sptr = P.scales + row * P.spr + (GROUPED ? (up >> P.glog) : 0);
+        const long long sstep = row_step * P.spr;
+        const bool scale_writer = GROUPED ? ((lane & ((1 << P.glog) - 1)) == 0) : (up == 0);
         int it = 0;
-        for (long long g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it) {
+        for (long long g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it, row += row_step, cptr += cstep, sptr += sstep) {
             const int s = it % STAGES;
             const unsigned ph = (it / STAGES) & 1;
             const bool ok = mbar_wait(&S->abort_flag, &S->tfull[s], ph, P.status, 4, false);
@@ -261,7 +270,6 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
                 if (lane == 0) mbar_arrive(&S->tempty[s]);
                 M = fwht32_absmax(r);
             }
-            const long long row = g * TOK + t;
             const unsigned gp = it & 1;
             if (GROUPED) {
                 for (int o = (1 << P.glog) >> 1; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
@@ -297,21 +305,17 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
                 }
                 continue;
             }
-            if (row < P.n_rows && up < P.U) {
-                const float a1 = (M > 0.f) ? (P.c_half / M) : 0.f;
+            if (lane_live && row < P.n_rows) {
+                const float a1 = (M > 0.f) ? __fdividef(P.c_half, M) : 0.f;
                 unsigned out[BITS];
                 quantize_pack32<BITS>(r, a1, out);
-                unsigned* dst = reinterpret_cast<unsigned*>(P.codes + row * P.code_row_bytes + up * (V * BITS / 8));
+                unsigned* dst = reinterpret_cast<unsigned*>(cptr);
                 if (BITS == 4) {
                     *reinterpret_cast<uint4*>(dst) = make_uint4(out[0], out[1], out[2], out[3]);
                 } else {
                     dst[0] = out[0]; dst[1] = out[1]; dst[2] = out[2];
                 }
-                if (GROUPED) {
-                    if ((lane & ((1 << P.glog) - 1)) == 0) P.scales[row * P.spr + (up >> P.glog)] = P.c_scale * M;
-                } else {
-                    if (up == 0) P.scales[row] = P.c_scale * M;
-                }
+                if (scale_writer) *sptr = P.c_scale * M;
                 if (P.y_opt) {
                     float4* yo = reinterpret_cast<float4*>(P.y_opt + row * (long long)P.d_pad + up * V);
 #pragma unroll
