@@ -74,7 +74,9 @@ typedef struct gbs_plan_info {
     int variant;                   /* kernel family chosen for bf16 rows: 0 = generic shared-memory path,
                                       1 = tensor-core path for d' = 32 * U with U = m * 2^j <= 128, U % 16 == 0,
                                       d % 32 == 0 and group in {0, 32 .. 1024}, 2 = tensor-core path for
-                                      d' = 128 rows (m = 1, group in {0, 32, 64, 128}) (set GBS_FORCE_GENERIC=1 in the
+                                      d' = 128 rows (m = 1, group in {0, 32, 64, 128}), 3 = tensor-core path for
+                                      4096 < d' = 32 * G * U <= 32768 (G in {2, 4, 8}, U as above, per-token
+                                      scales, d a multiple of 32 * G) (set GBS_FORCE_GENERIC=1 in the
                                       environment before gbs_plan_create to force 0; GBS_NO_PDL=1 launches it
                                       without programmatic stream serialization) */
 } gbs_plan_info_t;

@@ -119,11 +119,13 @@ extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bi
     const bool want_tc = !(force && force[0] == '1');
     const bool tc_uv = want_tc && gbs_tc_uv_supported(p);
     const bool tc_row = want_tc && !tc_uv && gbs_tc_row_supported(p);
-    if (tc_uv || tc_row) {
+    const int uvm_glog = (want_tc && !tc_uv && !tc_row) ? gbs_tc_uvm_glog(p) : 0;
+    if (tc_uv || tc_row || uvm_glog) {
         unsigned char* img = (unsigned char*)malloc(32768);
         if (!img) { cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC; }
         if (tc_uv) gbs_tc_uv_a_image(p, img);
-        else gbs_tc_sign_image(p->h_hm, 1, 7, 128, img);                 // H_128 itself
+        else if (tc_row) gbs_tc_sign_image(p->h_hm, 1, 7, 128, img);     // H_128 itself
+        else gbs_tc_sign_image(p->h_hm, p->m, p->k - 5 - uvm_glog, p->d_pad >> (5 + uvm_glog), img);
         e = cudaMalloc(&p->d_aimg, 32768);
         if (e == cudaSuccess) e = cudaMemcpy(p->d_aimg, img, 32768, cudaMemcpyHostToDevice);
         free(img);
@@ -132,7 +134,8 @@ extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bi
             if (p->d_aimg) cudaFree(p->d_aimg);
             cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC;
         }
-        p->variant = tc_uv ? GBS_VARIANT_TC_UV : GBS_VARIANT_TC_ROW;
+        p->variant = tc_uv ? GBS_VARIANT_TC_UV : (tc_row ? GBS_VARIANT_TC_ROW : GBS_VARIANT_TC_UVM);
+        p->uvm_glog = uvm_glog;
     }
     const char* nopdl = getenv("GBS_NO_PDL");
     p->pdl = (nopdl && nopdl[0] == '1') ? 0 : 1;
@@ -212,6 +215,8 @@ extern "C" int gbs_rotate_quantize(const gbs_plan_t* p, const void* x, int x_dty
     int e;
     if (p->variant == GBS_VARIANT_TC_UV && x_dtype == GBS_DTYPE_BF16)
         e = gbs_tc_uv_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
+    else if (p->variant == GBS_VARIANT_TC_UVM && x_dtype == GBS_DTYPE_BF16)
+        e = gbs_tc_uvm_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
     else if (p->variant == GBS_VARIANT_TC_ROW && x_dtype == GBS_DTYPE_BF16)
         e = gbs_tc_row_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
     else

@@ -9,6 +9,7 @@
 // Kernel families a plan can select for bf16 rows.
 enum gbs_variant {
     GBS_VARIANT_GENERIC = 0,   // shared-memory FWHT on the plain ALUs; any supported (m, k), any dtype
+    GBS_VARIANT_TC_UVM = 3,    // 4096 < d' = 32*G*U <= 32768, G in {2,4,8}: tensor cores + two register sweeps over TMEM
     GBS_VARIANT_TC_ROW = 2,    // d' = 128 (KV rows): X * H_128 on tcgen05 tensor cores, one thread owns one row
     GBS_VARIANT_TC_UV = 1,     // d' = U*32, U = m*2^j <= 128: (H_m (x) H_{2^j}) on tcgen05 tensor cores + H_32 in
                                // registers (bf16 rows)
@@ -28,6 +29,7 @@ struct gbs_plan {
     int variant;
     float* d_hm;           // device: H_m as floats, m*m row-major, followed by H_m^T (m*m)
     int pdl;               // tensor-core families launch with programmatic stream serialization
+    int uvm_glog;          // UVM family: log2 of the number of 32-value chunks per tensor-core output row
     unsigned char* d_aimg; // device: pre-swizzled bf16 image of H_m (x) H_{2^j} for the tensor-core family (32 KB)
     int* d_status;         // device status word: 0, or the code of the first bounded wait that expired
     int8_t h_hm[32 * 32];  // host copy of H_m (m <= 32)
@@ -54,6 +56,11 @@ int gbs_tc_uv_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int64
 void gbs_tc_uv_a_image(const gbs_plan* p, unsigned char* img32k);
 // image of H_m (x) H_{2^j} (U x U inside 128 x 128, bf16 +-1, K-major, 128-byte swizzle)
 void gbs_tc_sign_image(const int8_t* hm, int m, int j, int U, unsigned char* img32k);
+
+// gbs_tc_uvm.cu
+int gbs_tc_uvm_glog(const gbs_plan* p);        // 0 if the family does not apply
+int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
+                               float* scales, float* y_opt, cudaStream_t stream);
 
 // gbs_tc_row.cu
 bool gbs_tc_row_supported(const gbs_plan* p);

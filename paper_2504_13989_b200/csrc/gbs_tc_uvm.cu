@@ -1,0 +1,434 @@
+// Tensor-core family "UVM": bf16 rows of padded width d' = U * G * 32 with U = m * 2^j <= 128 and
+// G = 2, 4 or 8 (widths 4096 < d' <= 32768, e.g. the MLP width 20480 = 20 * 1024: U = 80, G = 8).
+//
+// A padded row is viewed as X[u][c][v] (flat index (u*G + c)*32 + v).  With 2^k = 2^j * G * 32 the rotation
+// factors as (H_m (x) H_{2^j}) (x) H_G (x) H_32 (Eq. (1) on the three bit fields of the Sylvester index,
+// Algorithm 2 for H_m):
+//   * A = H_m (x) H_{2^j} (U x U, +-1) runs on the tensor cores exactly as in the UV family, one token
+//     per MMA batch, N = G*32 columns: TMEM lane u' holds G chunks of 32 consecutive coordinates.
+//   * H_32 inside each chunk and H_G across the chunks are butterflies in registers, in two sweeps over
+//     TMEM (a thread cannot hold its 256 values at once): sweep 1 transforms each chunk in place,
+//     sweep 2 loads 4 columns of every chunk, runs the G-point butterflies, takes max|.| and writes back.
+//   * sweep 3 scales, rounds, clips (Sections 2.1, 3.1) and packs each chunk; per-token scales only.
+// All sixteen epilogue warps work on the same token: warp (q, w) serves lane quadrant q, chunks w, w+4 in
+// sweeps 1 and 3, and column groups 2w, 2w+1 in sweep 2; two 512-thread named barriers separate the
+// sweeps (the second also carries the per-token maximum).  Roles, pipeline, bounded waits and teardown
+// are those of the UV family.
+#include <math.h>
+#include <string.h>
+
+#include "gbs_internal.h"
+#include "gbs_tc_common.cuh"
+
+namespace {
+
+constexpr int V = 32;
+constexpr int UMAX = 128;
+constexpr int A_BYTES = UMAX * UMAX * 2;
+constexpr int B_BYTES = 160 * 1024;               // shared memory for the row stages
+constexpr int MAX_STAGES = 4;
+constexpr int EPI_WARPS = 16;
+constexpr int THREADS = 32 * (2 + EPI_WARPS);
+constexpr int TMEM_COLS = 512;
+
+struct __align__(1024) Smem {
+    unsigned char a[A_BYTES];
+    unsigned char b[B_BYTES];
+    unsigned long long full[MAX_STAGES], empty[MAX_STAGES], tfull[MAX_STAGES], tempty[MAX_STAGES];
+    unsigned long long abar;
+    __align__(16) float red[2][EPI_WARPS];     // [iteration parity][warp]: per-warp max of the token
+    int gabort[2];                             // [iteration parity]: an epilogue warp gave up waiting
+    unsigned tmem_base;
+    volatile int abort_flag;
+};
+
+struct UvmParams {
+    long long n_rows;
+    int U;                        // m * 2^j
+    int ksteps;                   // U / 16
+    int n_stages;                 // shared-memory stages in use
+    int stage_bytes;              // U * G * 64
+    int code_row_bytes;
+    int d_pad;
+    float c_scale, c_half, norm;
+    const unsigned char* a_img;
+    unsigned char* codes;
+    float* scales;
+    float* y_opt;
+    int* status;
+};
+
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, void* bar, int c0, int c1, int c2, int c3)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tmem_ld4_issue(unsigned taddr, unsigned r[4])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x4.b32 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st4(unsigned taddr, const unsigned r[4])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x4.b32 [%4], {%0, %1, %2, %3};"
+                 ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(unsigned taddr, const unsigned r[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%32], "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31};"
+        ::"r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]),
+          "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+// H_32 on 32 registers, in place, natural order (no max: the transform is not finished yet).
+__device__ __forceinline__ void fwht32(unsigned r[32])
+{
+    f32x2 p[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) p[i] = pk(r[2 * i], r[2 * i + 1]);
+#pragma unroll
+    for (int h = 1; h < 16; h <<= 1)
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+            if ((i & h) == 0) {
+                const f32x2 a = p[i], b = p[i + h];
+                p[i] = add2(a, b);
+                p[i + h] = sub2(a, b);
+            }
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+        unsigned ua, ub;
+        unpk(p[i], ua, ub);
+        const float a = __uint_as_float(ua), b = __uint_as_float(ub);
+        r[2 * i] = __float_as_uint(a + b);
+        r[2 * i + 1] = __float_as_uint(a - b);
+    }
+}
+
+// tcgen05.wait::ld that names the loaded registers, so that nothing using them is scheduled before it
+template <int N>
+__device__ __forceinline__ void tmem_ld_wait_n(unsigned* r);
+template <>
+__device__ __forceinline__ void tmem_ld_wait_n<8>(unsigned* r)
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7])::"memory");
+}
+template <>
+__device__ __forceinline__ void tmem_ld_wait_n<16>(unsigned* r)
+{
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+                 : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+                   "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15])
+                 ::"memory");
+}
+template <>
+__device__ __forceinline__ void tmem_ld_wait_n<32>(unsigned* r)
+{
+    tmem_ld_wait(r);
+}
+
+// ---------------------------------------------------------------------------------------------
+// kernel
+// ---------------------------------------------------------------------------------------------
+template <int BITS, int GLOG>
+__global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant__ CUtensorMap tmap,
+                                                          const __grid_constant__ UvmParams P)
+{
+    constexpr int G = 1 << GLOG;                  // chunks of 32 coordinates per TMEM lane
+    constexpr int NCOLS = G * V;                  // accumulator columns per token
+    constexpr int TSTAGES = (G == 8) ? 2 : 4;     // TMEM stages
+    extern __shared__ unsigned char smem_raw[];
+    Smem* S = reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int nst = P.n_stages;
+    const int n_tok = (int)P.n_rows;
+
+    int it_p = 0;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < MAX_STAGES; ++s) mbar_init(&S->full[s], 1);
+        mbar_init(&S->abar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        mbar_arrive_expect_tx(&S->abar, A_BYTES);
+        bulk_load(S->a, P.a_img, A_BYTES, &S->abar);          // plan-owned, immutable: needs no ordering
+        asm volatile("griddepcontrol.wait;" ::: "memory");   // nothing of the caller's memory is touched before
+        for (int tk = blockIdx.x; it_p < nst && tk < n_tok; tk += gridDim.x, ++it_p) {
+            mbar_arrive_expect_tx(&S->full[it_p], (unsigned)P.stage_bytes);
+            for (int c = 0; c < G; ++c)          // one box per chunk: U rows of 32 values
+                tma_load_4d(S->b + (size_t)it_p * P.stage_bytes + (size_t)c * (P.stage_bytes >> GLOG), &tmap,
+                            &S->full[it_p], 0, c, 0, tk);
+        }
+    }
+    if (threadIdx.x == 64) {
+        for (int s = 0; s < MAX_STAGES; ++s) {
+            mbar_init(&S->empty[s], 1);
+            mbar_init(&S->tfull[s], 1);
+            mbar_init(&S->tempty[s], EPI_WARPS);
+        }
+        S->gabort[0] = S->gabort[1] = 0;
+        S->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(&S->tmem_base, TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const unsigned tmem_base = S->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------ TMA producer ------------------------------
+        if (lane == 0) {
+            int it = it_p;
+            for (int tk = blockIdx.x + it * (int)gridDim.x; tk < n_tok; tk += gridDim.x, ++it) {
+                const int s = it % nst;
+                const unsigned ph = (it / nst) & 1;
+                if (!mbar_wait(&S->abort_flag, &S->empty[s], ph ^ 1, P.status, 1)) break;
+                mbar_arrive_expect_tx(&S->full[s], (unsigned)P.stage_bytes);
+                for (int c = 0; c < G; ++c)
+                    tma_load_4d(S->b + (size_t)s * P.stage_bytes + (size_t)c * (P.stage_bytes >> GLOG), &tmap,
+                                &S->full[s], 0, c, 0, tk);
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------ MMA issuer ------------------------------
+        if (lane == 0) {
+            constexpr unsigned IDESC = instr_desc(UMAX, NCOLS);
+            const unsigned a_base = smem_u32(S->a);
+            const unsigned chunk_bytes = (unsigned)(P.U * V * 2);     // one chunk (N atom of 32): U rows of 64 bytes
+            bool ok = mbar_wait(&S->abort_flag, &S->abar, 0, P.status, 6);
+            int it = 0;
+            for (int tk = blockIdx.x; ok && tk < n_tok; tk += gridDim.x, ++it) {
+                const int s = it % nst, ts = it % TSTAGES;
+                if (!mbar_wait(&S->abort_flag, &S->full[s], (it / nst) & 1, P.status, 2)) break;
+                if (!mbar_wait(&S->abort_flag, &S->tempty[ts], ((it / TSTAGES) & 1) ^ 1, P.status, 3)) break;
+                tc_fence_after();
+                const unsigned b_base = smem_u32(S->b + (size_t)s * P.stage_bytes);
+                for (int ks = 0; ks < P.ksteps; ++ks) {
+                    const unsigned long long ad = smem_desc(a_base + (ks >> 2) * (UMAX * 128) + (ks & 3) * 32, 16, 1024, 2);
+                    const unsigned long long bd = smem_desc(b_base + ks * 1024, chunk_bytes, 512, 4);
+                    umma_f16(tmem_base + ts * NCOLS, ad, bd, IDESC, ks > 0 ? 1u : 0u);
+                }
+                umma_commit(&S->empty[s]);
+                umma_commit(&S->tfull[ts]);
+            }
+        }
+    } else {
+        // ------------------------------ epilogue ------------------------------
+        const int w = (warp - 2) >> 2;            // 0..3: which chunks / column groups this warp takes
+        const int q = warp & 3;                   // TMEM lane quadrant this warp may access
+        const int ew = warp - 2;
+        const int up = q * 32 + lane;             // u'
+        const bool quad_live = q * 32 < P.U;      // a quadrant wholly beyond U has nothing to do
+        const bool lane_live = up < P.U;
+        const unsigned tq = tmem_base + ((unsigned)(q * 32) << 16);
+        int it = 0;
+        for (long long row = blockIdx.x; row < P.n_rows; row += gridDim.x, ++it) {
+            const int ts = it % TSTAGES;
+            const unsigned gp = it & 1;
+            const bool ok = mbar_wait(&S->abort_flag, &S->tfull[ts], (it / TSTAGES) & 1, P.status, 4, false);
+            if (!ok && lane == 0) S->gabort[gp] = 1;
+            const unsigned tcol = tq + ts * NCOLS;
+            unsigned r[32];
+            // sweep 1: H_32 inside the chunks this warp owns
+            if (ok && quad_live) {
+                tc_fence_after();
+#pragma unroll
+                for (int c = w; c < G; c += 4) {
+                    tmem_ld32_issue(tcol + c * V, r);
+                    tmem_ld_wait(r);
+                    fwht32(r);
+                    tmem_st32(tcol + c * V, r);
+                }
+                tmem_wait_st();
+                tc_fence_before();
+            }
+            asm volatile("bar.sync 1, 512;" ::: "memory");
+            if (S->gabort[gp]) break;
+            // sweep 2: H_G across the chunks, four columns at a time; max|.| of the finished transform
+            float M = 0.f;
+            if (quad_live) {
+                tc_fence_after();
+#pragma unroll
+                for (int cg = 0; cg < 2; ++cg) {
+                    const unsigned col0 = tcol + (2 * w + cg) * 4;
+                    unsigned x[G * 4];
+#pragma unroll
+                    for (int c = 0; c < G; ++c) tmem_ld4_issue(col0 + c * V, x + 4 * c);
+                    tmem_ld_wait_n<G * 4>(x);
+                    f32x2 p[G * 2];
+#pragma unroll
+                    for (int i = 0; i < G * 2; ++i) p[i] = pk(x[2 * i], x[2 * i + 1]);
+#pragma unroll
+                    for (int h = 1; h < G; h <<= 1)
+#pragma unroll
+                        for (int c = 0; c < G; ++c)
+                            if ((c & h) == 0) {
+#pragma unroll
+                                for (int i = 0; i < 2; ++i) {
+                                    const f32x2 a = p[2 * c + i], b = p[2 * (c + h) + i];
+                                    p[2 * c + i] = add2(a, b);
+                                    p[2 * (c + h) + i] = sub2(a, b);
+                                }
+                            }
+#pragma unroll
+                    for (int i = 0; i < G * 2; ++i) {
+                        unpk(p[i], x[2 * i], x[2 * i + 1]);
+                        M = max3(fabsf(__uint_as_float(x[2 * i])), fabsf(__uint_as_float(x[2 * i + 1])), M);
+                    }
+#pragma unroll
+                    for (int c = 0; c < G; ++c) tmem_st4(col0 + c * V, x + 4 * c);
+                }
+                tmem_wait_st();
+                tc_fence_before();
+            }
+            const unsigned mw = __reduce_max_sync(0xffffffffu, __float_as_uint(M));
+            if (lane == 0) S->red[gp][ew] = __uint_as_float(mw);
+            asm volatile("bar.sync 1, 512;" ::: "memory");
+            {
+                const float4* rp = reinterpret_cast<const float4*>(&S->red[gp][0]);
+                const float4 m0 = rp[0], m1 = rp[1], m2 = rp[2], m3 = rp[3];
+                M = fmaxf(fmaxf(fmaxf(m0.x, m0.y), fmaxf(m0.z, m0.w)), fmaxf(fmaxf(m1.x, m1.y), fmaxf(m1.z, m1.w)));
+                M = fmaxf(M, fmaxf(fmaxf(fmaxf(m2.x, m2.y), fmaxf(m2.z, m2.w)), fmaxf(fmaxf(m3.x, m3.y), fmaxf(m3.z, m3.w))));
+            }
+            // sweep 3: Delta, round / clip, pack, store
+            const float a1 = (M > 0.f) ? __fdividef(P.c_half, M) : 0.f;
+            if (quad_live) {
+                tc_fence_after();
+#pragma unroll
+                for (int c = w; c < G; c += 4) {
+                    tmem_ld32_issue(tcol + c * V, r);
+                    tmem_ld_wait(r);
+                    if (lane_live) {
+                        unsigned out[BITS];
+                        quantize_pack32<BITS>(r, a1, out);
+                        unsigned* dst = reinterpret_cast<unsigned*>(P.codes + row * P.code_row_bytes +
+                                                                    (size_t)(up * G + c) * (V * BITS / 8));
+                        if (BITS == 4) {
+                            *reinterpret_cast<uint4*>(dst) = make_uint4(out[0], out[1], out[2], out[3]);
+                        } else {
+                            dst[0] = out[0]; dst[1] = out[1]; dst[2] = out[2];
+                        }
+                        if (P.y_opt) {
+                            float4* yo = reinterpret_cast<float4*>(P.y_opt + row * (long long)P.d_pad + (size_t)(up * G + c) * V);
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                yo[i] = make_float4(__uint_as_float(r[4 * i]) * P.norm, __uint_as_float(r[4 * i + 1]) * P.norm,
+                                                    __uint_as_float(r[4 * i + 2]) * P.norm, __uint_as_float(r[4 * i + 3]) * P.norm);
+                        }
+                    }
+                }
+                tc_fence_before();
+            }
+            if (ew == 0 && lane == 0) P.scales[row] = P.c_scale * M;
+            // the accumulators have been read for the last time: hand the TMEM stage back to the MMA issuer
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&S->tempty[ts]);
+        }
+    }
+
+    // ---- teardown: every role leaves its loop (normally or through the abort flag), then TMEM is freed
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, TMEM_COLS);
+    }
+}
+
+template <typename KernelT>
+cudaError_t launch(KernelT kernel, int grid, int smem, cudaStream_t stream, bool pdl, const CUtensorMap& tmap,
+                   const UvmParams& P)
+{
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e != cudaSuccess) return e;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, tmap, P);
+}
+
+}  // namespace
+
+// Smallest G in {2, 4, 8} for which U = d' / (32 G) fits the tensor-core factor; 0 if the family does not apply.
+int gbs_tc_uvm_glog(const gbs_plan* p)
+{
+    if (p->group != 0 || p->d_pad <= 4096) return 0;
+    for (int g = 1; g <= 3; ++g) {
+        const int span = V << g;
+        if (p->d_pad % span != 0 || p->d % span != 0) continue;
+        const int U = p->d_pad / span;
+        if (U > UMAX || U % 16 != 0 || p->k - 5 - g < 0) continue;
+        if (get_encode() == nullptr || p->smem_optin < (int)(sizeof(Smem) + 1024)) return 0;
+        return g;
+    }
+    return 0;
+}
+
+int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
+                               float* scales, float* y_opt, cudaStream_t stream)
+{
+    EncodeTiledFn encode = get_encode();
+    if (!encode) return (int)cudaErrorNotSupported;
+    if (n_rows > (int64_t)0x7fffffff - 1) return (int)cudaErrorInvalidValue;      // TMA coordinates are 32-bit
+    const int glog = p->uvm_glog, G = 1 << glog;
+    const int U = p->d_pad / (V * G);
+    // dims: v (32 values), chunk c (G), u, token; one box = chunk c of one token: U rows of 32 values
+    CUtensorMap tmap;
+    const cuuint64_t gdim[4] = {(cuuint64_t)V, (cuuint64_t)G, (cuuint64_t)(p->d / (V * G)), (cuuint64_t)n_rows};
+    const cuuint64_t gstr[3] = {(cuuint64_t)(V * 2), (cuuint64_t)(V * G * 2), (cuuint64_t)(stride * 2)};
+    const cuuint32_t box[4] = {V, 1, (cuuint32_t)U, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    CUresult r = encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x), gdim, gstr, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return (int)cudaErrorInvalidValue;
+
+    UvmParams P;
+    memset(&P, 0, sizeof(P));
+    P.n_rows = n_rows;
+    P.U = U;
+    P.ksteps = U / 16;
+    P.stage_bytes = U * G * V * 2;
+    P.n_stages = B_BYTES / P.stage_bytes < MAX_STAGES ? B_BYTES / P.stage_bytes : MAX_STAGES;
+    P.code_row_bytes = p->d_pad * p->bits / 8;
+    P.d_pad = p->d_pad;
+    P.c_scale = p->c_scale;
+    P.c_half = (float)(1.0 / (2.0 * (double)p->alpha));
+    P.norm = p->norm;
+    P.a_img = p->d_aimg;
+    P.codes = (unsigned char*)codes;
+    P.scales = scales;
+    P.y_opt = y_opt;
+    P.status = p->d_status;
+    const int smem = (int)sizeof(Smem) + 1024;
+    const int grid = (int)(n_rows < p->sm_count ? n_rows : p->sm_count);
+    const bool pdl = p->pdl != 0;
+    cudaError_t e;
+    if (p->bits == 3) {
+        if (glog == 1) e = launch(k_tc_uvm_rq<3, 1>, grid, smem, stream, pdl, tmap, P);
+        else if (glog == 2) e = launch(k_tc_uvm_rq<3, 2>, grid, smem, stream, pdl, tmap, P);
+        else e = launch(k_tc_uvm_rq<3, 3>, grid, smem, stream, pdl, tmap, P);
+    } else {
+        if (glog == 1) e = launch(k_tc_uvm_rq<4, 1>, grid, smem, stream, pdl, tmap, P);
+        else if (glog == 2) e = launch(k_tc_uvm_rq<4, 2>, grid, smem, stream, pdl, tmap, P);
+        else e = launch(k_tc_uvm_rq<4, 3>, grid, smem, stream, pdl, tmap, P);
+    }
+    return (int)e;
+}

@@ -233,6 +233,43 @@ def test_tensor_core_family_shapes(d, d_pad, m, bits, group, alpha, rows):
         np.testing.assert_allclose(erows.cpu().double().numpy(), rref, rtol=1e-4, atol=1e-12)
 
 
+UVM_SHAPES = [
+    # d, d_pad, m, bits, alpha, rows
+    (8192, 8192, 1, 3, 0.9, 149),
+    (8192 - 64, 8192, 1, 4, 0.9, 1),
+    (16384, 16384, 1, 4, 0.8, 37),
+    (16000, 16384, 1, 3, 1.0, 150),
+    (12288, 12288, 12, 3, 0.9, 75),
+    (18944, 20480, 20, 4, 0.95, 301),
+    (20480, 20480, 20, 3, 0.9, 4),
+    (24576, 24576, 24, 4, 0.9, 33),
+    (28672, 28672, 28, 3, 0.85, 150),
+    (32768, 32768, 1, 4, 0.9, 31),
+]
+
+
+@pytest.mark.parametrize("d,d_pad,m,bits,alpha,rows", UVM_SHAPES)
+def test_wide_family_shapes(d, d_pad, m, bits, alpha, rows):
+    """4096 < d' <= 32768: tensor cores for H_m (x) H_{2^j}, two register sweeps over TMEM for the rest."""
+    rng = np.random.Generator(np.random.PCG64(d * 3 + m + bits + rows))
+    xs = rng.standard_t(3, size=(rows, d))
+    xs[:, rng.integers(0, d, 3)] *= 40
+    if rows > 2:
+        xs[2, :] = 0.0
+    x = torch.from_numpy(xs.astype(np.float32)).to(torch.bfloat16)
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(x), d, d_pad, m, bits, 0, alpha)
+    with Plan(d, d_pad, m, bits, 0, alpha) as plan:
+        assert plan.info.variant == 3, "the wide tensor-core family must be the one that runs for this plan"
+        codes, scales, y = _run_rq(plan, x.to(DEV), rows)
+        assert plan.device_status() == 0
+        stats = compare_rotate_quantize(x, ref, codes, scales, y, bits, 0, d_pad)
+        print(stats)
+        if rows > 2:
+            assert int(codes[2].max()) == 0 and float(scales[2].abs().max()) == 0.0
+        codes2, scales2, _ = _run_rq(plan, x.to(DEV), rows, want_y=False)
+        assert torch.equal(codes, codes2) and torch.equal(scales, scales2)
+
+
 ROW_SHAPES = [
     # d, bits, group, alpha, rows, stride
     (128, 3, 0, 1.0, 1, 128),
