@@ -10,9 +10,10 @@
 //     TMEM (a thread cannot hold its 256 values at once): sweep 1 transforms each chunk in place,
 //     sweep 2 loads 4 columns of every chunk, runs the G-point butterflies, takes max|.| and writes back.
 //   * sweep 3 scales, rounds, clips (Sections 2.1, 3.1) and packs each chunk; per-token scales only.
-// All sixteen epilogue warps work on the same token: warp (q, w) serves lane quadrant q, chunks w, w+4 in
-// sweeps 1 and 3, and column groups 2w, 2w+1 in sweep 2; two 512-thread named barriers separate the
-// sweeps (the second also carries the per-token maximum).  Roles, pipeline, bounded waits and teardown
+// The sixteen epilogue warps form two groups of eight that take alternate tokens (so that one group's
+// barrier waits are filled by the other's arithmetic): in a group, warp (q, w) serves lane quadrant q,
+// chunks w, w+2, .. in sweeps 1 and 3 and column groups 4w .. 4w+3 in sweep 2; two 256-thread named
+// barriers per token separate the sweeps (the second also carries the per-token maximum).  Roles, pipeline, bounded waits and teardown
 // are those of the UV family.
 #include <math.h>
 #include <string.h>
@@ -36,8 +37,8 @@ struct __align__(1024) Smem {
     unsigned char b[B_BYTES];
     unsigned long long full[MAX_STAGES], empty[MAX_STAGES], tfull[MAX_STAGES], tempty[MAX_STAGES];
     unsigned long long abar;
-    __align__(16) float red[2][EPI_WARPS];     // [iteration parity][warp]: per-warp max of the token
-    int gabort[2];                             // [iteration parity]: an epilogue warp gave up waiting
+    __align__(16) float red[2][2][8];          // [group][iteration parity][warp of the group]: max of the token
+    int gabort[2][2];                          // [group][iteration parity]: a warp of the group gave up waiting
     unsigned tmem_base;
     volatile int abort_flag;
 };
@@ -172,9 +173,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
         for (int s = 0; s < MAX_STAGES; ++s) {
             mbar_init(&S->empty[s], 1);
             mbar_init(&S->tfull[s], 1);
-            mbar_init(&S->tempty[s], EPI_WARPS);
+            mbar_init(&S->tempty[s], EPI_WARPS / 2);
         }
-        S->gabort[0] = S->gabort[1] = 0;
+        S->gabort[0][0] = S->gabort[0][1] = S->gabort[1][0] = S->gabort[1][1] = 0;
         S->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -224,26 +225,28 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
         }
     } else {
         // ------------------------------ epilogue ------------------------------
-        const int w = (warp - 2) >> 2;            // 0..3: which chunks / column groups this warp takes
+        const int grp = (warp - 2) >> 3;          // group: takes tokens it = grp, grp + 2, ..
+        const int w = ((warp - 2) >> 2) & 1;      // which chunks / column groups of the token this warp takes
         const int q = warp & 3;                   // TMEM lane quadrant this warp may access
-        const int ew = warp - 2;
+        const int ew = w * 4 + q;                 // index inside the group
         const int up = q * 32 + lane;             // u'
         const bool quad_live = q * 32 < P.U;      // a quadrant wholly beyond U has nothing to do
         const bool lane_live = up < P.U;
         const unsigned tq = tmem_base + ((unsigned)(q * 32) << 16);
-        int it = 0;
-        for (long long row = blockIdx.x; row < P.n_rows; row += gridDim.x, ++it) {
+        int it = grp, n = 0;
+        for (long long row = (long long)blockIdx.x + (long long)grp * gridDim.x; row < P.n_rows;
+             row += 2ll * gridDim.x, it += 2, ++n) {
             const int ts = it % TSTAGES;
-            const unsigned gp = it & 1;
+            const unsigned gp = n & 1;
             const bool ok = mbar_wait(&S->abort_flag, &S->tfull[ts], (it / TSTAGES) & 1, P.status, 4, false);
-            if (!ok && lane == 0) S->gabort[gp] = 1;
+            if (!ok && lane == 0) S->gabort[grp][gp] = 1;
             const unsigned tcol = tq + ts * NCOLS;
             unsigned r[32];
             // sweep 1: H_32 inside the chunks this warp owns
             if (ok && quad_live) {
                 tc_fence_after();
 #pragma unroll
-                for (int c = w; c < G; c += 4) {
+                for (int c = w; c < G; c += 2) {
                     tmem_ld32_issue(tcol + c * V, r);
                     tmem_ld_wait(r);
                     fwht32(r);
@@ -252,15 +255,15 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
                 tmem_wait_st();
                 tc_fence_before();
             }
-            asm volatile("bar.sync 1, 512;" ::: "memory");
-            if (S->gabort[gp]) break;
+            asm volatile("bar.sync %0, 256;" ::"r"(1 + grp) : "memory");
+            if (S->gabort[grp][gp]) break;
             // sweep 2: H_G across the chunks, four columns at a time; max|.| of the finished transform
             float M = 0.f;
             if (quad_live) {
                 tc_fence_after();
 #pragma unroll
-                for (int cg = 0; cg < 2; ++cg) {
-                    const unsigned col0 = tcol + (2 * w + cg) * 4;
+                for (int cg = 0; cg < 4; ++cg) {
+                    const unsigned col0 = tcol + (4 * w + cg) * 4;
                     unsigned x[G * 4];
 #pragma unroll
                     for (int c = 0; c < G; ++c) tmem_ld4_issue(col0 + c * V, x + 4 * c);
@@ -292,20 +295,19 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
                 tc_fence_before();
             }
             const unsigned mw = __reduce_max_sync(0xffffffffu, __float_as_uint(M));
-            if (lane == 0) S->red[gp][ew] = __uint_as_float(mw);
-            asm volatile("bar.sync 1, 512;" ::: "memory");
+            if (lane == 0) S->red[grp][gp][ew] = __uint_as_float(mw);
+            asm volatile("bar.sync %0, 256;" ::"r"(1 + grp) : "memory");
             {
-                const float4* rp = reinterpret_cast<const float4*>(&S->red[gp][0]);
-                const float4 m0 = rp[0], m1 = rp[1], m2 = rp[2], m3 = rp[3];
+                const float4* rp = reinterpret_cast<const float4*>(&S->red[grp][gp][0]);
+                const float4 m0 = rp[0], m1 = rp[1];
                 M = fmaxf(fmaxf(fmaxf(m0.x, m0.y), fmaxf(m0.z, m0.w)), fmaxf(fmaxf(m1.x, m1.y), fmaxf(m1.z, m1.w)));
-                M = fmaxf(M, fmaxf(fmaxf(fmaxf(m2.x, m2.y), fmaxf(m2.z, m2.w)), fmaxf(fmaxf(m3.x, m3.y), fmaxf(m3.z, m3.w))));
             }
             // sweep 3: Delta, round / clip, pack, store
             const float a1 = (M > 0.f) ? __fdividef(P.c_half, M) : 0.f;
             if (quad_live) {
                 tc_fence_after();
 #pragma unroll
-                for (int c = w; c < G; c += 4) {
+                for (int c = w; c < G; c += 2) {
                     tmem_ld32_issue(tcol + c * V, r);
                     tmem_ld_wait(r);
                     if (lane_live) {
