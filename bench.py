@@ -496,6 +496,13 @@ def extras(device, stream, args, peak):
                                           "peak": alu_peak / 1e9, "frac": 5 * evals / ms / 1e6 / (alu_peak / 1e9),
                                           "note": "5 fp32 operations per value and candidate; peak = 148 SMs x 128 "
                                                   "lanes x 1.965 GHz"}}
+    # Algorithm 1's bracket search on the same sample (eps = 1/64): rounds of <= 31 probes, blocking
+    t0 = time.perf_counter()
+    res = pl.search_clip_ratio(xc, 1.0 / 64, stream=stream)
+    dt = time.perf_counter() - t0
+    out["search_clip_ratio_eps_1_64"] = {"alpha": res.alpha, "iterations": res.iterations, "rounds": res.rounds,
+                                         "evaluations": res.evaluations, "wall_ms": dt * 1e3,
+                                         "wall_ms_per_layer_262144_tokens": dt * 8e3}
     return out
 
 

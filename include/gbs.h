@@ -188,6 +188,37 @@ int gbs_clip_error(const gbs_plan_t* plan, const void* x, int x_dtype, int64_t n
                    float* err_rows_opt, void* cuda_stream);
 
 /*
+ * Result of gbs_search_clip_ratio (host memory).
+ */
+typedef struct gbs_search_result {
+    float alpha;        /* the clip ratio kept at the end (m of Algorithm 1)                       */
+    float a, b;         /* the final bracket, b - a <= eps                                          */
+    double err;         /* the objective at alpha: sum over rows and coordinates of (y - yhat)^2   */
+    int iterations;     /* passes through the loop body of Algorithm 1                              */
+    int evaluations;    /* objective values the algorithm consumed: iterations + 1                  */
+    int rounds;         /* gbs_clip_error launches used to obtain them                              */
+} gbs_search_result_t;
+
+/*
+ * The bracket search of Algorithm 1 (Gradual Binary Search, the loop for one projection) for the clip
+ * ratio of the rows in x, with the quantization error of gbs_clip_error as the objective (the paper
+ * minimises perplexity; this library has no model to evaluate, Sections 3.1 and 4.1).
+ * Start a = 0, b = 1, m = 1/2; on even iterations probe (a+m)/2, on odd ones (b+m)/2; a probe that
+ * lowers the objective becomes the new m and halves the bracket towards it, otherwise the bracket end
+ * on the probe's side moves to the probe; stop when b - a <= eps.  The states visited are those of the
+ * algorithm as printed; evaluations are grouped: each round scores the probes of the next five
+ * iterations' decision tree (at most 31 clip ratios) in one gbs_clip_error launch.
+ *   x, x_dtype, n_rows, x_row_stride   as for gbs_clip_error (n_rows >= 1)
+ *   eps        0 < eps < 1 (1/64 gives 9 to 13 iterations)
+ *   work_dev   device, GBS_MAX_CANDIDATES doubles, 8-byte aligned, overwritten
+ *   out_host   host, written on success
+ * BLOCKS: after every round the call waits for `cuda_stream` to read the K sums back.
+ */
+int gbs_search_clip_ratio(const gbs_plan_t* plan, const void* x, int x_dtype, int64_t n_rows,
+                          int64_t x_row_stride, float eps, double* work_dev, gbs_search_result_t* out_host,
+                          void* cuda_stream);
+
+/*
  * Host-only helper: write the m x m sign matrix H_m (row-major, +1 / -1) the plans use
  * (Algorithm 2).  `out_host` must hold m*m bytes.  Needs no device.
  */

@@ -250,3 +250,46 @@ def dequantize_rows(packed, delta, d: int, d_pad: int, m: int, bits: int, group:
                                         int(inverse), _dp(out), nthreads)
     _check(rc, "dequantize_rows")
     return out
+
+
+def gradual_binary_search(evaluate, eps: float, trace: list | None = None):
+    """Algorithm 1 (Gradual Binary Search), the loop for ONE projection, in the paper's order and notation:
+    a, b, m, f_m, the probe x on the left of m on even iterations and on the right on odd ones, the four
+    bracket updates, until b - a <= eps.  `evaluate(x)` is the objective (the paper uses perplexity).
+    Returns (m, f_m, iterations); `trace` (optional list) receives (iteration, x, f_x, a, b, m) per pass.
+    PARITY UNPINNED by the paper (it prints no trace): pinned by a hand-worked trace, by the bracket
+    invariants and by convergence on convex objectives."""
+    a, b = 0.0, 1.0
+    m = (a + b) / 2
+    f_m = evaluate(m)
+    iteration = 0
+    while b - a > eps:
+        if iteration % 2 == 0:
+            x = (a + m) / 2
+        else:
+            x = (b + m) / 2
+        f_x = evaluate(x)
+        if f_x < f_m:
+            if x < m:
+                b = m
+            else:
+                a = m
+            m, f_m = x, f_x
+        else:
+            if x < m:
+                a = x
+            else:
+                b = x
+        iteration += 1
+        if trace is not None:
+            trace.append((iteration, x, f_x, a, b, m))
+    return m, f_m, iteration
+
+
+def search_clip_ratio_rows(x, d: int, d_pad: int, m: int, bits: int, group: int, eps: float,
+                           trace: list | None = None):
+    """Algorithm 1's loop with the quantization error of the rows in x as the objective (clip ratios
+    are evaluated at their float32 value, the type the library's entry point takes)."""
+    def evaluate(alpha):
+        return float(clip_error_rows(x, d, d_pad, m, bits, group, np.array([np.float32(alpha)], dtype=np.float64))[0])
+    return gradual_binary_search(evaluate, eps, trace)

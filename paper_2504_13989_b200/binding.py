@@ -27,7 +27,8 @@ GBS_MAX_D_PAD = 32768
 GBS_MAX_CANDIDATES = 64
 
 EXPORTS = ("gbs_plan_create", "gbs_plan_destroy", "gbs_plan_info", "gbs_plan_device_status", "gbs_rotate_quantize",
-           "gbs_rotate_quantize_static", "gbs_dequantize", "gbs_clip_error", "gbs_hadamard_m", "gbs_status_string")
+           "gbs_rotate_quantize_static", "gbs_dequantize", "gbs_clip_error", "gbs_search_clip_ratio",
+           "gbs_hadamard_m", "gbs_status_string")
 GBS_STATIC_MAX_D_PAD = 4096
 
 
@@ -43,6 +44,11 @@ class PlanInfo(ctypes.Structure):
                 ("levels", ctypes.c_int), ("q_lo", ctypes.c_int), ("q_hi", ctypes.c_int),
                 ("code_bytes_per_row", ctypes.c_int64), ("scales_per_row", ctypes.c_int),
                 ("variant", ctypes.c_int)]
+
+
+class SearchResult(ctypes.Structure):
+    _fields_ = [("alpha", ctypes.c_float), ("a", ctypes.c_float), ("b", ctypes.c_float), ("err", ctypes.c_double),
+                ("iterations", ctypes.c_int), ("evaluations", ctypes.c_int), ("rounds", ctypes.c_int)]
 
 
 _lib = None
@@ -73,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.gbs_dequantize.restype = i32
         L.gbs_clip_error.argtypes = [vp, vp, i32, i64, i64, ctypes.POINTER(ctypes.c_float), i32, vp, vp, vp]
         L.gbs_clip_error.restype = i32
+        L.gbs_search_clip_ratio.argtypes = [vp, vp, i32, i64, i64, ctypes.c_float, vp, ctypes.POINTER(SearchResult), vp]
+        L.gbs_search_clip_ratio.restype = i32
         L.gbs_hadamard_m.argtypes = [i32, vp]
         L.gbs_hadamard_m.restype = i32
         L.gbs_status_string.argtypes = [i32]
@@ -203,6 +211,21 @@ def gbs_clip_error(plan: int, x: torch.Tensor, alphas, err_sum: torch.Tensor,
            "gbs_clip_error")
 
 
+def gbs_search_clip_ratio(plan: int, x: torch.Tensor, eps: float, work: torch.Tensor | None = None,
+                          stream=None) -> SearchResult:
+    """Algorithm 1's bracket search for the clip ratio of the rows in x (objective: quantization error).
+    Blocks on the stream after every round of up to 31 probes."""
+    info = gbs_plan_info(plan)
+    xv, n_rows, stride = _rows_view(x, info.d)
+    if work is None:
+        work = torch.empty(GBS_MAX_CANDIDATES, dtype=torch.float64, device=x.device)
+    res = SearchResult()
+    _check(lib().gbs_search_clip_ratio(ctypes.c_void_p(plan), xv.data_ptr(), _dtype_code(xv), n_rows, stride,
+                                       float(eps), work.data_ptr(), ctypes.byref(res), _stream_ptr(stream)),
+           "gbs_search_clip_ratio")
+    return res
+
+
 # ----------------------------------------------------------------------------------------------
 # convenience object: owns a plan handle and allocates outputs with torch
 # ----------------------------------------------------------------------------------------------
@@ -264,6 +287,9 @@ class Plan:
         rows = torch.empty((n_rows, K), dtype=torch.float32, device=x.device) if want_rows else None
         gbs_clip_error(self.handle, x, alphas, err_sum, rows, stream)
         return (err_sum, rows) if want_rows else err_sum
+
+    def search_clip_ratio(self, x: torch.Tensor, eps: float = 1.0 / 64, stream=None) -> SearchResult:
+        return gbs_search_clip_ratio(self.handle, x, eps, stream=stream)
 
     def rotate_quantize_host(self, x_host: torch.Tensor, codes_host: torch.Tensor, scales_host: torch.Tensor,
                              device="cuda:0", stream=None):
