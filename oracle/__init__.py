@@ -293,3 +293,59 @@ def search_clip_ratio_rows(x, d: int, d_pad: int, m: int, bits: int, group: int,
     def evaluate(alpha):
         return float(clip_error_rows(x, d, d_pad, m, bits, group, np.array([np.float32(alpha)], dtype=np.float64))[0])
     return gradual_binary_search(evaluate, eps, trace)
+
+
+# ----------------------------------------------------------------------------------------------
+# Asymmetric uniform quantizer (the KV-cache setting of Section 5.1: "asymmetric quantization with a
+# group size of 128"; the paper gives no formula, so this is the textbook definition with the clip
+# ratio of Section 3.1 shrinking both ends of the range).  PARITY UNPINNED by the paper; pinned by a
+# hand-worked example, the code range, the reproduction of both range ends at alpha = 1 and the
+# half-step error bound.
+# ----------------------------------------------------------------------------------------------
+def quantize_asym(y, bits: int, group: int = 0, alpha: float = 1.0):
+    """Per group of `group` consecutive values (0 = the whole row): lo = alpha*min(y), hi = alpha*max(y),
+    Delta = (hi - lo) / (2^bits - 1), q = clamp(rint((y - lo) / Delta), 0, 2^bits - 1) (round half to even),
+    yhat = q * Delta + lo.  A constant group (hi == lo) gives codes 0 and Delta 0.
+    Returns (q int32 [n], delta float64 [groups], zero float64 [groups])."""
+    y = np.ascontiguousarray(y, dtype=np.float64)
+    n = y.shape[0]
+    g = group if group else n
+    L = (1 << bits) - 1
+    q = np.zeros(n, dtype=np.int32)
+    delta = np.zeros(n // g, dtype=np.float64)
+    zero = np.zeros(n // g, dtype=np.float64)
+    for i in range(n // g):
+        seg = y[i * g:(i + 1) * g]
+        lo, hi = alpha * seg.min(), alpha * seg.max()
+        zero[i] = lo
+        if hi > lo:
+            delta[i] = (hi - lo) / L
+            q[i * g:(i + 1) * g] = np.clip(np.rint((seg - lo) / delta[i]), 0, L).astype(np.int32)
+    return q, delta, zero
+
+
+def rotate_quantize_asym_rows(x, d: int, d_pad: int, m: int, bits: int, group: int, alpha: float):
+    """Pad -> rotate (the symmetric path's rotation) -> asymmetric quantizer -> pack, row by row.
+    Returns dict(y, q (0 .. 2^bits-1), packed, delta [n,spr], zero [n,spr])."""
+    y = rotate_quantize_rows(x, d, d_pad, m, bits, 0, 1.0, want_q=False, want_packed=False)["y"]
+    n = y.shape[0]
+    spr = d_pad // group if group else 1
+    q = np.empty((n, d_pad), dtype=np.int32)
+    delta = np.empty((n, spr), dtype=np.float64)
+    zero = np.empty((n, spr), dtype=np.float64)
+    for r in range(n):
+        q[r], delta[r], zero[r] = quantize_asym(y[r], bits, group, alpha)
+    packed = np.stack([pack(q[r], bits) for r in range(n)]) if n else np.empty((0, d_pad * bits // 8), np.uint8)
+    return dict(y=y, q=q, packed=packed, delta=delta, zero=zero)
+
+
+def dequantize_asym_rows(packed, delta, zero, d_pad: int, bits: int, group: int) -> np.ndarray:
+    """yhat = q * Delta + zero in the rotated domain (fields are unsigned)."""
+    packed = np.ascontiguousarray(packed, dtype=np.uint8)
+    n = packed.shape[0]
+    g = group if group else d_pad
+    out = np.empty((n, d_pad), dtype=np.float64)
+    for r in range(n):
+        q = unpack(packed[r], d_pad, bits) & ((1 << bits) - 1)
+        out[r] = q * np.repeat(np.asarray(delta[r], dtype=np.float64), g) + np.repeat(np.asarray(zero[r], np.float64), g)
+    return out
