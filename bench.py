@@ -460,6 +460,17 @@ def extras(device, stream, args, peak):
             del sets, pl
         del xb
         torch.cuda.empty_cache()
+    # the asymmetric KV quantizer (group 128 = one row) on the same KV tensor
+    w = synth.WORKLOADS["kv128"]
+    xb = synth.make_device("kv128", device=str(device))
+    pl = Plan(w.d, w.d_pad, w.m, 3, 128, 1.0, asymmetric=True)
+    nbytes = w.n_rows * (w.d * 2 + w.d_pad * 3 // 8 + 8)
+    sets = build_sets([pl], xb, 2, device)
+    ms = timed_graph_loop([pl], sets, 40, 3, stream, False) / 40
+    out["kv128_b3_asymmetric_group128"] = {"us_per_launch": ms * 1e3, "gbs": nbytes / ms / 1e6,
+                                           "frac_of_measured": nbytes / ms / 1e6 / peak}
+    del sets, pl, xb
+    torch.cuda.empty_cache()
     # steady state of the d=4096 kernel: 65536 tokens per launch (the batch tiled 16 times)
     w = synth.WORKLOADS["llama4096"]
     xb = synth.make_host("llama4096").repeat(16, 1)

@@ -52,6 +52,9 @@ extern "C" {
 #define GBS_DTYPE_F32 0
 #define GBS_DTYPE_BF16 1
 
+/* gbs_plan_create_ex flags */
+#define GBS_PLAN_ASYMMETRIC 1    /* asymmetric quantizer (KV entries, Section 5.1): see gbs_plan_create_ex */
+
 /* gbs_dequantize flags */
 #define GBS_INVERSE_ROTATE 1
 
@@ -71,6 +74,8 @@ typedef struct gbs_plan_info {
     int q_lo, q_hi;                /* -D, +D                                          */
     int64_t code_bytes_per_row;    /* d' * bits / 8                                   */
     int scales_per_row;            /* group ? d'/group : 1                            */
+    int asymmetric;                /* 1 for a GBS_PLAN_ASYMMETRIC plan                */
+    int scale_floats_per_row;      /* scales_per_row, or 2 * scales_per_row when asymmetric */
     int variant;                   /* kernel family chosen for bf16 rows: 0 = generic shared-memory path,
                                       1 = tensor-core path for d' = 32 * U with U = m * 2^j <= 128, U % 16 == 0,
                                       d % 32 == 0 and group in {0, 32 .. 1024}, 2 = tensor-core path for
@@ -95,6 +100,21 @@ typedef struct gbs_plan_info {
  * and may be used from several threads / streams at once.  *out is written only on success.
  */
 int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bits, int group, float alpha);
+
+/*
+ * gbs_plan_create with flags.  flags = 0 is gbs_plan_create.
+ * GBS_PLAN_ASYMMETRIC selects the asymmetric uniform quantizer the paper uses for KV entries
+ * (Section 5.1 names it, with "a group size of 128", but prints no formula; this is the textbook one,
+ * with the clip ratio of Section 3.1 shrinking both ends of the range).  Per token or group:
+ *     lo = alpha * min y,  hi = alpha * max y,  Delta = (hi - lo) / (2^bits - 1),
+ *     code = clamp(rint((y - lo) / Delta), 0, 2^bits - 1)  (round half to even),  yhat = code * Delta + lo;
+ * a constant group gives codes 0 and Delta 0.  Codes are UNSIGNED `bits`-bit fields, packed as usual;
+ * `scales` holds the pair (Delta, lo) per group: layout [n_rows, scales_per_row, 2].
+ * Limits: d' = 128 rows (m = 1), group 0, 32, 64 or 128, bf16 input; other shapes return
+ * GBS_ERR_UNSUPPORTED.  gbs_clip_error and gbs_search_clip_ratio return GBS_ERR_UNSUPPORTED for such a
+ * plan; gbs_dequantize (both forms) honours it.
+ */
+int gbs_plan_create_ex(gbs_plan_t** out, int d, int d_pad, int m, int bits, int group, float alpha, int flags);
 
 /* Free a plan.  NULL is accepted.  Work already enqueued with the plan must have finished. */
 int gbs_plan_destroy(gbs_plan_t* plan);

@@ -26,7 +26,8 @@ GBS_INVERSE_ROTATE = 1
 GBS_MAX_D_PAD = 32768
 GBS_MAX_CANDIDATES = 64
 
-EXPORTS = ("gbs_plan_create", "gbs_plan_destroy", "gbs_plan_info", "gbs_plan_device_status", "gbs_rotate_quantize",
+GBS_PLAN_ASYMMETRIC = 1
+EXPORTS = ("gbs_plan_create", "gbs_plan_create_ex", "gbs_plan_destroy", "gbs_plan_info", "gbs_plan_device_status", "gbs_rotate_quantize",
            "gbs_rotate_quantize_static", "gbs_dequantize", "gbs_clip_error", "gbs_search_clip_ratio",
            "gbs_hadamard_m", "gbs_status_string")
 GBS_STATIC_MAX_D_PAD = 4096
@@ -43,6 +44,7 @@ class PlanInfo(ctypes.Structure):
                 ("bits", ctypes.c_int), ("group", ctypes.c_int), ("alpha", ctypes.c_float),
                 ("levels", ctypes.c_int), ("q_lo", ctypes.c_int), ("q_hi", ctypes.c_int),
                 ("code_bytes_per_row", ctypes.c_int64), ("scales_per_row", ctypes.c_int),
+                ("asymmetric", ctypes.c_int), ("scale_floats_per_row", ctypes.c_int),
                 ("variant", ctypes.c_int)]
 
 
@@ -65,6 +67,8 @@ def lib() -> ctypes.CDLL:
         vp, i32, i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
         L.gbs_plan_create.argtypes = [ctypes.POINTER(vp), i32, i32, i32, i32, i32, ctypes.c_float]
         L.gbs_plan_create.restype = i32
+        L.gbs_plan_create_ex.argtypes = [ctypes.POINTER(vp), i32, i32, i32, i32, i32, ctypes.c_float, i32]
+        L.gbs_plan_create_ex.restype = i32
         L.gbs_plan_destroy.argtypes = [vp]
         L.gbs_plan_destroy.restype = i32
         L.gbs_plan_info.argtypes = [vp, ctypes.POINTER(PlanInfo)]
@@ -138,6 +142,13 @@ def gbs_plan_create(d: int, d_pad: int, m: int, bits: int, group: int, alpha: fl
     """Returns an opaque plan handle (int).  See include/gbs.h for the argument ranges."""
     h = ctypes.c_void_p()
     _check(lib().gbs_plan_create(ctypes.byref(h), d, d_pad, m, bits, group, alpha), "gbs_plan_create")
+    return h.value
+
+
+def gbs_plan_create_ex(d: int, d_pad: int, m: int, bits: int, group: int, alpha: float, flags: int) -> int:
+    """gbs_plan_create with flags (GBS_PLAN_ASYMMETRIC: the asymmetric quantizer for d' = 128 KV rows)."""
+    h = ctypes.c_void_p()
+    _check(lib().gbs_plan_create_ex(ctypes.byref(h), d, d_pad, m, bits, group, alpha, flags), "gbs_plan_create_ex")
     return h.value
 
 
@@ -233,9 +244,9 @@ class Plan:
     """RAII wrapper of a gbs plan; allocates output tensors with torch and forwards to the C ABI."""
 
     def __init__(self, d: int, d_pad: int | None = None, m: int = 1, bits: int = 4, group: int = 0,
-                 alpha: float = 1.0):
+                 alpha: float = 1.0, asymmetric: bool = False):
         d_pad = d if d_pad is None else d_pad
-        self.handle = gbs_plan_create(d, d_pad, m, bits, group, alpha)
+        self.handle = gbs_plan_create_ex(d, d_pad, m, bits, group, alpha, GBS_PLAN_ASYMMETRIC if asymmetric else 0)
         self.info = gbs_plan_info(self.handle)
 
     def close(self):
@@ -260,7 +271,7 @@ class Plan:
 
     def alloc_outputs(self, n_rows: int, device, want_y: bool = False):
         codes = torch.empty((n_rows, self.info.code_bytes_per_row), dtype=torch.uint8, device=device)
-        scales = torch.empty((n_rows, self.info.scales_per_row), dtype=torch.float32, device=device)
+        scales = torch.empty((n_rows, self.info.scale_floats_per_row), dtype=torch.float32, device=device)
         y = torch.empty((n_rows, self.info.d_pad), dtype=torch.float32, device=device) if want_y else None
         return codes, scales, y
 

@@ -24,6 +24,7 @@ constexpr unsigned FULL = 0xffffffffu;
 struct GenericParams {
     int d, d_pad, k, m, n2;          // n2 = 2^k
     int group, G, spr;               // G = group ? group : d_pad ; spr = scales per row
+    int asym;                        // dequantize: asymmetric plan (unsigned codes, (Delta, lo) pairs)
     int levels;
     float norm, c_scale, c_inv;
     int tt_log2, rows_per_cta;       // team = 1 << tt_log2 threads per row
@@ -431,8 +432,10 @@ __global__ void __launch_bounds__(NT) k_clip_error(GenericParams P, ClipConsts C
 // ======================================================================================
 // dequantize
 // ======================================================================================
+// asym: unsigned fields, v = field * delta + zero (the asymmetric quantizer); else two's-complement fields.
 template <int BITS>
-__device__ __forceinline__ void unpack8(const unsigned char* src, float delta, float v[8])
+__device__ __forceinline__ void unpack8(const unsigned char* src, float delta, float v[8], bool asym = false,
+                                        float zero = 0.f)
 {
     unsigned word;
     if (BITS == 4) word = (unsigned)src[0] | ((unsigned)src[1] << 8) | ((unsigned)src[2] << 16) | ((unsigned)src[3] << 24);
@@ -440,8 +443,8 @@ __device__ __forceinline__ void unpack8(const unsigned char* src, float delta, f
 #pragma unroll
     for (int e = 0; e < 8; ++e) {
         int f = (int)((word >> (BITS * e)) & ((1u << BITS) - 1u));
-        f = (f << (32 - BITS)) >> (32 - BITS);    // sign-extend
-        v[e] = (float)f * delta;
+        if (!asym) f = (f << (32 - BITS)) >> (32 - BITS);    // sign-extend
+        v[e] = fmaf((float)f, delta, zero);
     }
 }
 
@@ -467,7 +470,7 @@ __device__ __forceinline__ void store1(__nv_bfloat16* dst, float v) { *dst = __f
 
 // yhat = q * Delta, rotated domain: pure streaming, one thread per chunk of 8 codes.
 template <typename OutT, int BITS>
-__global__ void __launch_bounds__(NT) k_dequantize_plain(int d_pad, int G, int spr, long long n_chunks,
+__global__ void __launch_bounds__(NT) k_dequantize_plain(int d_pad, int G, int spr, int asym, long long n_chunks,
                                                          const unsigned char* __restrict__ codes,
                                                          const float* __restrict__ scales,
                                                          OutT* __restrict__ out)
@@ -476,9 +479,11 @@ __global__ void __launch_bounds__(NT) k_dequantize_plain(int d_pad, int G, int s
     for (long long g = (long long)blockIdx.x * NT + threadIdx.x; g < n_chunks; g += (long long)gridDim.x * NT) {
         const long long row = g / chunks;
         const int ch = (int)(g - row * chunks);
-        const float delta = __ldg(scales + row * spr + (ch * 8) / G);
+        const long long si = (row * spr + (ch * 8) / G) * (asym ? 2 : 1);
+        const float delta = __ldg(scales + si);
+        const float zero = asym ? __ldg(scales + si + 1) : 0.f;
         float v[8];
-        unpack8<BITS>(codes + g * BITS, delta, v);
+        unpack8<BITS>(codes + g * BITS, delta, v, asym != 0, zero);
         store8(out + g * 8, v);
     }
 }
@@ -505,7 +510,8 @@ __global__ void __launch_bounds__(NT) k_dequantize_inverse(GenericParams P, cons
             const unsigned char* crow = codes + row * P.row_bytes;
             for (int ch = j; ch < P.chunks; ch += tt) {
                 float v[8];
-                unpack8<BITS>(crow + ch * BITS, __ldg(scales + row * P.spr + (ch * 8) / P.G), v);
+                const long long si = (row * P.spr + (ch * 8) / P.G) * (P.asym ? 2 : 1);
+                unpack8<BITS>(crow + ch * BITS, __ldg(scales + si), v, P.asym != 0, P.asym ? __ldg(scales + si + 1) : 0.f);
                 butterflies<8>(v);
                 const int p = ch * 8 + (ch >> 2);
 #pragma unroll
@@ -536,6 +542,7 @@ void fill_params(const gbs_plan* p, GenericParams& P, int64_t n_rows, int64_t st
     P.d = p->d; P.d_pad = p->d_pad; P.k = p->k; P.m = p->m; P.n2 = 1 << p->k;
     P.group = p->group; P.G = p->group ? p->group : p->d_pad;
     P.spr = p->group ? p->d_pad / p->group : 1;
+    P.asym = p->asym;
     P.levels = p->levels;
     P.norm = p->norm; P.c_scale = p->c_scale; P.c_inv = p->c_inv;
     P.chunks = p->d_pad / 8;
@@ -667,7 +674,7 @@ int gbs_generic_dequantize(const gbs_plan* p, const void* codes, const float* sc
         const int grid = (int)(blocks < cap ? blocks : cap);
 #define LAUNCH_DP(T, B)                                                                            \
     do {                                                                                           \
-        k_dequantize_plain<T, B><<<grid, NT, 0, stream>>>(P.d_pad, P.G, P.spr, n_chunks,            \
+        k_dequantize_plain<T, B><<<grid, NT, 0, stream>>>(P.d_pad, P.G, P.spr, P.asym, n_chunks,    \
                                                           (const unsigned char*)codes, scales, (T*)out); \
         e = cudaGetLastError();                                                                    \
     } while (0)

@@ -79,7 +79,14 @@ extern "C" const char* gbs_status_string(int status)
 
 extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bits, int group, float alpha)
 {
+    return gbs_plan_create_ex(out, d, d_pad, m, bits, group, alpha, 0);
+}
+
+extern "C" int gbs_plan_create_ex(gbs_plan_t** out, int d, int d_pad, int m, int bits, int group, float alpha,
+                                  int flags)
+{
     if (!out) return GBS_ERR_INVALID_ARG;
+    if (flags & ~GBS_PLAN_ASYMMETRIC) return GBS_ERR_INVALID_ARG;
     if (d < 1 || d_pad < d || m < 1) return GBS_ERR_INVALID_ARG;
     if (bits != 3 && bits != 4) return GBS_ERR_INVALID_ARG;
     if (!(alpha > 0.f) || !(alpha <= 1.f)) return GBS_ERR_INVALID_ARG;     // also rejects NaN
@@ -91,6 +98,9 @@ extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bi
     }
     if (!supported_m(m)) return GBS_ERR_UNSUPPORTED;
     if (d_pad > GBS_MAX_D_PAD) return GBS_ERR_UNSUPPORTED;
+    if ((flags & GBS_PLAN_ASYMMETRIC) &&
+        !(d_pad == 128 && m == 1 && (group == 0 || group == 32 || group == 64 || group == 128)))
+        return GBS_ERR_UNSUPPORTED;
 
     gbs_plan* p = new (std::nothrow) gbs_plan;
     if (!p) return GBS_ERR_ALLOC;
@@ -102,6 +112,7 @@ extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bi
     p->c_scale = (float)((double)alpha / ((double)p->levels * rootn));
     p->c_inv = (float)((double)p->levels / (double)alpha);
     p->variant = GBS_VARIANT_GENERIC;
+    p->asym = (flags & GBS_PLAN_ASYMMETRIC) ? 1 : 0;
     int rc = gbs_build_hadamard_m(m, p->h_hm);
     if (rc != GBS_OK) { delete p; return rc; }
 
@@ -136,6 +147,12 @@ extern "C" int gbs_plan_create(gbs_plan_t** out, int d, int d_pad, int m, int bi
         }
         p->variant = tc_uv ? GBS_VARIANT_TC_UV : (tc_row ? GBS_VARIANT_TC_ROW : GBS_VARIANT_TC_UVM);
         p->uvm_glog = uvm_glog;
+    }
+    if (p->asym && p->variant != GBS_VARIANT_TC_ROW) {          // only the row family has the asymmetric quantizer
+        if (p->d_aimg) cudaFree(p->d_aimg);
+        cudaFree(p->d_status);
+        delete p;
+        return GBS_ERR_UNSUPPORTED;
     }
     const char* nopdl = getenv("GBS_NO_PDL");
     p->pdl = (nopdl && nopdl[0] == '1') ? 0 : 1;
@@ -181,6 +198,8 @@ extern "C" int gbs_plan_info(const gbs_plan_t* p, gbs_plan_info_t* out)
     out->levels = p->levels; out->q_lo = -p->levels; out->q_hi = p->levels;
     out->code_bytes_per_row = (int64_t)p->d_pad * p->bits / 8;
     out->scales_per_row = p->group ? p->d_pad / p->group : 1;
+    out->asymmetric = p->asym;
+    out->scale_floats_per_row = out->scales_per_row * (p->asym ? 2 : 1);
     out->variant = p->variant;
     return GBS_OK;
 }
@@ -209,6 +228,7 @@ extern "C" int gbs_rotate_quantize(const gbs_plan_t* p, const void* x, int x_dty
     if (!codes || !scales) return GBS_ERR_INVALID_ARG;
     if (!aligned16(codes) || (y_opt && !aligned16(y_opt)) || (reinterpret_cast<uintptr_t>(scales) & 3u))
         return GBS_ERR_ALIGNMENT;
+    if (p->asym && !(p->variant == GBS_VARIANT_TC_ROW && x_dtype == GBS_DTYPE_BF16)) return GBS_ERR_UNSUPPORTED;
     DeviceGuard g;
     if (g.enter(p->device) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -250,6 +270,7 @@ extern "C" int gbs_clip_error(const gbs_plan_t* p, const void* x, int x_dtype, i
     int rc = check_rows(p, x, x_dtype, n_rows, x_row_stride);
     if (rc != GBS_OK) return rc;
     if (K < 1 || K > GBS_MAX_CANDIDATES || !alphas_host) return GBS_ERR_INVALID_ARG;
+    if (p->asym) return GBS_ERR_UNSUPPORTED;
     float c_scale[GBS_MAX_CANDIDATES], c_inv[GBS_MAX_CANDIDATES];
     const double rootn = sqrt((double)p->d_pad);
     for (int i = 0; i < K; ++i) {

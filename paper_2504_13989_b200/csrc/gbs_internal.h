@@ -29,6 +29,7 @@ struct gbs_plan {
     int variant;
     float* d_hm;           // device: H_m as floats, m*m row-major, followed by H_m^T (m*m)
     int pdl;               // tensor-core families launch with programmatic stream serialization
+    int asym;              // asymmetric quantizer (GBS_PLAN_ASYMMETRIC)
     int uvm_glog;          // UVM family: log2 of the number of 32-value chunks per tensor-core output row
     unsigned char* d_aimg; // device: pre-swizzled bf16 image of H_m (x) H_{2^j} for the tensor-core family (32 KB)
     int* d_status;         // device status word: 0, or the code of the first bounded wait that expired

@@ -204,6 +204,60 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, v
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
 }
 
+__device__ __forceinline__ float min3(float a, float b, float c)
+{
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// min and max of 32 registers.
+__device__ __forceinline__ void minmax32(const unsigned r[32], float& mn, float& mx)
+{
+    mn = __uint_as_float(r[0]);
+    mx = mn;
+#pragma unroll
+    for (int i = 0; i < 32; i += 2) {
+        mn = min3(__uint_as_float(r[i]), __uint_as_float(r[i + 1]), mn);
+        mx = max3(__uint_as_float(r[i]), __uint_as_float(r[i + 1]), mx);
+    }
+}
+
+// 32 consecutive UNSIGNED codes (asymmetric quantizer) -> packed little-endian bit stream.
+//   w = sat(Y * a1 + c0) maps the clipped range [lo, hi] onto [0, 1]; s = w * (2^BITS - 1) + 2^23 leaves
+//   rint(.) in the low mantissa bits (round-half-even by the FMA's own rounding).
+template <int BITS>
+__device__ __forceinline__ void quantize_pack32_u(const unsigned r[32], float a1, float c0, unsigned out[BITS])
+{
+    const float L = (float)((1 << BITS) - 1);
+    const float MAGIC = 8388608.f;                        // 2^23
+    unsigned acc[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+        unsigned a = 0;
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+            const float w = __saturatef(fmaf(__uint_as_float(r[8 * g + e]), a1, c0));
+            const unsigned s = __float_as_uint(fmaf(w, L, MAGIC));
+            unsigned t;
+            asm("shf.l.clamp.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(0u), "r"(s), "r"((unsigned)(BITS * e)));
+            a += t;
+        }
+        acc[g] = a;
+    }
+    if (BITS == 4) {
+        constexpr unsigned C = 0x4B000000u + 0xB0000000u;   // sum_e 0x4B000000 << 4e (mod 2^32)
+#pragma unroll
+        for (int g = 0; g < 4; ++g) out[g] = acc[g] - C;
+    } else {
+#pragma unroll
+        for (int g = 0; g < 4; ++g) acc[g] &= 0x00ffffffu;  // the exponent pattern only touches bits >= 24
+        out[0] = acc[0] | (acc[1] << 24);
+        out[1] = (acc[1] >> 8) | (acc[2] << 16);
+        out[2] = (acc[2] >> 16) | (acc[3] << 8);
+    }
+}
+
 // max|.| of 32 registers.
 __device__ __forceinline__ float absmax32(const unsigned r[32])
 {

@@ -49,6 +49,9 @@ struct RowParams {
     float c_scale;                // alpha / (D sqrt(d'))
     float c_half;                 // 1 / (2 alpha)
     float norm;                   // 1 / sqrt(d')
+    float alpha;                  // asymmetric plans: clip ratio
+    float a_delta;                // asymmetric plans: alpha / (sqrt(d') (2^bits - 1))
+    float a_zero;                 // asymmetric plans: alpha / sqrt(d')
     const unsigned char* h_img;   // pre-swizzled shared-memory image of H_128 (bf16), plan-owned
     unsigned char* codes;
     float* scales;
@@ -56,7 +59,8 @@ struct RowParams {
     int* status;
 };
 
-template <int BITS>
+// ASYM = true: the asymmetric quantizer (range [alpha*min, alpha*max], unsigned codes, scales = (Delta, lo)).
+template <int BITS, bool ASYM>
 __global__ void __launch_bounds__(THREADS, 1) k_tc_row_rq(const __grid_constant__ CUtensorMap tmap,
                                                           const __grid_constant__ RowParams P)
 {
@@ -150,18 +154,25 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_row_rq(const __grid_constant_
             const long long row = t * TILE + q * 32 + lane;
             unsigned r[32];
             // sweep 1: max|.| of each chunk of 32 rotated coordinates of this thread's row
-            float mc[4];
+            float mc[4];                              // max|.| (symmetric) or max (asymmetric) per chunk
+            float lc[4];                              // min per chunk (asymmetric only)
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 tmem_ld32_issue(taddr + c * 32, r);
                 tmem_ld_wait(r);
-                mc[c] = absmax32(r);
+                if (ASYM) minmax32(r, lc[c], mc[c]);
+                else mc[c] = absmax32(r);
             }
             if (cpg == 4) {
                 mc[0] = mc[1] = mc[2] = mc[3] = fmaxf(fmaxf(mc[0], mc[1]), fmaxf(mc[2], mc[3]));
+                if (ASYM) lc[0] = lc[1] = lc[2] = lc[3] = fminf(fminf(lc[0], lc[1]), fminf(lc[2], lc[3]));
             } else if (cpg == 2) {
                 mc[0] = mc[1] = fmaxf(mc[0], mc[1]);
                 mc[2] = mc[3] = fmaxf(mc[2], mc[3]);
+                if (ASYM) {
+                    lc[0] = lc[1] = fminf(lc[0], lc[1]);
+                    lc[2] = lc[3] = fminf(lc[2], lc[3]);
+                }
             }
             // sweep 2: Delta, round / clip, pack
             unsigned out[4 * BITS];
@@ -176,8 +187,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_row_rq(const __grid_constant_
                     __syncwarp();
                     if (lane == 0) mbar_arrive(&S->tempty[e]);
                 }
-                const float a1 = (mc[c] > 0.f) ? (P.c_half / mc[c]) : 0.f;
-                quantize_pack32<BITS>(r, a1, out + c * BITS);
+                if (ASYM) {
+                    const float range = P.alpha * (mc[c] - lc[c]);          // hi - lo of the clipped range
+                    const float a1 = (range > 0.f) ? (1.f / range) : 0.f;
+                    quantize_pack32_u<BITS>(r, a1, -(P.alpha * lc[c]) * a1, out + c * BITS);
+                } else {
+                    const float a1 = (mc[c] > 0.f) ? (P.c_half / mc[c]) : 0.f;
+                    quantize_pack32<BITS>(r, a1, out + c * BITS);
+                }
                 if (P.y_opt && live) {
                     float4* yo = reinterpret_cast<float4*>(P.y_opt + row * DP + c * 32);
 #pragma unroll
@@ -190,8 +207,17 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_row_rq(const __grid_constant_
                 uint4* dst = reinterpret_cast<uint4*>(P.codes + row * P.code_row_bytes);
 #pragma unroll
                 for (int i = 0; i < BITS; ++i) dst[i] = make_uint4(out[4 * i], out[4 * i + 1], out[4 * i + 2], out[4 * i + 3]);
-                float* sc = P.scales + row * P.spr;
-                if (cpg == 4) {
+                float* sc = P.scales + row * P.spr * (ASYM ? 2 : 1);
+                if (ASYM) {
+                    // (Delta, lo) per group
+#pragma unroll
+                    for (int c = 0; c < 4; c += 1) {
+                        if (c % cpg == 0) {
+                            sc[2 * (c / cpg)] = P.a_delta * (mc[c] - lc[c]);
+                            sc[2 * (c / cpg) + 1] = P.a_zero * lc[c];
+                        }
+                    }
+                } else if (cpg == 4) {
                     sc[0] = P.c_scale * mc[0];
                 } else if (cpg == 2) {
                     sc[0] = P.c_scale * mc[0];
@@ -264,6 +290,9 @@ int gbs_tc_row_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
     P.c_scale = p->c_scale;
     P.c_half = (float)(1.0 / (2.0 * (double)p->alpha));
     P.norm = p->norm;
+    P.alpha = p->alpha;
+    P.a_delta = (float)((double)p->alpha / (sqrt((double)DP) * (double)((1 << p->bits) - 1)));
+    P.a_zero = (float)((double)p->alpha / sqrt((double)DP));
     P.h_img = p->d_aimg;
     P.codes = (unsigned char*)codes;
     P.scales = scales;
@@ -275,12 +304,19 @@ int gbs_tc_row_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
     static bool attr_done[64] = {false};
     cudaError_t e = cudaSuccess;
     if (p->device < 0 || p->device >= 64 || !attr_done[p->device]) {
-        e = cudaFuncSetAttribute(k_tc_row_rq<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_row_rq<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        e = cudaFuncSetAttribute(k_tc_row_rq<3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_row_rq<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_row_rq<3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_row_rq<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
         if (e != cudaSuccess) return (int)e;
         if (p->device >= 0 && p->device < 64) attr_done[p->device] = true;
     }
-    if (p->bits == 3) e = launch(k_tc_row_rq<3>, grid, smem, stream, p->pdl != 0, tmap, P);
-    else e = launch(k_tc_row_rq<4>, grid, smem, stream, p->pdl != 0, tmap, P);
+    if (p->asym) {
+        if (p->bits == 3) e = launch(k_tc_row_rq<3, true>, grid, smem, stream, p->pdl != 0, tmap, P);
+        else e = launch(k_tc_row_rq<4, true>, grid, smem, stream, p->pdl != 0, tmap, P);
+    } else {
+        if (p->bits == 3) e = launch(k_tc_row_rq<3, false>, grid, smem, stream, p->pdl != 0, tmap, P);
+        else e = launch(k_tc_row_rq<4, false>, grid, smem, stream, p->pdl != 0, tmap, P);
+    }
     return (int)e;
 }
