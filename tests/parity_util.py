@@ -1,4 +1,4 @@
-"""Helpers for the GPU-vs-oracle parity tests.  The tolerances are the ones the task fixes:
+"""Helpers for the GPU-vs-oracle parity tests.  The tolerances:
 rotated fp32 values within 1e-5 relative L2 per row, scales within 1e-6 relative, integer codes
 identical except at rounding ties (mismatch fraction <= 1e-4, never more than one level),
 clip-error sums within 1e-5 relative."""
