@@ -58,6 +58,9 @@ void gbs_tc_uv_a_image(const gbs_plan* p, unsigned char* img32k);
 // image of H_m (x) H_{2^j} (U x U inside 128 x 128, bf16 +-1, K-major, 128-byte swizzle)
 void gbs_tc_sign_image(const int8_t* hm, int m, int j, int U, unsigned char* img32k);
 
+int gbs_tc_row_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, const float* alphas, int K,
+                          double* err_sum, float* err_rows, cudaStream_t stream);
+
 // gbs_tc_uvm.cu
 int gbs_tc_uvm_glog(const gbs_plan* p);        // 0 if the family does not apply
 int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,

@@ -258,6 +258,41 @@ __device__ __forceinline__ void quantize_pack32_u(const unsigned r[32], float a1
     }
 }
 
+// Fold 8 per-thread sums across the 32 lanes of a warp: after three halving exchanges lane l holds
+// candidate ((l>>4)&1)*4 + ((l>>3)&1)*2 + ((l>>2)&1) summed over 8 lanes; two more exchanges finish the
+// warp sum (returned in every lane for that lane's candidate).
+__device__ __forceinline__ float warp_fold8(const float acc[8], int lane)
+{
+    float h4[4], h2[2], h1;
+    {
+        const bool up = (lane & 16) != 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const float send = up ? acc[i] : acc[i + 4];
+            const float keep = up ? acc[i + 4] : acc[i];
+            h4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
+        }
+    }
+    {
+        const bool up = (lane & 8) != 0;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const float send = up ? h4[i] : h4[i + 2];
+            const float keep = up ? h4[i + 2] : h4[i];
+            h2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
+        }
+    }
+    {
+        const bool up = (lane & 4) != 0;
+        const float send = up ? h2[0] : h2[1];
+        const float keep = up ? h2[1] : h2[0];
+        h1 = keep + __shfl_xor_sync(0xffffffffu, send, 4);
+    }
+    h1 += __shfl_xor_sync(0xffffffffu, h1, 2);
+    h1 += __shfl_xor_sync(0xffffffffu, h1, 1);
+    return h1;
+}
+
 // max|.| of 32 registers.
 __device__ __forceinline__ float absmax32(const unsigned r[32])
 {

@@ -36,6 +36,7 @@ struct __align__(1024) Smem {
     unsigned char x[STAGES][TILE_BYTES];
     unsigned long long full[STAGES], empty[STAGES], tfull[STAGES], tempty[STAGES];
     unsigned long long hbar;               // the image of H_128 has landed
+    double csum[GBS_MAX_CANDIDATES];       // clip scoring: this CTA's error totals per candidate
     unsigned tmem_base;
     volatile int abort_flag;
 };
@@ -57,10 +58,19 @@ struct RowParams {
     float* scales;
     float* y_opt;
     int* status;
+    // clip-ratio scoring (the CLIP instantiation only)
+    int K;                        // candidates
+    int levels;                   // D
+    float norm2;                  // 1 / d'
+    float clip_half[GBS_MAX_CANDIDATES];    // 1 / (2 alpha_k), zero beyond K
+    float clip_scale[GBS_MAX_CANDIDATES];   // alpha_k / D,     zero beyond K
+    double* err_sum;
+    float* err_rows;
 };
 
 // ASYM = true: the asymmetric quantizer (range [alpha*min, alpha*max], unsigned codes, scales = (Delta, lo)).
-template <int BITS, bool ASYM>
+// CLIP = true: instead of quantizing, score K clip ratios (symmetric quantizer) from the thread's own row.
+template <int BITS, bool ASYM, bool CLIP>
 __global__ void __launch_bounds__(THREADS, 1) k_tc_row_rq(const __grid_constant__ CUtensorMap tmap,
                                                           const __grid_constant__ RowParams P)
 {
@@ -92,6 +102,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_row_rq(const __grid_constant_
             mbar_init(&S->tempty[s], 4);
         }
         S->abort_flag = 0;
+        for (int k = 0; k < GBS_MAX_CANDIDATES; ++k) S->csum[k] = 0.0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(&S->tmem_base, TMEM_COLS);
@@ -174,9 +185,61 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_row_rq(const __grid_constant_
                     lc[2] = lc[3] = fminf(lc[2], lc[3]);
                 }
             }
+            const bool live = row < P.n_rows;
+            if constexpr (CLIP) {
+                // Squared quantization error of this thread's row under every candidate clip ratio (Sections
+                // 2.1, 3.1), eight candidates per sweep over the four chunks: per value and candidate clamp
+                // (fma.sat), round half-even (magic add), residual, square-accumulate.  The row's sums are
+                // thread-local; the totals are folded across the warp and added to the CTA's fp64 sums.
+                const float twoD = (float)(2 * P.levels);
+                const float MAGIC = 8388608.f;
+                const float mD = MAGIC + (float)P.levels;
+                float rM[4];
+#pragma unroll
+                for (int c = 0; c < 4; ++c) rM[c] = (mc[c] > 0.f) ? (1.f / mc[c]) : 0.f;
+                for (int k0 = 0; k0 < P.K; k0 += 8) {
+                    float acc[8];
+#pragma unroll
+                    for (int kk = 0; kk < 8; ++kk) acc[kk] = 0.f;
+#pragma unroll 1
+                    for (int c = 0; c < 4; ++c) {
+                        tmem_ld32_issue(taddr + c * 32, r);
+                        tmem_ld_wait(r);
+                        float a1[8], dl[8];
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) {
+                            a1[kk] = P.clip_half[k0 + kk] * rM[c];
+                            dl[kk] = -P.clip_scale[k0 + kk] * mc[c];
+                        }
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) {
+                            const float y = __uint_as_float(r[i]);
+#pragma unroll
+                            for (int kk = 0; kk < 8; ++kk) {
+                                const float w = __saturatef(fmaf(y, a1[kk], 0.5f));
+                                const float qv = fmaf(w, twoD, MAGIC) - mD;
+                                const float err = fmaf(qv, dl[kk], y);
+                                acc[kk] = fmaf(err, err, acc[kk]);
+                            }
+                        }
+                    }
+                    if (P.err_rows && live) {
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk)
+                            if (k0 + kk < P.K) P.err_rows[row * P.K + k0 + kk] = acc[kk] * P.norm2;
+                    }
+                    const float h1 = warp_fold8(acc, lane);
+                    const int kk = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
+                    if ((lane & 3) == 0 && k0 + kk < P.K) atomicAdd(&S->csum[k0 + kk], (double)h1);
+                }
+                // the accumulators have been read for the last time: hand the TMEM stage back
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&S->tempty[e]);
+                continue;
+            }
             // sweep 2: Delta, round / clip, pack
             unsigned out[4 * BITS];
-            const bool live = row < P.n_rows;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 tmem_ld32_issue(taddr + c * 32, r);
@@ -237,6 +300,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_row_rq(const __grid_constant_
         tc_fence_after();
         tmem_dealloc(tmem_base, TMEM_COLS);
     }
+    if (CLIP && (int)threadIdx.x < P.K) atomicAdd(&P.err_sum[threadIdx.x], S->csum[threadIdx.x] * (double)P.norm2);
 }
 
 template <typename KernelT>
@@ -265,58 +329,99 @@ bool gbs_tc_row_supported(const gbs_plan* p)
     return get_encode() != nullptr && p->smem_optin >= (int)(sizeof(Smem) + 1024);
 }
 
-int gbs_tc_row_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
-                               float* scales, float* y_opt, cudaStream_t stream)
+namespace {
+
+int row_prepare(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, CUtensorMap* tmap, RowParams* P)
 {
     EncodeTiledFn encode = get_encode();
     if (!encode) return (int)cudaErrorNotSupported;
     if (n_rows > (int64_t)0x7fffffff - TILE) return (int)cudaErrorInvalidValue;      // TMA coordinates are 32-bit
-    CUtensorMap tmap;
     const cuuint64_t gdim[2] = {(cuuint64_t)p->d, (cuuint64_t)n_rows};
     const cuuint64_t gstr[1] = {(cuuint64_t)(stride * 2)};
     const cuuint32_t box[2] = {64, TILE};
     const cuuint32_t estr[2] = {1, 1};
-    CUresult r = encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), gdim, gstr, box, estr,
+    CUresult r = encode(tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(x), gdim, gstr, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return (int)cudaErrorInvalidValue;
+    memset(P, 0, sizeof(*P));
+    P->n_rows = n_rows;
+    P->n_tiles = (int)((n_rows + TILE - 1) / TILE);
+    P->code_row_bytes = DP * p->bits / 8;
+    P->chunks_per_group = (p->group ? p->group : DP) / 32;
+    P->spr = p->group ? DP / p->group : 1;
+    P->c_scale = p->c_scale;
+    P->c_half = (float)(1.0 / (2.0 * (double)p->alpha));
+    P->norm = p->norm;
+    P->alpha = p->alpha;
+    P->a_delta = (float)((double)p->alpha / (sqrt((double)DP) * (double)((1 << p->bits) - 1)));
+    P->a_zero = (float)((double)p->alpha / sqrt((double)DP));
+    P->h_img = p->d_aimg;
+    P->status = p->d_status;
+    P->levels = p->levels;
+    P->norm2 = (float)(1.0 / (double)DP);
+    return 0;
+}
 
+// opt in to the large dynamic shared memory once per device (not a stream operation)
+cudaError_t row_opt_in(const gbs_plan* p, int smem)
+{
+    static bool attr_done[64] = {false};
+    if (p->device >= 0 && p->device < 64 && attr_done[p->device]) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(k_tc_row_rq<3, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_row_rq<4, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_row_rq<3, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_row_rq<4, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_row_rq<4, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    if (e == cudaSuccess && p->device >= 0 && p->device < 64) attr_done[p->device] = true;
+    return e;
+}
+
+}  // namespace
+
+int gbs_tc_row_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
+                               float* scales, float* y_opt, cudaStream_t stream)
+{
+    CUtensorMap tmap;
     RowParams P;
-    P.n_rows = n_rows;
-    P.n_tiles = (int)((n_rows + TILE - 1) / TILE);
-    P.code_row_bytes = DP * p->bits / 8;
-    P.chunks_per_group = (p->group ? p->group : DP) / 32;
-    P.spr = p->group ? DP / p->group : 1;
-    P.c_scale = p->c_scale;
-    P.c_half = (float)(1.0 / (2.0 * (double)p->alpha));
-    P.norm = p->norm;
-    P.alpha = p->alpha;
-    P.a_delta = (float)((double)p->alpha / (sqrt((double)DP) * (double)((1 << p->bits) - 1)));
-    P.a_zero = (float)((double)p->alpha / sqrt((double)DP));
-    P.h_img = p->d_aimg;
+    const int rc = row_prepare(p, x, n_rows, stride, &tmap, &P);
+    if (rc != 0) return rc;
     P.codes = (unsigned char*)codes;
     P.scales = scales;
     P.y_opt = y_opt;
-    P.status = p->d_status;
     const int smem = (int)sizeof(Smem) + 1024;
     const int grid = P.n_tiles < p->sm_count ? P.n_tiles : p->sm_count;
-    // opt in to the large dynamic shared memory once per device (not a stream operation)
-    static bool attr_done[64] = {false};
-    cudaError_t e = cudaSuccess;
-    if (p->device < 0 || p->device >= 64 || !attr_done[p->device]) {
-        e = cudaFuncSetAttribute(k_tc_row_rq<3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_row_rq<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_row_rq<3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_row_rq<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return (int)e;
-        if (p->device >= 0 && p->device < 64) attr_done[p->device] = true;
-    }
+    cudaError_t e = row_opt_in(p, smem);
+    if (e != cudaSuccess) return (int)e;
     if (p->asym) {
-        if (p->bits == 3) e = launch(k_tc_row_rq<3, true>, grid, smem, stream, p->pdl != 0, tmap, P);
-        else e = launch(k_tc_row_rq<4, true>, grid, smem, stream, p->pdl != 0, tmap, P);
+        if (p->bits == 3) e = launch(k_tc_row_rq<3, true, false>, grid, smem, stream, p->pdl != 0, tmap, P);
+        else e = launch(k_tc_row_rq<4, true, false>, grid, smem, stream, p->pdl != 0, tmap, P);
     } else {
-        if (p->bits == 3) e = launch(k_tc_row_rq<3, false>, grid, smem, stream, p->pdl != 0, tmap, P);
-        else e = launch(k_tc_row_rq<4, false>, grid, smem, stream, p->pdl != 0, tmap, P);
+        if (p->bits == 3) e = launch(k_tc_row_rq<3, false, false>, grid, smem, stream, p->pdl != 0, tmap, P);
+        else e = launch(k_tc_row_rq<4, false, false>, grid, smem, stream, p->pdl != 0, tmap, P);
     }
+    return (int)e;
+}
+
+// Clip-ratio scoring for d' = 128 rows: the same contraction, the row stays in the thread's TMEM lane.
+int gbs_tc_row_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, const float* alphas, int K,
+                          double* err_sum, float* err_rows, cudaStream_t stream)
+{
+    CUtensorMap tmap;
+    RowParams P;
+    const int rc = row_prepare(p, x, n_rows, stride, &tmap, &P);
+    if (rc != 0) return rc;
+    P.K = K;
+    for (int i = 0; i < K; ++i) {
+        P.clip_half[i] = (float)(1.0 / (2.0 * (double)alphas[i]));
+        P.clip_scale[i] = (float)((double)alphas[i] / (double)p->levels);
+    }
+    P.err_sum = err_sum;
+    P.err_rows = err_rows;
+    const int smem = (int)sizeof(Smem) + 1024;
+    const int grid = P.n_tiles < p->sm_count ? P.n_tiles : p->sm_count;
+    cudaError_t e = row_opt_in(p, smem);
+    if (e != cudaSuccess) return (int)e;
+    e = launch(k_tc_row_rq<4, false, true>, grid, smem, stream, p->pdl != 0, tmap, P);
     return (int)e;
 }

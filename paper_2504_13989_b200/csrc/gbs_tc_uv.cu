@@ -117,35 +117,7 @@ __device__ __forceinline__ void clip_score32(const unsigned r[32], float M, cons
                 acc[kk] = fmaf(err, err, acc[kk]);
             }
         }
-        // fold 8 sums x 32 lanes: after three halving exchanges lane l holds candidate ((l>>4)&1)*4 +
-        // ((l>>3)&1)*2 + ((l>>2)&1) summed over 8 lanes; two more exchanges finish the warp sum
-        float h4[4], h2[2], h1;
-        {
-            const bool up = (lane & 16) != 0;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float send = up ? acc[i] : acc[i + 4];
-                const float keep = up ? acc[i + 4] : acc[i];
-                h4[i] = keep + __shfl_xor_sync(0xffffffffu, send, 16);
-            }
-        }
-        {
-            const bool up = (lane & 8) != 0;
-#pragma unroll
-            for (int i = 0; i < 2; ++i) {
-                const float send = up ? h4[i] : h4[i + 2];
-                const float keep = up ? h4[i + 2] : h4[i];
-                h2[i] = keep + __shfl_xor_sync(0xffffffffu, send, 8);
-            }
-        }
-        {
-            const bool up = (lane & 4) != 0;
-            const float send = up ? h2[0] : h2[1];
-            const float keep = up ? h2[1] : h2[0];
-            h1 = keep + __shfl_xor_sync(0xffffffffu, send, 4);
-        }
-        h1 += __shfl_xor_sync(0xffffffffu, h1, 2);
-        h1 += __shfl_xor_sync(0xffffffffu, h1, 1);
+        const float h1 = warp_fold8(acc, lane);
         const int kk = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
         if ((lane & 3) == 0 && k0 + kk < P.K) part_q[k0 + kk] = h1;
     }

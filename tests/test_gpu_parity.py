@@ -307,6 +307,16 @@ def test_row_family_shapes(d, bits, group, alpha, rows, stride):
             assert int(codes[2].max()) == 0 and float(scales[2].abs().max()) == 0.0
         codes2, scales2, _ = _run_rq(plan, xd, rows, want_y=False)
         assert torch.equal(codes, codes2) and torch.equal(scales, scales2)
+        # clip-ratio scoring from the thread-owned row
+        K = (3, 8, 11, 33, 64)[(d + bits + group + rows) % 5]
+        alphas = np.linspace(0.3, 1.0, K)
+        err, erows = plan.clip_error(xd, alphas, want_rows=True)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+        eref, rref = oracle.clip_error_rows(synth.to_oracle_array(x.contiguous()), d, 128, 1, bits, group, alphas,
+                                            want_rows=True)
+        np.testing.assert_allclose(err.cpu().numpy(), eref, rtol=TOL_CLIP)
+        np.testing.assert_allclose(erows.cpu().double().numpy(), rref, rtol=1e-4, atol=1e-12)
 
 
 def test_back_to_back_launches_on_one_stream():
