@@ -38,7 +38,7 @@ HEADLINE = "llama4096"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused kernel on the headline
 # workload, from the ncu capture summarised under profiles/ (None until a capture exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 33_610_240   # reads 33.61 MB; the codes are still in L2 when the kernel ends
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 33_608_960   # reads 33.61 MB; the codes are still in L2 when the kernel ends
 
 
 def algorithmic_bytes(n_rows: int, d: int, d_pad: int, bits: int, group: int, in_bytes: int) -> int:
@@ -211,17 +211,20 @@ def build_sets(plan_list, x_base, nsets, device):
     return sets
 
 
-def run_step(plan_list, st):
-    x, outs = st
-    for pl, o in zip(plan_list, outs):
-        pl.rotate_quantize(x, out=o)
+def run_step(plan_list, sets, i):
+    """One step: every plan's launch over one batch.  Launch j of step i reads the batch copy of buffer set
+    i + j * nsets / len(plans), so that no launch finds its input in L2 from the launch before it."""
+    nsets = len(sets)
+    for j, pl in enumerate(plan_list):
+        x = sets[(i + j * (nsets // len(plan_list))) % nsets][0]
+        pl.rotate_quantize(x, out=sets[i % nsets][1][j])
 
 
 def capture(plan_list, sets, idx_list, stream):
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g, stream=stream):
         for i in idx_list:
-            run_step(plan_list, sets[i])
+            run_step(plan_list, sets, i)
     return g
 
 
@@ -230,7 +233,7 @@ def timed_graph_loop(plan_list, sets, steps, warmup, stream, dist_ok, sampler=No
     nsets = len(sets)
     with torch.cuda.stream(stream):
         for i in range(max(warmup, 3)):
-            run_step(plan_list, sets[i % nsets])
+            run_step(plan_list, sets, i % nsets)
     stream.synchronize()
     g_all = capture(plan_list, sets, list(range(nsets)), stream)
     rem = steps % nsets
@@ -388,7 +391,8 @@ def main():
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": "%s: %d tokens x d=%d bf16, H_%d, b=3 and b=4 (one launch each per step), "
                                    "per-token scales, alpha=%.2f" % (HEADLINE, w.n_rows, w.d, w.d_pad, w.alpha),
-                       "replicas": world, "l2": "inputs rotate over %d buffer sets (%.0f MB > 4x L2)" %
+                       "replicas": world, "l2": "inputs rotate over %d buffer sets (%.0f MB > 4x L2); the b=3 and b=4 launches of a step read "
+                       "different copies" %
                        (args.nsets, args.nsets * (step_bytes + w.n_rows * w.d * 2) / 1e6),
                        "launch": "CUDA graph replay", "levels": "D=2^(b-1)-1"},
             "mtokens_per_s": total_tokens / (total_ms * 1e-3) / 1e6,
