@@ -138,7 +138,8 @@ int gbs_plan_device_status(const gbs_plan_t* plan, int* out);
  *                r * x_row_stride.  Must be 16-byte aligned with x_row_stride * sizeof(elem)
  *                a multiple of 16, x_row_stride >= d.
  *   codes        device, n_rows * d' * bits / 8 bytes, 16-byte aligned
- *   scales       device, n_rows * scales_per_row floats
+ *   scales       device, n_rows * scale_floats_per_row floats (scales_per_row Deltas per row; (Delta, lo)
+ *                pairs for an asymmetric plan)
  *   y_opt        NULL, or device n_rows * d' floats receiving the rotated normalised values
  *                (16-byte aligned)
  * n_rows = 0 is a successful no-op.
