@@ -471,3 +471,19 @@ def test_quantizer_invariants_on_device():
         spike[0, 0] = 200.0; spike[1, 1777] = 200.0; spike[2, d - 1] = -200.0
         _, _, ys = _run_rq(plan, spike.to(DEV), 3)
         np.testing.assert_allclose(ys.abs().cpu().numpy(), 200.0 / 64.0, rtol=1e-6)
+
+
+@pytest.mark.parametrize("d,d_pad,m", [(3584, 3584, 28), (18944, 20480, 20), (4000, 4096, 1), (96, 128, 1)])
+def test_expansion_identity_of_eq_2_through_the_library(d, d_pad, m):
+    """Eq. (2): with activations and weight rows both zero-padded to d' and rotated by the same
+    normalised Hadamard, (X_pad H^T)(H W_pad^T) = X W^T.  Rotating the rows of W^T is the weight-side
+    half of the expansion; both halves go through gbs_rotate_quantize's rotated output here."""
+    rng = np.random.Generator(np.random.PCG64(d + m))
+    x = torch.from_numpy(rng.standard_normal((24, d)).astype(np.float32)).to(torch.bfloat16)
+    wt = torch.from_numpy((rng.standard_normal((40, d)) / np.sqrt(d)).astype(np.float32)).to(torch.bfloat16)
+    with Plan(d, d_pad, m, 4, 0, 1.0) as plan:
+        _, _, yx = _run_rq(plan, x.to(DEV), 24)
+        _, _, yw = _run_rq(plan, wt.to(DEV), 40)
+    got = (yx.double() @ yw.double().T).cpu().numpy()
+    want = x.double().numpy() @ wt.double().numpy().T
+    np.testing.assert_allclose(got, want, rtol=0, atol=2e-5 * np.abs(want).max() + 1e-6)
