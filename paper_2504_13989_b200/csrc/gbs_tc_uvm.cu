@@ -9,7 +9,10 @@
 //   * H_32 inside each chunk and H_G across the chunks are butterflies in registers, in two sweeps over
 //     TMEM (a thread cannot hold its 256 values at once): sweep 1 transforms each chunk in place,
 //     sweep 2 loads 4 columns of every chunk, runs the G-point butterflies, takes max|.| and writes back.
-//   * sweep 3 scales, rounds, clips (Sections 2.1, 3.1) and packs each chunk; per-token scales only.
+//   * sweep 3 scales, rounds, clips (Sections 2.1, 3.1) and packs each chunk.  Scales are per token, or
+//     per group of 32 * 2^e consecutive coordinates (GROUPED): a group is 2^e chunks of one lane, or,
+//     beyond the G chunks of a lane, up to 32 whole lanes of a warp; the two warps that share a lane
+//     quadrant exchange their per-chunk maxima through shared memory at the second barrier.
 // The sixteen epilogue warps form two groups of eight that take alternate tokens (so that one group's
 // barrier waits are filled by the other's arithmetic): in a group, warp (q, w) serves lane quadrant q,
 // chunks w, w+2, .. in sweeps 1 and 3 and column groups 4w .. 4w+3 in sweep 2; two 256-thread named
@@ -39,6 +42,9 @@ struct __align__(1024) Smem {
     unsigned long long abar;
     __align__(16) float red[2][2][8];          // [group][iteration parity][warp of the group]: max of the token
     int gabort[2][2];                          // [group][iteration parity]: a warp of the group gave up waiting
+    // GROUPED: [group][warp half w][lane u'][chunk]: max|.| of the chunk's scale group over the columns warp w
+    // swept.  Written between a token's two barriers and read after the second, so one copy is enough.
+    __align__(16) float gm[2][2][UMAX][8];
     unsigned tmem_base;
     volatile int abort_flag;
 };
@@ -51,6 +57,8 @@ struct UvmParams {
     int stage_bytes;              // U * G * 64
     int code_row_bytes;
     int d_pad;
+    int gsh;                      // GROUPED: scale group = 2^gsh chunks of 32 coordinates
+    int spr;                      // scales per row
     float c_scale, c_half, norm;
     const unsigned char* a_img;
     unsigned char* codes;
@@ -141,7 +149,7 @@ __device__ __forceinline__ void tmem_ld_wait_n<32>(unsigned* r)
 // ---------------------------------------------------------------------------------------------
 // kernel
 // ---------------------------------------------------------------------------------------------
-template <int BITS, int GLOG>
+template <int BITS, int GLOG, bool GROUPED>
 __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant__ CUtensorMap tmap,
                                                           const __grid_constant__ UvmParams P)
 {
@@ -259,6 +267,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
             if (S->gabort[grp][gp]) break;
             // sweep 2: H_G across the chunks, four columns at a time; max|.| of the finished transform
             float M = 0.f;
+            float Mc[G];                                  // GROUPED: max|.| per chunk, then per scale group
+#pragma unroll
+            for (int c = 0; c < G; ++c) Mc[c] = 0.f;
             if (quad_live) {
                 tc_fence_after();
 #pragma unroll
@@ -286,31 +297,76 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
 #pragma unroll
                     for (int i = 0; i < G * 2; ++i) {
                         unpk(p[i], x[2 * i], x[2 * i + 1]);
-                        M = max3(fabsf(__uint_as_float(x[2 * i])), fabsf(__uint_as_float(x[2 * i + 1])), M);
+                        if (GROUPED)
+                            Mc[i >> 1] = max3(fabsf(__uint_as_float(x[2 * i])), fabsf(__uint_as_float(x[2 * i + 1])), Mc[i >> 1]);
+                        else
+                            M = max3(fabsf(__uint_as_float(x[2 * i])), fabsf(__uint_as_float(x[2 * i + 1])), M);
                     }
 #pragma unroll
                     for (int c = 0; c < G; ++c) tmem_st4(col0 + c * V, x + 4 * c);
                 }
                 tmem_wait_st();
                 tc_fence_before();
+                if (GROUPED) {
+                    // chunk maxima -> group maxima: over the 2^gsh chunks of a group inside the lane, then, for
+                    // a group of several whole lanes, over those lanes (every chunk of the lane is in it)
+#pragma unroll
+                    for (int h = 1; h < G; h <<= 1)
+                        if (h < (1 << P.gsh)) {
+#pragma unroll
+                            for (int c = 0; c < G; ++c)
+                                if ((c & h) == 0) Mc[c] = Mc[c + h] = fmaxf(Mc[c], Mc[c + h]);
+                        }
+                    if (P.gsh > GLOG) {
+                        float m = Mc[0];
+                        for (int o = 1; o < (1 << (P.gsh - GLOG)); o <<= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+#pragma unroll
+                        for (int c = 0; c < G; ++c) Mc[c] = m;
+                    }
+                    float* gw = &S->gm[grp][w][up][0];
+                    if (G == 2) {
+                        *reinterpret_cast<float2*>(gw) = make_float2(Mc[0], Mc[1]);
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < G; c += 4)
+                            *reinterpret_cast<float4*>(gw + c) = make_float4(Mc[c], Mc[c + 1], Mc[(c + 2) % G], Mc[(c + 3) % G]);
+                    }
+                }
             }
-            const unsigned mw = __reduce_max_sync(0xffffffffu, __float_as_uint(M));
-            if (lane == 0) S->red[grp][gp][ew] = __uint_as_float(mw);
+            if (!GROUPED) {
+                const unsigned mw = __reduce_max_sync(0xffffffffu, __float_as_uint(M));
+                if (lane == 0) S->red[grp][gp][ew] = __uint_as_float(mw);
+            }
             asm volatile("bar.sync %0, 256;" ::"r"(1 + grp) : "memory");
-            {
+            float Ms[G / 2];                              // GROUPED: group maximum for chunk 2 i + w
+            if (GROUPED) {
+                // the other warp of this lane quadrant swept the other sixteen columns of every chunk
+                const float* go = &S->gm[grp][w ^ 1][up][0];
+#pragma unroll
+                for (int i = 0; i < G / 2; ++i) Ms[i] = fmaxf(w ? Mc[2 * i + 1] : Mc[2 * i], go[2 * i + w]);
+            } else {
                 const float4* rp = reinterpret_cast<const float4*>(&S->red[grp][gp][0]);
                 const float4 m0 = rp[0], m1 = rp[1];
                 M = fmaxf(fmaxf(fmaxf(m0.x, m0.y), fmaxf(m0.z, m0.w)), fmaxf(fmaxf(m1.x, m1.y), fmaxf(m1.z, m1.w)));
             }
             // sweep 3: Delta, round / clip, pack, store
-            const float a1 = (M > 0.f) ? __fdividef(P.c_half, M) : 0.f;
+            float a1 = (M > 0.f) ? __fdividef(P.c_half, M) : 0.f;
             if (quad_live) {
                 tc_fence_after();
 #pragma unroll
-                for (int c = w; c < G; c += 2) {
+                for (int i = 0; i < G / 2; ++i) {
+                    const int c = 2 * i + w;
                     tmem_ld32_issue(tcol + c * V, r);
                     tmem_ld_wait(r);
                     if (lane_live) {
+                        if (GROUPED) {
+                            const float mg = Ms[i];
+                            a1 = (mg > 0.f) ? __fdividef(P.c_half, mg) : 0.f;
+                            // one writer per group: its first chunk, in its first lane
+                            const bool writer = (P.gsh <= GLOG) ? ((c & ((1 << P.gsh) - 1)) == 0)
+                                                                : (c == 0 && (lane & ((1 << (P.gsh - GLOG)) - 1)) == 0);
+                            if (writer) P.scales[row * P.spr + ((up * G + c) >> P.gsh)] = P.c_scale * mg;
+                        }
                         unsigned out[BITS];
                         quantize_pack32<BITS>(r, a1, out);
                         unsigned* dst = reinterpret_cast<unsigned*>(P.codes + row * P.code_row_bytes +
@@ -331,7 +387,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
                 }
                 tc_fence_before();
             }
-            if (ew == 0 && lane == 0) P.scales[row] = P.c_scale * M;
+            if (!GROUPED && ew == 0 && lane == 0) P.scales[row] = P.c_scale * M;
             // the accumulators have been read for the last time: hand the TMEM stage back to the MMA issuer
             __syncwarp();
             if (lane == 0) mbar_arrive(&S->tempty[ts]);
@@ -371,10 +427,17 @@ cudaError_t launch(KernelT kernel, int grid, int smem, cudaStream_t stream, bool
 // Smallest G in {2, 4, 8} for which U = d' / (32 G) fits the tensor-core factor; 0 if the family does not apply.
 int gbs_tc_uvm_glog(const gbs_plan* p)
 {
-    if (p->group != 0 || p->d_pad <= 4096) return 0;
+    if (p->d_pad <= 4096) return 0;
+    int gsh = 0;                                   // group = 32 * 2^gsh coordinates
+    if (p->group != 0) {
+        if (p->group % V != 0) return 0;
+        while ((V << gsh) < p->group) ++gsh;
+        if ((V << gsh) != p->group) return 0;
+    }
     for (int g = 1; g <= 3; ++g) {
         const int span = V << g;
         if (p->d_pad % span != 0 || p->d % span != 0) continue;
+        if (p->group != 0 && gsh > g + 5) continue;          // a group may span at most the 32 lanes of a warp
         const int U = p->d_pad / span;
         if (U > UMAX || U % 16 != 0 || p->k - 5 - g < 0) continue;
         if (get_encode() == nullptr || p->smem_optin < (int)(sizeof(Smem) + 1024)) return 0;
@@ -411,6 +474,10 @@ int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
     P.n_stages = B_BYTES / P.stage_bytes < MAX_STAGES ? B_BYTES / P.stage_bytes : MAX_STAGES;
     P.code_row_bytes = p->d_pad * p->bits / 8;
     P.d_pad = p->d_pad;
+    if (p->group != 0) {
+        while ((V << P.gsh) < p->group) ++P.gsh;
+    }
+    P.spr = p->group ? p->d_pad / p->group : 1;
     P.c_scale = p->c_scale;
     P.c_half = (float)(1.0 / (2.0 * (double)p->alpha));
     P.norm = p->norm;
@@ -423,14 +490,18 @@ int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
     const int grid = (int)(n_rows < p->sm_count ? n_rows : p->sm_count);
     const bool pdl = p->pdl != 0;
     cudaError_t e;
+#define GBS_UVM_LAUNCH(B, GL)                                                                   \
+    (p->group ? launch(k_tc_uvm_rq<B, GL, true>, grid, smem, stream, pdl, tmap, P)               \
+              : launch(k_tc_uvm_rq<B, GL, false>, grid, smem, stream, pdl, tmap, P))
     if (p->bits == 3) {
-        if (glog == 1) e = launch(k_tc_uvm_rq<3, 1>, grid, smem, stream, pdl, tmap, P);
-        else if (glog == 2) e = launch(k_tc_uvm_rq<3, 2>, grid, smem, stream, pdl, tmap, P);
-        else e = launch(k_tc_uvm_rq<3, 3>, grid, smem, stream, pdl, tmap, P);
+        if (glog == 1) e = GBS_UVM_LAUNCH(3, 1);
+        else if (glog == 2) e = GBS_UVM_LAUNCH(3, 2);
+        else e = GBS_UVM_LAUNCH(3, 3);
     } else {
-        if (glog == 1) e = launch(k_tc_uvm_rq<4, 1>, grid, smem, stream, pdl, tmap, P);
-        else if (glog == 2) e = launch(k_tc_uvm_rq<4, 2>, grid, smem, stream, pdl, tmap, P);
-        else e = launch(k_tc_uvm_rq<4, 3>, grid, smem, stream, pdl, tmap, P);
+        if (glog == 1) e = GBS_UVM_LAUNCH(4, 1);
+        else if (glog == 2) e = GBS_UVM_LAUNCH(4, 2);
+        else e = GBS_UVM_LAUNCH(4, 3);
     }
+#undef GBS_UVM_LAUNCH
     return (int)e;
 }

@@ -234,35 +234,52 @@ def test_tensor_core_family_shapes(d, d_pad, m, bits, group, alpha, rows):
 
 
 UVM_SHAPES = [
-    # d, d_pad, m, bits, alpha, rows
-    (8192, 8192, 1, 3, 0.9, 149),
-    (8192 - 64, 8192, 1, 4, 0.9, 1),
-    (16384, 16384, 1, 4, 0.8, 37),
-    (16000, 16384, 1, 3, 1.0, 150),
-    (12288, 12288, 12, 3, 0.9, 75),
-    (18944, 20480, 20, 4, 0.95, 301),
-    (20480, 20480, 20, 3, 0.9, 4),
-    (24576, 24576, 24, 4, 0.9, 33),
-    (28672, 28672, 28, 3, 0.85, 150),
-    (32768, 32768, 1, 4, 0.9, 31),
+    # d, d_pad, m, bits, alpha, rows, group
+    (8192, 8192, 1, 3, 0.9, 149, 0),
+    (8192 - 64, 8192, 1, 4, 0.9, 1, 0),
+    (16384, 16384, 1, 4, 0.8, 37, 0),
+    (16000, 16384, 1, 3, 1.0, 150, 0),
+    (12288, 12288, 12, 3, 0.9, 75, 0),
+    (18944, 20480, 20, 4, 0.95, 301, 0),
+    (20480, 20480, 20, 3, 0.9, 4, 0),
+    (24576, 24576, 24, 4, 0.9, 33, 0),
+    (28672, 28672, 28, 3, 0.85, 150, 0),
+    (32768, 32768, 1, 4, 0.9, 31, 0),
+    # per-group scales: a group is part of a lane's chunks, one lane, or several lanes of a warp
+    (8192, 8192, 1, 3, 0.9, 149, 32),
+    (8192, 8192, 1, 4, 0.9, 30, 64),
+    (8192 - 64, 8192, 1, 3, 0.8, 151, 128),
+    (8192, 8192, 1, 4, 1.0, 17, 2048),
+    (8192, 8192, 1, 3, 0.9, 40, 4096),
+    (12288, 12288, 12, 4, 0.9, 75, 64),
+    (12288, 12288, 12, 3, 0.9, 150, 128),
+    (16384, 16384, 1, 3, 0.9, 37, 256),
+    (18944, 20480, 20, 4, 0.95, 301, 128),
+    (18944, 20480, 20, 3, 0.9, 149, 32),
+    (18944, 20480, 20, 3, 0.9, 33, 256),
+    (20480, 20480, 20, 4, 0.85, 150, 512),
+    (18944, 20480, 20, 4, 0.9, 9, 1024),
+    (16000, 16384, 1, 3, 1.0, 150, 4096),
+    (28672, 28672, 28, 4, 0.9, 50, 128),
+    (32768, 32768, 1, 3, 0.9, 31, 8192),
 ]
 
 
-@pytest.mark.parametrize("d,d_pad,m,bits,alpha,rows", UVM_SHAPES)
-def test_wide_family_shapes(d, d_pad, m, bits, alpha, rows):
+@pytest.mark.parametrize("d,d_pad,m,bits,alpha,rows,group", UVM_SHAPES)
+def test_wide_family_shapes(d, d_pad, m, bits, alpha, rows, group):
     """4096 < d' <= 32768: tensor cores for H_m (x) H_{2^j}, two register sweeps over TMEM for the rest."""
-    rng = np.random.Generator(np.random.PCG64(d * 3 + m + bits + rows))
+    rng = np.random.Generator(np.random.PCG64(d * 3 + m + bits + rows + group))
     xs = rng.standard_t(3, size=(rows, d))
     xs[:, rng.integers(0, d, 3)] *= 40
     if rows > 2:
         xs[2, :] = 0.0
     x = torch.from_numpy(xs.astype(np.float32)).to(torch.bfloat16)
-    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(x), d, d_pad, m, bits, 0, alpha)
-    with Plan(d, d_pad, m, bits, 0, alpha) as plan:
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(x), d, d_pad, m, bits, group, alpha)
+    with Plan(d, d_pad, m, bits, group, alpha) as plan:
         assert plan.info.variant == 3, "the wide tensor-core family must be the one that runs for this plan"
         codes, scales, y = _run_rq(plan, x.to(DEV), rows)
         assert plan.device_status() == 0
-        stats = compare_rotate_quantize(x, ref, codes, scales, y, bits, 0, d_pad)
+        stats = compare_rotate_quantize(x, ref, codes, scales, y, bits, group, d_pad)
         print(stats)
         if rows > 2:
             assert int(codes[2].max()) == 0 and float(scales[2].abs().max()) == 0.0
