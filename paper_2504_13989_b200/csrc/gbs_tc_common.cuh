@@ -79,6 +79,15 @@ __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, v
         ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2) : "memory");
 }
 
+// L2 prefetch of the box a later tma_load_3d with the same coordinates will fetch.  It moves lines from
+// DRAM into L2 only, and L2 is where all global writes of the device land, so it is harmless to issue
+// while an earlier kernel in the stream may still be writing the tensor: nothing is read into the SM.
+__device__ __forceinline__ void tma_prefetch_3d(const CUtensorMap* map, int c0, int c1, int c2)
+{
+    asm volatile("cp.async.bulk.prefetch.tensor.3d.L2.global [%0, {%1, %2, %3}];"
+                 ::"l"(map), "r"(c0), "r"(c1), "r"(c2) : "memory");
+}
+
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, void* bar)
 {
     asm volatile(

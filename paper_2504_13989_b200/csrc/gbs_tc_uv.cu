@@ -146,7 +146,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         mbar_arrive_expect_tx(&S->abar, A_BYTES);
         bulk_load(S->a, P.a_img, A_BYTES, &S->abar);          // plan-owned, immutable: needs no ordering
-        // programmatic dependent launch: nothing of the caller's memory is touched before this point
+        // programmatic dependent launch: until the wait below returns, an earlier kernel of the stream may
+        // still be writing the rows.  Nothing of the caller's memory reaches this SM before it; the first
+        // tile is only pulled from DRAM into L2 meanwhile, so that the load that follows the wait hits there
+        // (one tile, not all four stages: more prefetches queue ahead of the other CTAs' first loads).
+        if ((int)blockIdx.x < P.n_groups) tma_prefetch_3d(&tmap, 0, 0, blockIdx.x * TOK);
         asm volatile("griddepcontrol.wait;" ::: "memory");
         for (int g = blockIdx.x; it_p < STAGES && g < P.n_groups; g += gridDim.x, ++it_p) {
             mbar_arrive_expect_tx(&S->full[it_p], stage_bytes);
