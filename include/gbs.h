@@ -91,8 +91,9 @@ typedef struct gbs_plan_info {
  * Section 2.1 / 3.1 for bits and alpha).
  *   d       row width, 1 <= d <= d_pad
  *   d_pad   d' = m * 2^k with 2^k >= 8 and d' <= GBS_MAX_D_PAD
- *   m       1 (pure Sylvester), or 12, 20, 24 (Algorithm 2 with p = m-1), or 28 (Algorithm 2
- *           over GF(27) = GF(3)[x]/(x^3+2x+1), elements indexed c0 + 3 c1 + 9 c2)
+ *   m       1 (pure Sylvester); 12, 20, 24, 44, 48, 60, 68, 72, 80, 84, 104 or 108 (Algorithm 2 with the
+ *           prime p = m-1 = 3 mod 4); or 28 (Algorithm 2 over GF(27) = GF(3)[x]/(x^3+2x+1), elements
+ *           indexed c0 + 3 c1 + 9 c2).  Other orders return GBS_ERR_UNSUPPORTED.
  *   bits    3 or 4
  *   group   0, or a power of two >= 8 dividing 2^k (so a group never straddles a block of H_m)
  *   alpha   0 < alpha <= 1

@@ -129,6 +129,9 @@ __device__ __forceinline__ void paley_mix(float* row, const float* hm_s, int n2,
     }
 }
 
+// WIDE selects the orders above 28: their register-held columns (up to 108 values per thread) would
+// double the register count of every kernel here, so they get instantiations of their own.
+template <bool WIDE>
 __device__ __forceinline__ void run_passes_and_mix(const GenericParams& P, float* row, const float* hm_s,
                                                    int j, int tt)
 {
@@ -144,18 +147,30 @@ __device__ __forceinline__ void run_passes_and_mix(const GenericParams& P, float
     }
     if (P.m > 1) {
         __syncthreads();
-        switch (P.m) {
-            case 12: paley_mix<12>(row, hm_s, P.n2, j, tt); break;
-            case 20: paley_mix<20>(row, hm_s, P.n2, j, tt); break;
-            case 24: paley_mix<24>(row, hm_s, P.n2, j, tt); break;
-            default: paley_mix<28>(row, hm_s, P.n2, j, tt); break;
+        if constexpr (!WIDE) {
+            switch (P.m) {
+                case 12: paley_mix<12>(row, hm_s, P.n2, j, tt); break;
+                case 20: paley_mix<20>(row, hm_s, P.n2, j, tt); break;
+                case 24: paley_mix<24>(row, hm_s, P.n2, j, tt); break;
+                default: paley_mix<28>(row, hm_s, P.n2, j, tt); break;
+            }
+        } else switch (P.m) {
+            case 44: paley_mix<44>(row, hm_s, P.n2, j, tt); break;
+            case 48: paley_mix<48>(row, hm_s, P.n2, j, tt); break;
+            case 60: paley_mix<60>(row, hm_s, P.n2, j, tt); break;
+            case 68: paley_mix<68>(row, hm_s, P.n2, j, tt); break;
+            case 72: paley_mix<72>(row, hm_s, P.n2, j, tt); break;
+            case 80: paley_mix<80>(row, hm_s, P.n2, j, tt); break;
+            case 84: paley_mix<84>(row, hm_s, P.n2, j, tt); break;
+            case 104: paley_mix<104>(row, hm_s, P.n2, j, tt); break;
+            default: paley_mix<108>(row, hm_s, P.n2, j, tt); break;
         }
     }
     __syncthreads();
 }
 
 // Load + pad + first three butterfly stages in registers -> shared memory, then the rest.
-template <typename InT>
+template <typename InT, bool WIDE>
 __device__ __forceinline__ void rotate_row_to_smem(const GenericParams& P, const InT* x, long long row,
                                                    bool active, float* rowbuf, const float* hm_s, int j,
                                                    int tt)
@@ -171,7 +186,7 @@ __device__ __forceinline__ void rotate_row_to_smem(const GenericParams& P, const
             for (int e = 0; e < 8; ++e) rowbuf[p + e] = v[e];
         }
     }
-    run_passes_and_mix(P, rowbuf, hm_s, j, tt);
+    run_passes_and_mix<WIDE>(P, rowbuf, hm_s, j, tt);
 }
 
 // max|.| of a group of G consecutive values, each thread holding the max of its 8-value chunk.
@@ -256,7 +271,7 @@ __device__ __forceinline__ void clear_gmax(const GenericParams& P, unsigned* gma
 // ======================================================================================
 // rotate + quantize + pack
 // ======================================================================================
-template <typename InT, int BITS>
+template <typename InT, int BITS, bool WIDE>
 __global__ void __launch_bounds__(NT) k_rotate_quantize(GenericParams P, const InT* __restrict__ x,
                                                         unsigned char* __restrict__ codes,
                                                         float* __restrict__ scales, float* __restrict__ y_opt)
@@ -279,7 +294,7 @@ __global__ void __launch_bounds__(NT) k_rotate_quantize(GenericParams P, const I
         const long long row = row0 + team;
         const bool active = row < P.n_rows;
         clear_gmax(P, L.gmax);
-        rotate_row_to_smem<InT>(P, x, row, active, rowbuf, L.hm_s, j, tt);
+        rotate_row_to_smem<InT, WIDE>(P, x, row, active, rowbuf, L.hm_s, j, tt);
         row_group_max(P, rowbuf, gmax, active, j, tt);
 
         if (active) {
@@ -337,7 +352,7 @@ struct ClipConsts {
     float c_inv[GBS_MAX_CANDIDATES];     // D / alpha_k
 };
 
-template <typename InT>
+template <typename InT, bool WIDE>
 __global__ void __launch_bounds__(NT) k_clip_error(GenericParams P, ClipConsts C, int K,
                                                    const InT* __restrict__ x, double* __restrict__ err_sum,
                                                    float* __restrict__ err_rows)
@@ -366,7 +381,7 @@ __global__ void __launch_bounds__(NT) k_clip_error(GenericParams P, ClipConsts C
         const bool active = row < P.n_rows;
         clear_gmax(P, L.gmax);
         for (int i = threadIdx.x; i < P.rows_per_cta * GBS_MAX_CANDIDATES; i += NT) row_err_all[i] = 0.f;
-        rotate_row_to_smem<InT>(P, x, row, active, rowbuf, L.hm_s, j, tt);
+        rotate_row_to_smem<InT, WIDE>(P, x, row, active, rowbuf, L.hm_s, j, tt);
         row_group_max(P, rowbuf, gmax, active, j, tt);
 
         for (int k0 = 0; k0 < K; k0 += KT) {
@@ -489,7 +504,7 @@ __global__ void __launch_bounds__(NT) k_dequantize_plain(int d_pad, int G, int s
 }
 
 // xhat = (H^T yhat / sqrt(d'))[0:d]: same shared-memory machinery with the transposed H_m.
-template <typename OutT, int BITS>
+template <typename OutT, int BITS, bool WIDE>
 __global__ void __launch_bounds__(NT) k_dequantize_inverse(GenericParams P, const unsigned char* __restrict__ codes,
                                                            const float* __restrict__ scales,
                                                            OutT* __restrict__ out)
@@ -518,7 +533,7 @@ __global__ void __launch_bounds__(NT) k_dequantize_inverse(GenericParams P, cons
                 for (int e = 0; e < 8; ++e) rowbuf[p + e] = v[e];
             }
         }
-        run_passes_and_mix(P, rowbuf, L.hm_s, j, tt);
+        run_passes_and_mix<WIDE>(P, rowbuf, L.hm_s, j, tt);
         if (active) {
             OutT* orow = out + row * P.d;
             for (int i = j; i < P.d; i += tt) store1(orow + i, rowbuf[pidx(i)] * P.norm);
@@ -616,17 +631,22 @@ int gbs_generic_rotate_quantize(const gbs_plan* p, const void* x, int x_dtype, i
     const size_t smem = base_smem(P) + (size_t)P.rows_per_cta * P.stage_bytes;
     const int grid = grid_for(p, P, smem);
     cudaError_t e;
-#define LAUNCH_RQ(T, B)                                                                       \
+#define LAUNCH_RQ_W(T, B, W)                                                                  \
     do {                                                                                      \
-        e = prep(k_rotate_quantize<T, B>, smem);                                              \
+        e = prep(k_rotate_quantize<T, B, W>, smem);                                           \
         if (e == cudaSuccess) {                                                               \
-            k_rotate_quantize<T, B><<<grid, NT, smem, stream>>>(P, (const T*)x, (unsigned char*)codes, scales, y_opt); \
+            k_rotate_quantize<T, B, W><<<grid, NT, smem, stream>>>(P, (const T*)x, (unsigned char*)codes, scales, y_opt); \
             e = cudaGetLastError();                                                           \
         }                                                                                     \
+    } while (0)
+#define LAUNCH_RQ(T, B)                                                                       \
+    do {                                                                                      \
+        if (p->m > 28) LAUNCH_RQ_W(T, B, true); else LAUNCH_RQ_W(T, B, false);                \
     } while (0)
     if (x_dtype == GBS_DTYPE_F32) { if (p->bits == 3) LAUNCH_RQ(float, 3); else LAUNCH_RQ(float, 4); }
     else { if (p->bits == 3) LAUNCH_RQ(__nv_bfloat16, 3); else LAUNCH_RQ(__nv_bfloat16, 4); }
 #undef LAUNCH_RQ
+#undef LAUNCH_RQ_W
     return (int)e;
 }
 
@@ -645,19 +665,17 @@ int gbs_generic_clip_error(const gbs_plan* p, const void* x, int x_dtype, int64_
                        sizeof(float) * (size_t)P.rows_per_cta * GBS_MAX_CANDIDATES;
     const int grid = grid_for(p, P, smem);
     cudaError_t e;
-    if (x_dtype == GBS_DTYPE_F32) {
-        e = prep(k_clip_error<float>, smem);
-        if (e == cudaSuccess) {
-            k_clip_error<float><<<grid, NT, smem, stream>>>(P, C, K, (const float*)x, err_sum, err_rows);
-            e = cudaGetLastError();
-        }
-    } else {
-        e = prep(k_clip_error<__nv_bfloat16>, smem);
-        if (e == cudaSuccess) {
-            k_clip_error<__nv_bfloat16><<<grid, NT, smem, stream>>>(P, C, K, (const __nv_bfloat16*)x, err_sum, err_rows);
-            e = cudaGetLastError();
-        }
-    }
+#define LAUNCH_CE(T, W)                                                                       \
+    do {                                                                                      \
+        e = prep(k_clip_error<T, W>, smem);                                                   \
+        if (e == cudaSuccess) {                                                               \
+            k_clip_error<T, W><<<grid, NT, smem, stream>>>(P, C, K, (const T*)x, err_sum, err_rows); \
+            e = cudaGetLastError();                                                           \
+        }                                                                                     \
+    } while (0)
+    if (x_dtype == GBS_DTYPE_F32) { if (p->m > 28) LAUNCH_CE(float, true); else LAUNCH_CE(float, false); }
+    else { if (p->m > 28) LAUNCH_CE(__nv_bfloat16, true); else LAUNCH_CE(__nv_bfloat16, false); }
+#undef LAUNCH_CE
     return (int)e;
 }
 
@@ -685,16 +703,21 @@ int gbs_generic_dequantize(const gbs_plan* p, const void* codes, const float* sc
     }
     const size_t smem = base_smem(P);
     const int grid = grid_for(p, P, smem);
-#define LAUNCH_DI(T, B)                                                                            \
+#define LAUNCH_DI_W(T, B, W)                                                                       \
     do {                                                                                           \
-        e = prep(k_dequantize_inverse<T, B>, smem);                                                \
+        e = prep(k_dequantize_inverse<T, B, W>, smem);                                             \
         if (e == cudaSuccess) {                                                                    \
-            k_dequantize_inverse<T, B><<<grid, NT, smem, stream>>>(P, (const unsigned char*)codes, scales, (T*)out); \
+            k_dequantize_inverse<T, B, W><<<grid, NT, smem, stream>>>(P, (const unsigned char*)codes, scales, (T*)out); \
             e = cudaGetLastError();                                                                \
         }                                                                                          \
+    } while (0)
+#define LAUNCH_DI(T, B)                                                                            \
+    do {                                                                                           \
+        if (p->m > 28) LAUNCH_DI_W(T, B, true); else LAUNCH_DI_W(T, B, false);                     \
     } while (0)
     if (out_dtype == GBS_DTYPE_F32) { if (p->bits == 3) LAUNCH_DI(float, 3); else LAUNCH_DI(float, 4); }
     else { if (p->bits == 3) LAUNCH_DI(__nv_bfloat16, 3); else LAUNCH_DI(__nv_bfloat16, 4); }
 #undef LAUNCH_DI
+#undef LAUNCH_DI_W
     return (int)e;
 }

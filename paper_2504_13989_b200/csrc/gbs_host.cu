@@ -19,7 +19,7 @@ int log2_exact(int v)
     return l;
 }
 
-bool supported_m(int m) { return m == 1 || m == 12 || m == 20 || m == 24 || m == 28; }
+bool supported_m(int m) { return gbs_supported_m(m); }
 
 int elem_size(int dtype) { return dtype == GBS_DTYPE_F32 ? 4 : 2; }
 
@@ -158,15 +158,17 @@ extern "C" int gbs_plan_create_ex(gbs_plan_t** out, int d, int d_pad, int m, int
     p->pdl = (nopdl && nopdl[0] == '1') ? 0 : 1;
 
     if (m > 1) {
-        float h[2 * 32 * 32];
+        float* h = new (std::nothrow) float[(size_t)2 * m * m];
+        if (!h) { cudaFree(p->d_status); if (p->d_aimg) cudaFree(p->d_aimg); delete p; return GBS_ERR_ALLOC; }
         for (int i = 0; i < m; ++i)
             for (int j = 0; j < m; ++j) {
                 h[i * m + j] = (float)p->h_hm[i * m + j];
                 h[m * m + j * m + i] = (float)p->h_hm[i * m + j];     // transpose, for the inverse rotation
             }
         e = cudaMalloc(&p->d_hm, sizeof(float) * 2 * m * m);
-        if (e != cudaSuccess) { cudaGetLastError(); cudaFree(p->d_status); if (p->d_aimg) cudaFree(p->d_aimg); delete p; return GBS_ERR_ALLOC; }
+        if (e != cudaSuccess) { delete[] h; cudaGetLastError(); cudaFree(p->d_status); if (p->d_aimg) cudaFree(p->d_aimg); delete p; return GBS_ERR_ALLOC; }
         e = cudaMemcpy(p->d_hm, h, sizeof(float) * 2 * m * m, cudaMemcpyHostToDevice);
+        delete[] h;
         if (e != cudaSuccess) { cudaGetLastError(); cudaFree(p->d_hm); cudaFree(p->d_status); if (p->d_aimg) cudaFree(p->d_aimg); delete p; return GBS_ERR_CUDA; }
     }
     *out = p;

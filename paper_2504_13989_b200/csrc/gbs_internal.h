@@ -6,6 +6,9 @@
 
 #include "gbs.h"
 
+// Largest order of the small Hadamard factor H_m a plan accepts.
+#define GBS_MAX_M 108
+
 // Kernel families a plan can select for bf16 rows.
 enum gbs_variant {
     GBS_VARIANT_GENERIC = 0,   // shared-memory FWHT on the plain ALUs; any supported (m, k), any dtype
@@ -33,11 +36,12 @@ struct gbs_plan {
     int uvm_glog;          // UVM family: log2 of the number of 32-value chunks per tensor-core output row
     unsigned char* d_aimg; // device: pre-swizzled bf16 image of H_m (x) H_{2^j} for the tensor-core family (32 KB)
     int* d_status;         // device status word: 0, or the code of the first bounded wait that expired
-    int8_t h_hm[32 * 32];  // host copy of H_m (m <= 32)
+    int8_t h_hm[GBS_MAX_M * GBS_MAX_M];  // host copy of H_m
 };
 
 // gbs_paley.cu
 int gbs_build_hadamard_m(int m, int8_t* out);   // 0 or GBS_ERR_UNSUPPORTED
+bool gbs_supported_m(int m);                    // the orders a plan accepts
 
 // gbs_generic.cu : launches on `stream`; return a cudaError_t cast to int (0 = success)
 int gbs_generic_rotate_quantize(const gbs_plan* p, const void* x, int x_dtype, int64_t n_rows,

@@ -67,6 +67,16 @@ int gf27_minus(int e, int f)
 
 }  // namespace
 
+// Orders with a construction here: 1 (no Paley factor), p + 1 for the primes p = 3 (mod 4) up to 107
+// that are multiples of 4 not covered by a smaller factor times a power of two, and 28 = 27 + 1.
+bool gbs_supported_m(int m)
+{
+    static const int orders[] = {1, 12, 20, 24, 28, 44, 48, 60, 68, 72, 80, 84, 104, 108};
+    for (int o : orders)
+        if (m == o) return true;
+    return false;
+}
+
 int gbs_build_hadamard_m(int m, int8_t* H)
 {
     if (m == 1) { H[0] = 1; return GBS_OK; }

@@ -62,9 +62,10 @@ struct __align__(1024) Smem {
 struct UvParams {
     long long n_rows;
     int n_groups;                 // ceil(n_rows / TOK)
-    int U;                        // m * 2^j, multiple of 16, <= 128
+    int U;                        // m * 2^j, 16 <= U <= 128
+    int Upad;                     // U rounded up to a multiple of 16: rows of a token in shared memory
     int j;                        // log2 of the Sylvester part of A
-    int ksteps;                   // U / 16
+    int ksteps;                   // Upad / 16
     int code_row_bytes;           // d' * bits / 8
     int d_pad;
     int glog;                     // lane-group mode: log2(lanes per quantization group)
@@ -135,7 +136,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
     extern __shared__ unsigned char smem_raw[];
     Smem* S = reinterpret_cast<Smem*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const unsigned stage_bytes = (unsigned)(TOK * P.U * V * 2);
+    const unsigned stage_bytes = (unsigned)(TOK * P.Upad * V * 2);
 
     // ---- set-up.  Thread 0 arms the load barriers and starts the first loads at once; one thread of
     // warp 2 arms the remaining barriers; warp 1 allocates TMEM.  One block barrier joins the three.
@@ -191,7 +192,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
         if (lane == 0) {
             constexpr unsigned IDESC = instr_desc(UMAX, STAGE_COLS);
             const unsigned a_base = smem_u32(S->a);
-            const unsigned tok_bytes = (unsigned)(P.U * V * 2);
+            const unsigned tok_bytes = (unsigned)(P.Upad * V * 2);
             bool ok = mbar_wait(&S->abort_flag, &S->abar, 0, P.status, 6);
             int it = 0;
             for (int g = blockIdx.x; ok && g < P.n_groups; g += gridDim.x, ++it) {
@@ -377,7 +378,7 @@ bool gbs_tc_uv_supported(const gbs_plan* p)
 {
     if (p->d_pad % V != 0 || p->d % V != 0 || p->k < 5) return false;
     const int U = p->d_pad / V;
-    if (U > UMAX || U % 16 != 0) return false;
+    if (U > UMAX || U < 16) return false;          // U = m 2^j is a multiple of 4; the contraction is padded to 16
     if (p->group != 0 && (p->group < V || p->group / V > 32)) return false;
     return get_encode() != nullptr && p->smem_optin >= (int)(sizeof(Smem) + 1024);
 }
@@ -393,7 +394,10 @@ int uv_prepare(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride,
     const int U = p->d_pad / V;
     const cuuint64_t gdim[3] = {(cuuint64_t)V, (cuuint64_t)(p->d / V), (cuuint64_t)n_rows};
     const cuuint64_t gstr[2] = {(cuuint64_t)(V * 2), (cuuint64_t)(stride * 2)};
-    const cuuint32_t box[3] = {V, (cuuint32_t)U, TOK};
+    // rows u of the box beyond d / 32 (the zero-pad expansion, and the padding of U to a multiple of the
+    // MMA's K = 16) are filled with zeros by TMA
+    const int Upad = (U + 15) & ~15;
+    const cuuint32_t box[3] = {V, (cuuint32_t)Upad, TOK};
     const cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = encode(tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), gdim, gstr, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -404,7 +408,8 @@ int uv_prepare(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride,
     P->n_groups = (int)((n_rows + TOK - 1) / TOK);
     P->U = U;
     P->j = p->k - 5;
-    P->ksteps = U / 16;
+    P->Upad = Upad;
+    P->ksteps = Upad / 16;
     P->code_row_bytes = p->d_pad * p->bits / 8;
     P->d_pad = p->d_pad;
     P->glog = p->group ? ilog2(p->group / V) : 0;

@@ -52,9 +52,10 @@ struct __align__(1024) Smem {
 struct UvmParams {
     long long n_rows;
     int U;                        // m * 2^j
-    int ksteps;                   // U / 16
+    int Upad;                     // U rounded up to a multiple of 16
+    int ksteps;                   // Upad / 16
     int n_stages;                 // shared-memory stages in use
-    int stage_bytes;              // U * G * 64
+    int stage_bytes;              // Upad * G * 64
     int code_row_bytes;
     int d_pad;
     int gsh;                      // GROUPED: scale group = 2^gsh chunks of 32 coordinates
@@ -213,7 +214,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
         if (lane == 0) {
             constexpr unsigned IDESC = instr_desc(UMAX, NCOLS);
             const unsigned a_base = smem_u32(S->a);
-            const unsigned chunk_bytes = (unsigned)(P.U * V * 2);     // one chunk (N atom of 32): U rows of 64 bytes
+            const unsigned chunk_bytes = (unsigned)(P.Upad * V * 2);  // one chunk (N atom of 32): Upad rows of 64 bytes
             bool ok = mbar_wait(&S->abort_flag, &S->abar, 0, P.status, 6);
             int it = 0;
             for (int tk = blockIdx.x; ok && tk < n_tok; tk += gridDim.x, ++it) {
@@ -439,7 +440,7 @@ int gbs_tc_uvm_glog(const gbs_plan* p)
         if (p->d_pad % span != 0 || p->d % span != 0) continue;
         if (p->group != 0 && gsh > g + 5) continue;          // a group may span at most the 32 lanes of a warp
         const int U = p->d_pad / span;
-        if (U > UMAX || U % 16 != 0 || p->k - 5 - g < 0) continue;
+        if (U > UMAX || U < 16 || p->k - 5 - g < 0) continue;
         if (get_encode() == nullptr || p->smem_optin < (int)(sizeof(Smem) + 1024)) return 0;
         return g;
     }
@@ -458,7 +459,8 @@ int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
     CUtensorMap tmap;
     const cuuint64_t gdim[4] = {(cuuint64_t)V, (cuuint64_t)G, (cuuint64_t)(p->d / (V * G)), (cuuint64_t)n_rows};
     const cuuint64_t gstr[3] = {(cuuint64_t)(V * 2), (cuuint64_t)(V * G * 2), (cuuint64_t)(stride * 2)};
-    const cuuint32_t box[4] = {V, 1, (cuuint32_t)U, 1};
+    const int Upad = (U + 15) & ~15;       // the contraction is padded to the MMA's K = 16; TMA zero-fills the rows
+    const cuuint32_t box[4] = {V, 1, (cuuint32_t)Upad, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     CUresult r = encode(&tmap, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(x), gdim, gstr, box, estr,
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -469,8 +471,9 @@ int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
     memset(&P, 0, sizeof(P));
     P.n_rows = n_rows;
     P.U = U;
-    P.ksteps = U / 16;
-    P.stage_bytes = U * G * V * 2;
+    P.Upad = Upad;
+    P.ksteps = Upad / 16;
+    P.stage_bytes = Upad * G * V * 2;
     P.n_stages = B_BYTES / P.stage_bytes < MAX_STAGES ? B_BYTES / P.stage_bytes : MAX_STAGES;
     P.code_row_bytes = p->d_pad * p->bits / 8;
     P.d_pad = p->d_pad;

@@ -39,7 +39,7 @@ def test_status_strings(lib):
     assert "unknown" in binding.status_string(-99)
 
 
-@pytest.mark.parametrize("m", [1, 12, 20, 24, 28])
+@pytest.mark.parametrize("m", [1, 12, 20, 24, 28, 44, 48, 60, 68, 72, 80, 84, 104, 108])
 def test_library_and_oracle_build_the_same_small_hadamard(m, lib):
     """Two independently written constructions (Euler criterion / discrete logs in the library,
     exhaustive squaring in the oracle) must give one canonical matrix (Algorithm 2)."""
@@ -50,7 +50,7 @@ def test_library_and_oracle_build_the_same_small_hadamard(m, lib):
 
 def test_hadamard_m_rejects_unsupported_orders(lib):
     buf = (ctypes.c_int8 * 4096)()
-    for m in (2, 3, 6, 16, 36, 44):
+    for m in (2, 3, 6, 16, 36, 52, 112):
         assert lib.gbs_hadamard_m(m, buf) == binding.GBS_ERR_UNSUPPORTED
     assert lib.gbs_hadamard_m(0, buf) == binding.GBS_ERR_INVALID_ARG
     assert lib.gbs_hadamard_m(12, None) == binding.GBS_ERR_INVALID_ARG
@@ -73,7 +73,7 @@ BAD_PLANS = [
     (128, 128, 1, 4, 256, 1.0, binding.GBS_ERR_INVALID_ARG),   # group > 2^k
     (3584, 3584, 28, 3, 256, 1.0, binding.GBS_ERR_INVALID_ARG),  # group straddles blocks of H_28
     (128, 128, 16, 4, 0, 1.0, binding.GBS_ERR_UNSUPPORTED),    # no construction for m = 16
-    (352, 352, 44, 4, 0, 1.0, binding.GBS_ERR_UNSUPPORTED),    # m = 44 not in the build list
+    (416, 416, 52, 4, 0, 1.0, binding.GBS_ERR_UNSUPPORTED),    # 51 is not prime: no construction for m = 52
     (65536, 65536, 1, 4, 0, 1.0, binding.GBS_ERR_UNSUPPORTED),  # d' too large
 ]
 

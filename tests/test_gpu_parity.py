@@ -199,6 +199,20 @@ UV_SHAPES = [
     (3520, 3584, 28, 3, 32, 1.0, 21),
     (4096, 4096, 1, 3, 1024, 0.9, 50),
     (4096, 4096, 1, 4, 128, 0.9, 50),
+    # orders beyond 28, and factors U = m 2^j that are not multiples of the MMA's K = 16 (zero-padded)
+    (768, 768, 12, 4, 0, 0.9, 33),
+    (1408, 1408, 44, 3, 32, 0.9, 41),
+    (2816, 2816, 44, 4, 0, 0.9, 77),
+    (3072, 3072, 48, 4, 64, 0.9, 30),
+    (1920, 1920, 60, 3, 0, 0.9, 150),
+    (3840, 3840, 60, 4, 64, 0.8, 35),
+    (2176, 2176, 68, 3, 0, 1.0, 20),
+    (2304, 2304, 72, 4, 32, 0.9, 20),
+    (2560, 2560, 80, 3, 32, 0.9, 20),
+    (2688, 2688, 84, 3, 0, 0.9, 149),
+    (3328, 3328, 104, 4, 0, 0.9, 20),
+    (3456, 3456, 108, 4, 32, 0.85, 75),
+    (3296, 3456, 108, 3, 0, 0.9, 9),
 ]
 
 
@@ -262,6 +276,13 @@ UVM_SHAPES = [
     (16000, 16384, 1, 3, 1.0, 150, 4096),
     (28672, 28672, 28, 4, 0.9, 50, 128),
     (32768, 32768, 1, 3, 0.9, 31, 8192),
+    # orders beyond 28 (11008 -> 11264 = 44 * 256 and 13824 = 108 * 128 are MLP widths of 7B / 13B models)
+    (11008, 11264, 44, 4, 0.9, 75, 0),
+    (11008, 11264, 44, 3, 0.9, 40, 128),
+    (13824, 13824, 108, 4, 0.9, 33, 0),
+    (13824, 13824, 108, 3, 0.85, 33, 128),
+    (7680, 7680, 60, 3, 0.9, 50, 0),
+    (8704, 8704, 68, 4, 0.9, 21, 64),
 ]
 
 
@@ -388,6 +409,17 @@ SHAPES = [
     (32768, 32768, 1, 3, 0, 1.0, 2, torch.float32),
     (20480, 20480, 20, 3, 1024, 0.9, 3, torch.bfloat16),
     (28672, 28672, 28, 4, 0, 0.9, 2, torch.bfloat16),
+    # orders beyond 28 on the generic family
+    (352, 352, 44, 4, 8, 0.9, 21, torch.float32),
+    (384, 384, 48, 3, 0, 0.9, 21, torch.bfloat16),
+    (480, 480, 60, 3, 8, 1.0, 11, torch.bfloat16),
+    (544, 544, 68, 4, 0, 0.9, 11, torch.float32),
+    (570, 576, 72, 3, 8, 0.9, 11, torch.float32),
+    (640, 640, 80, 4, 0, 0.9, 11, torch.bfloat16),
+    (672, 672, 84, 3, 0, 0.7, 11, torch.float32),
+    (832, 832, 104, 4, 8, 0.9, 5, torch.float32),
+    (864, 864, 108, 3, 0, 0.9, 9, torch.float32),
+    (13824, 13824, 108, 4, 128, 0.9, 3, torch.float32),
 ]
 
 
