@@ -269,6 +269,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--nsets", type=int, default=16)
+    ap.add_argument("--e2e-chunks", type=int, default=4, help="row chunks of the host-buffer pipeline (copies overlap)")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-extras", action="store_true", help="skip the context legs under `also`")
     ap.add_argument("--profile", default=None, metavar="WORKLOAD[:ROWS]",
@@ -298,7 +299,7 @@ def main():
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=device)
 
-    from paper_2504_13989_b200 import Plan, synth
+    from paper_2504_13989_b200 import HostPipeline, Plan, synth
     from paper_2504_13989_b200 import build as gbs_build
     gbs_build.build()
 
@@ -341,13 +342,10 @@ def main():
                           torch.empty((w.n_rows, pl.info.scales_per_row), dtype=torch.float32).pin_memory()))
     e2e_steps = max(3, min(args.steps, 20))
 
+    pipe = HostPipeline(plans, w.n_rows, device=device, chunks=args.e2e_chunks)
+
     def e2e_step():
-        with torch.cuda.stream(stream):
-            xd = x_pin.to(device, non_blocking=True)
-            for pl, (ch, sh) in zip(plans, host_outs):
-                c, s, _ = pl.rotate_quantize(xd, stream=stream)
-                ch.copy_(c, non_blocking=True)
-                sh.copy_(s, non_blocking=True)
+        pipe.run(x_pin, host_outs, stream=stream)
     for _ in range(3):
         e2e_step()
     stream.synchronize()

@@ -317,3 +317,45 @@ class Plan:
             scales_host.copy_(scales, non_blocking=True)
         s.synchronize()
         return codes_host, scales_host
+
+
+class HostPipeline:
+    """Host-resident rows through one or more plans: pinned host -> device -> kernels -> pinned host.
+
+    The rows are cut into `chunks` row ranges.  Chunk i+1 is copied to the device on a copy stream
+    while chunk i is quantized and its codes and scales travel back on the compute stream, so the
+    two PCIe directions work at the same time.  Only copies, events and the plans' launches happen
+    here; staging buffers on the device are allocated once.
+    """
+
+    def __init__(self, plans, n_rows: int, device="cuda:0", chunks: int = 4, dtype=torch.bfloat16):
+        self.plans = list(plans)
+        d = self.plans[0].info.d
+        assert all(p.info.d == d for p in self.plans)
+        self.n_rows, self.d = n_rows, d
+        chunks = max(1, min(chunks, n_rows)) if n_rows else 1
+        step = (n_rows + chunks - 1) // chunks if n_rows else 0
+        self.ranges = [(r, min(n_rows, r + step)) for r in range(0, n_rows, step)] if n_rows else []
+        self.x_dev = torch.empty((n_rows, d), dtype=dtype, device=device)
+        self.outs = [p.alloc_outputs(n_rows, device) for p in self.plans]
+        self.copy_stream = torch.cuda.Stream(device=device)
+        self.ev_in = [torch.cuda.Event() for _ in self.ranges]
+        self.ev_start = torch.cuda.Event()
+
+    def run(self, x_host: torch.Tensor, outs_host, stream=None):
+        """outs_host: one (codes_host, scales_host) pair per plan.  Work is enqueued on `stream` (and the
+        internal copy stream, joined to it); the caller synchronises `stream`."""
+        s = stream or torch.cuda.current_stream()
+        self.ev_start.record(s)
+        self.copy_stream.wait_event(self.ev_start)          # staging buffers of the previous call are free
+        for i, (r0, r1) in enumerate(self.ranges):
+            with torch.cuda.stream(self.copy_stream):
+                self.x_dev[r0:r1].copy_(x_host[r0:r1], non_blocking=True)
+                self.ev_in[i].record(self.copy_stream)
+            with torch.cuda.stream(s):
+                s.wait_event(self.ev_in[i])
+                for p, (codes, scales, _), (ch, sh) in zip(self.plans, self.outs, outs_host):
+                    gbs_rotate_quantize(p.handle, self.x_dev[r0:r1], codes[r0:r1], scales[r0:r1], None, s)
+                    ch[r0:r1].copy_(codes[r0:r1], non_blocking=True)
+                    sh[r0:r1].copy_(scales[r0:r1], non_blocking=True)
+        return outs_host

@@ -536,3 +536,26 @@ def test_expansion_identity_of_eq_2_through_the_library(d, d_pad, m):
     got = (yx.double() @ yw.double().T).cpu().numpy()
     want = x.double().numpy() @ wt.double().numpy().T
     np.testing.assert_allclose(got, want, rtol=0, atol=2e-5 * np.abs(want).max() + 1e-6)
+
+
+@pytest.mark.parametrize("rows,chunks", [(1000, 4), (3, 8), (257, 1), (0, 4)])
+def test_host_pipeline_equals_the_one_shot_call(rows, chunks):
+    """Pinned host rows through two plans in overlapping chunks: byte-identical to device-resident calls."""
+    from paper_2504_13989_b200 import HostPipeline
+    d = 512
+    rng = np.random.Generator(np.random.PCG64(rows + chunks))
+    x = torch.from_numpy(rng.standard_t(3, size=(rows, d)).astype(np.float32)).to(torch.bfloat16).pin_memory()
+    with Plan(d, d, 1, 3, 0, 0.9) as p3, Plan(d, d, 1, 4, 64, 0.8) as p4:
+        plans = [p3, p4]
+        outs = [(torch.zeros((rows, p.info.code_bytes_per_row), dtype=torch.uint8).pin_memory(),
+                 torch.zeros((rows, p.info.scales_per_row), dtype=torch.float32).pin_memory()) for p in plans]
+        pipe = HostPipeline(plans, rows, device=DEV, chunks=chunks)
+        st = torch.cuda.Stream()
+        for _ in range(2):                      # twice: the staging buffers are reused
+            pipe.run(x, outs, stream=st)
+        st.synchronize()
+        for p, (ch, sh) in zip(plans, outs):
+            if rows == 0:
+                continue
+            c, s, _ = _run_rq(p, x.to(DEV), rows, want_y=False)
+            assert torch.equal(ch, c.cpu()) and torch.equal(sh, s.cpu())
