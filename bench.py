@@ -493,6 +493,11 @@ def extras(device, stream, args, peak):
     ms = time_loop(lambda i: pl.dequantize(codes, scales, out=yhat, stream=stream), 50)
     dq_bytes = w.n_rows * (w.d_pad * 3 // 8 + 4 + w.d_pad * 2)
     out["dequantize_b3_bf16"] = {"us_per_launch": ms * 1e3, "gbs": dq_bytes / ms / 1e6}
+    xhat = torch.empty((w.n_rows, w.d), dtype=torch.bfloat16, device=device)
+    ms = time_loop(lambda i: pl.dequantize(codes, scales, inverse=True, out=xhat, stream=stream), 50)
+    out["dequantize_inverse_rotate_b3_bf16"] = {"us_per_launch": ms * 1e3,
+                                                "gbs": w.n_rows * (w.d_pad * 3 // 8 + 4 + w.d * 2) / ms / 1e6}
+    del xhat
     # clip-ratio scoring, K = 32, on a 32768-token sample of one calibration layer (262144 tokens x 4096)
     del x, codes, scales, yhat
     wc = synth.WORKLOADS["calib4096"]

@@ -132,14 +132,32 @@ extern "C" int gbs_plan_create_ex(gbs_plan_t** out, int d, int d_pad, int m, int
     const bool tc_row = want_tc && !tc_uv && gbs_tc_row_supported(p);
     const int uvm_glog = (want_tc && !tc_uv && !tc_row) ? gbs_tc_uvm_glog(p) : 0;
     if (tc_uv || tc_row || uvm_glog) {
-        unsigned char* img = (unsigned char*)malloc(32768);
+        // the UV family with one symmetric scale per token also gets the image of the transpose, behind the
+        // first one in the same allocation, for gbs_dequantize's inverse rotation on the tensor cores
+        const bool with_t = tc_uv && p->group == 0 && !p->asym;
+        const size_t img_bytes = with_t ? 65536 : 32768;
+        unsigned char* img = (unsigned char*)malloc(img_bytes);
         if (!img) { cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC; }
         if (tc_uv) gbs_tc_uv_a_image(p, img);
+        if (with_t) {
+            const int j = p->k - 5, U = p->d_pad / 32;
+            gbs_tc_sign_image(p->h_hm, p->m, j, U, img + 32768, true);
+            for (int c = 0; c < U; ++c) {
+                int sum = 0;
+                for (int r = 0; r < U; ++r) {
+                    int sign = p->h_hm[(r >> j) * p->m + (c >> j)];
+                    if (__builtin_popcount((unsigned)(r & c & ((1 << j) - 1))) & 1) sign = -sign;
+                    sum += sign;
+                }
+                p->a_colsum[c] = sum;
+            }
+        }
         else if (tc_row) gbs_tc_sign_image(p->h_hm, 1, 7, 128, img);     // H_128 itself
         else gbs_tc_sign_image(p->h_hm, p->m, p->k - 5 - uvm_glog, p->d_pad >> (5 + uvm_glog), img);
-        e = cudaMalloc(&p->d_aimg, 32768);
-        if (e == cudaSuccess) e = cudaMemcpy(p->d_aimg, img, 32768, cudaMemcpyHostToDevice);
+        e = cudaMalloc(&p->d_aimg, img_bytes);
+        if (e == cudaSuccess) e = cudaMemcpy(p->d_aimg, img, img_bytes, cudaMemcpyHostToDevice);
         free(img);
+        if (e == cudaSuccess && with_t) p->d_aimg_t = p->d_aimg + 32768;
         if (e != cudaSuccess) {
             cudaGetLastError();
             if (p->d_aimg) cudaFree(p->d_aimg);
@@ -260,7 +278,11 @@ extern "C" int gbs_dequantize(const gbs_plan_t* p, const void* codes, const floa
         return GBS_ERR_ALIGNMENT;
     DeviceGuard g;
     if (g.enter(p->device) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
-    int e = gbs_generic_dequantize(p, codes, scales, n_rows, out, out_dtype, (flags & GBS_INVERSE_ROTATE) != 0,
+    int e;
+    if ((flags & GBS_INVERSE_ROTATE) && gbs_tc_uvinv_supported(p))
+        e = gbs_tc_uvinv_dequantize(p, codes, scales, n_rows, out, out_dtype, static_cast<cudaStream_t>(cuda_stream));
+    else
+        e = gbs_generic_dequantize(p, codes, scales, n_rows, out, out_dtype, (flags & GBS_INVERSE_ROTATE) != 0,
                                    static_cast<cudaStream_t>(cuda_stream));
     return e == 0 ? GBS_OK : GBS_ERR_CUDA;
 }

@@ -35,6 +35,8 @@ struct gbs_plan {
     int asym;              // asymmetric quantizer (GBS_PLAN_ASYMMETRIC)
     int uvm_glog;          // UVM family: log2 of the number of 32-value chunks per tensor-core output row
     unsigned char* d_aimg; // device: pre-swizzled bf16 image of H_m (x) H_{2^j} for the tensor-core family (32 KB)
+    unsigned char* d_aimg_t; // device: image of its transpose (UV family, one scale per token: inverse rotation), or null
+    int a_colsum[128];     // column sums of H_m (x) H_{2^j} (UV family), for the inverse path's offset correction
     int* d_status;         // device status word: 0, or the code of the first bounded wait that expired
     int8_t h_hm[GBS_MAX_M * GBS_MAX_M];  // host copy of H_m
 };
@@ -54,13 +56,18 @@ int gbs_generic_dequantize(const gbs_plan* p, const void* codes, const float* sc
                            void* out, int out_dtype, int inverse, cudaStream_t stream);
 size_t gbs_generic_smem_bytes(const gbs_plan* p, int* rows_per_cta);
 
+// gbs_tc_uvinv.cu : gbs_dequantize with inverse rotation on the tensor cores
+bool gbs_tc_uvinv_supported(const gbs_plan* p);
+int gbs_tc_uvinv_dequantize(const gbs_plan* p, const void* codes, const float* scales, int64_t n_rows, void* out,
+                            int out_dtype, cudaStream_t stream);
+
 // gbs_tc_uv.cu
 bool gbs_tc_uv_supported(const gbs_plan* p);
 int gbs_tc_uv_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, const float* alphas, int K,
                          double* err_sum, float* err_rows, cudaStream_t stream);
 void gbs_tc_uv_a_image(const gbs_plan* p, unsigned char* img32k);
 // image of H_m (x) H_{2^j} (U x U inside 128 x 128, bf16 +-1, K-major, 128-byte swizzle)
-void gbs_tc_sign_image(const int8_t* hm, int m, int j, int U, unsigned char* img32k);
+void gbs_tc_sign_image(const int8_t* hm, int m, int j, int U, unsigned char* img32k, bool transpose = false);
 
 int gbs_tc_row_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, const float* alphas, int K,
                           double* err_sum, float* err_rows, cudaStream_t stream);

@@ -349,7 +349,8 @@ cudaError_t launch(KernelT kernel, int grid, int smem, cudaStream_t stream, bool
 // Shared-memory image of A = H_m (x) H_{2^j} as bf16 (+-1; zero outside U x U): two blocks of 64
 // k-columns, 128 rows of 128 bytes each, 16-byte chunks XOR-swizzled with the row index (the 128-byte
 // swizzle the MMA descriptor names).  Row = output index u', column = input index u (y = H x).
-void gbs_tc_sign_image(const int8_t* hm, int m, int j, int U, unsigned char* img)
+// transpose: the image of A^T instead (row = input index, column = output index: for x = H^T y).
+void gbs_tc_sign_image(const int8_t* hm, int m, int j, int U, unsigned char* img, bool transpose)
 {
     const int jm = (1 << j) - 1;
     unsigned short* h = reinterpret_cast<unsigned short*>(img);
@@ -360,7 +361,7 @@ void gbs_tc_sign_image(const int8_t* hm, int m, int j, int U, unsigned char* img
                     const int k = kb * 64 + c * 8 + e;
                     unsigned short v = 0;
                     if (r < U && k < U) {
-                        int sign = hm[(r >> j) * m + (k >> j)];
+                        int sign = transpose ? hm[(k >> j) * m + (r >> j)] : hm[(r >> j) * m + (k >> j)];
                         if (__builtin_popcount((unsigned)(r & k & jm)) & 1) sign = -sign;
                         v = sign < 0 ? 0xBF80 : 0x3F80;
                     }

@@ -559,3 +559,48 @@ def test_host_pipeline_equals_the_one_shot_call(rows, chunks):
                 continue
             c, s, _ = _run_rq(p, x.to(DEV), rows, want_y=False)
             assert torch.equal(ch, c.cpu()) and torch.equal(sh, s.cpu())
+
+
+INV_SHAPES = [
+    # d, d_pad, m, bits, rows
+    (4096, 4096, 1, 4, 4096 // 8 + 3),
+    (4096, 4096, 1, 3, 149),
+    (4000 // 32 * 32, 4096, 1, 4, 5),
+    (512, 512, 1, 3, 1),
+    (2560, 2560, 20, 4, 148 * 4 + 1),
+    (3584, 3584, 28, 3, 77),
+    (3456, 3456, 108, 4, 33),          # U = 108: the contraction is padded to 112
+    (1408, 1408, 44, 3, 9),
+]
+
+
+@pytest.mark.parametrize("d,d_pad,m,bits,rows", INV_SHAPES)
+def test_inverse_dequantize_on_the_tensor_cores(d, d_pad, m, bits, rows, monkeypatch):
+    """gbs_dequantize with GBS_INVERSE_ROTATE for per-token plans of the tensor-core family:
+    xhat = (H^T (q Delta) / sqrt(d'))[0:d] against the oracle, in fp32 and bf16, and against the generic kernel."""
+    rng = np.random.Generator(np.random.PCG64(d + m * 7 + bits + rows))
+    x = torch.from_numpy(rng.standard_t(3, size=(rows, d)).astype(np.float32)).to(torch.bfloat16)
+    with Plan(d, d_pad, m, bits, 0, 0.9) as plan:
+        assert plan.info.variant == 1
+        codes, scales, _ = _run_rq(plan, x.to(DEV), rows, want_y=False)
+        want = oracle.dequantize_rows(codes.cpu().numpy(), scales.cpu().double().numpy(), d, d_pad, m, bits, 0,
+                                      inverse=True)
+        for _ in range(2):                                     # twice: pipeline state does not leak between launches
+            got32 = plan.dequantize(codes, scales, inverse=True, dtype=torch.float32)
+        got16 = plan.dequantize(codes, scales, inverse=True, dtype=torch.bfloat16)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+    assert got32.shape == (rows, d) and got16.shape == (rows, d)
+    g = got32.cpu().double().numpy()
+    num = np.linalg.norm(g - want, axis=1)
+    den = np.linalg.norm(want, axis=1)
+    assert np.all(num <= 2e-7 * den + 1e-30), float((num / np.maximum(den, 1e-30)).max())   # exact rotation, one rounding
+    g16 = got16.cpu().double().numpy()
+    assert np.all(np.abs(g16 - want) <= 2.0 ** -8 * np.abs(want) + 1e-30)
+    monkeypatch.setenv("GBS_FORCE_GENERIC", "1")
+    with Plan(d, d_pad, m, bits, 0, 0.9) as gen:
+        assert gen.info.variant == 0
+        ref32 = gen.dequantize(codes, scales, inverse=True, dtype=torch.float32)
+        torch.cuda.synchronize()
+    num = np.linalg.norm(g - ref32.cpu().double().numpy(), axis=1)
+    assert np.all(num <= TOL_ROT_L2 * den + 1e-30)
