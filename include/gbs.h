@@ -192,8 +192,9 @@ int gbs_rotate_quantize_static(int d, int d_pad, int m, int bits, int group, flo
  *   out            device, n_rows * (d' or d) elements of out_dtype, rows contiguous,
  *                  16-byte aligned
  * The inverse rotation of plans with one symmetric scale per token in the tensor-core family
- * (bf16-shaped widths d' = 32 U, 16 <= U <= 128, d a multiple of 32) runs on the tensor cores: the
- * integer codes are rotated exactly and multiplied by Delta / sqrt(d') once at the end.
+ * (widths d' = 32 U, 16 <= U <= 128, d a multiple of 32), and of d' = 128 rows with one scale or
+ * (Delta, lo) pair per row, runs on the tensor cores: the integer codes are rotated exactly and
+ * multiplied by Delta / sqrt(d') once at the end.
  */
 int gbs_dequantize(const gbs_plan_t* plan, const void* codes, const float* scales, int64_t n_rows,
                    void* out, int out_dtype, int flags, void* cuda_stream);

@@ -281,6 +281,8 @@ extern "C" int gbs_dequantize(const gbs_plan_t* p, const void* codes, const floa
     int e;
     if ((flags & GBS_INVERSE_ROTATE) && gbs_tc_uvinv_supported(p))
         e = gbs_tc_uvinv_dequantize(p, codes, scales, n_rows, out, out_dtype, static_cast<cudaStream_t>(cuda_stream));
+    else if ((flags & GBS_INVERSE_ROTATE) && gbs_tc_rowinv_supported(p, scales))
+        e = gbs_tc_rowinv_dequantize(p, codes, scales, n_rows, out, out_dtype, static_cast<cudaStream_t>(cuda_stream));
     else
         e = gbs_generic_dequantize(p, codes, scales, n_rows, out, out_dtype, (flags & GBS_INVERSE_ROTATE) != 0,
                                    static_cast<cudaStream_t>(cuda_stream));

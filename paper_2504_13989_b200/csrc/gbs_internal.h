@@ -61,6 +61,11 @@ bool gbs_tc_uvinv_supported(const gbs_plan* p);
 int gbs_tc_uvinv_dequantize(const gbs_plan* p, const void* codes, const float* scales, int64_t n_rows, void* out,
                             int out_dtype, cudaStream_t stream);
 
+// gbs_tc_rowinv.cu : the same for d' = 128 rows with one scale (pair) per row
+bool gbs_tc_rowinv_supported(const gbs_plan* p, const float* scales);
+int gbs_tc_rowinv_dequantize(const gbs_plan* p, const void* codes, const float* scales, int64_t n_rows, void* out,
+                             int out_dtype, cudaStream_t stream);
+
 // gbs_tc_uv.cu
 bool gbs_tc_uv_supported(const gbs_plan* p);
 int gbs_tc_uv_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, const float* alphas, int K,

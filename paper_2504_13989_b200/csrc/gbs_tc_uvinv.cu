@@ -18,10 +18,9 @@
 #include <math.h>
 #include <string.h>
 
-#include <cuda_bf16.h>
-
 #include "gbs_internal.h"
 #include "gbs_tc_common.cuh"
+#include "gbs_tc_inv.cuh"
 
 namespace {
 
@@ -60,80 +59,6 @@ struct InvParams {
     int* status;
     float corr[UMAX];             // 32 * OFF * sum_u A[u][u']  (what the offset of the stored codes adds to coordinate 0)
 };
-
-// Eight offset codes, even ones in the bytes of y and odd ones in the bytes of z (each byte = q + 2^(b-1)),
-// -> four words of two bf16 numbers 128 + byte: [y.b0 z.b0] [y.b1 z.b1] [y.b2 z.b2] [y.b3 z.b3].
-__device__ __forceinline__ uint4 bytes_to_bf16x8(unsigned y, unsigned z)
-{
-    uint4 o;
-    o.x = (__byte_perm(y, z, 0x4400) & 0x00ff00ffu) | 0x43004300u;
-    o.y = (__byte_perm(y, z, 0x5511) & 0x00ff00ffu) | 0x43004300u;
-    o.z = (__byte_perm(y, z, 0x6622) & 0x00ff00ffu) | 0x43004300u;
-    o.w = (__byte_perm(y, z, 0x7733) & 0x00ff00ffu) | 0x43004300u;
-    return o;
-}
-
-// The 32 codes of one row segment (coordinates 32 u .. 32 u + 31 of a token) -> 32 bf16 numbers q + OFF,
-// as the four 16-byte chunks of the operand row.
-template <int BITS>
-__device__ __forceinline__ void unpack_row(const unsigned char* src, uint4 chunk[4])
-{
-    if (BITS == 4) {
-        const uint4 w = __ldg(reinterpret_cast<const uint4*>(src));
-        const unsigned ws[4] = {w.x, w.y, w.z, w.w};
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const unsigned x = ws[c] ^ 0x88888888u;                  // two's-complement nibble -> q + 8
-            chunk[c] = bytes_to_bf16x8(x & 0x0f0f0f0fu, (x >> 4) & 0x0f0f0f0fu);
-        }
-    } else {
-        const unsigned* s = reinterpret_cast<const unsigned*>(src);
-        const unsigned a0 = __ldg(s), a1 = __ldg(s + 1), a2 = __ldg(s + 2);
-        // 24 bits (eight 3-bit fields) per chunk
-        const unsigned g[4] = {a0 & 0xffffffu, ((a0 >> 24) | (a1 << 8)) & 0xffffffu, ((a1 >> 16) | (a2 << 16)) & 0xffffffu,
-                               a2 >> 8};
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const unsigned e = g[c], o = g[c] >> 3;                  // even fields at bits 6k, odd ones too after >> 3
-            unsigned y = (e & 0x7u) | ((e << 2) & 0x700u) | ((e << 4) & 0x70000u) | ((e << 6) & 0x7000000u);
-            unsigned z = (o & 0x7u) | ((o << 2) & 0x700u) | ((o << 4) & 0x70000u) | ((o << 6) & 0x7000000u);
-            chunk[c] = bytes_to_bf16x8(y ^ 0x04040404u, z ^ 0x04040404u);   // two's-complement field -> q + 4
-        }
-    }
-}
-
-__device__ __forceinline__ void st_shared_v4(unsigned addr, uint4 v)
-{
-    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-
-template <typename OutT>
-__device__ __forceinline__ void store_row32(OutT* dst, const unsigned r[32], float sc);
-template <>
-__device__ __forceinline__ void store_row32<float>(float* dst, const unsigned r[32], float sc)
-{
-    float4* o = reinterpret_cast<float4*>(dst);
-#pragma unroll
-    for (int i = 0; i < 8; ++i)
-        o[i] = make_float4(__uint_as_float(r[4 * i]) * sc, __uint_as_float(r[4 * i + 1]) * sc,
-                           __uint_as_float(r[4 * i + 2]) * sc, __uint_as_float(r[4 * i + 3]) * sc);
-}
-template <>
-__device__ __forceinline__ void store_row32<__nv_bfloat16>(__nv_bfloat16* dst, const unsigned r[32], float sc)
-{
-    uint4* o = reinterpret_cast<uint4*>(dst);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        unsigned w[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(r[8 * i + 2 * k]) * sc,
-                                                           __uint_as_float(r[8 * i + 2 * k + 1]) * sc);
-            w[k] = *reinterpret_cast<const unsigned*>(&h);
-        }
-        o[i] = make_uint4(w[0], w[1], w[2], w[3]);
-    }
-}
 
 // ---------------------------------------------------------------------------------------------
 // kernel
@@ -212,7 +137,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_inv(const __grid_constant_
             if (up < P.Upad) {
                 uint4 chunk[4];
                 if (up < P.U && row < P.n_rows) {
-                    unpack_row<BITS>(P.codes + row * P.code_row_bytes + up * (V * BITS / 8), chunk);
+                    unpack_row<BITS, false>(P.codes + row * P.code_row_bytes + up * (V * BITS / 8), chunk);
                 } else {
                     // rows that pad U to a multiple of 16 and tokens beyond the last: bf16 zeros (A^T has zero
                     // columns for the former, the latter are never stored)
@@ -250,7 +175,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_inv(const __grid_constant_
             r[0] = __float_as_uint(__uint_as_float(r[0]) - corr);      // the offset of the stored codes
             if (row < P.n_rows && up * V < P.d) {
                 const float sc = __ldg(P.scales + row) * P.norm;
-                store_row32<OutT>(reinterpret_cast<OutT*>(P.out) + row * (long long)P.d + up * V, r, sc);
+                store_row32<OutT>(reinterpret_cast<OutT*>(P.out) + row * (long long)P.d + up * V, r, sc, 0.f);
             }
         }
     }

@@ -604,3 +604,40 @@ def test_inverse_dequantize_on_the_tensor_cores(d, d_pad, m, bits, rows, monkeyp
         torch.cuda.synchronize()
     num = np.linalg.norm(g - ref32.cpu().double().numpy(), axis=1)
     assert np.all(num <= TOL_ROT_L2 * den + 1e-30)
+
+
+@pytest.mark.parametrize("d,bits,group,asym,rows", [
+    (128, 3, 0, False, 1), (128, 4, 128, False, 127), (128, 3, 0, False, 148 * 128 * 4 + 129),
+    (96, 4, 0, False, 300), (64, 3, 128, False, 129), (32, 4, 0, False, 77),
+    (128, 3, 128, True, 1000), (128, 4, 0, True, 129), (96, 3, 128, True, 515), (64, 4, 0, True, 5),
+])
+def test_inverse_dequantize_of_kv_rows_on_the_tensor_cores(d, bits, group, asym, rows):
+    """d' = 128 rows with one scale (pair) per row: xhat = (H_128 yhat / sqrt(128))[0:d] with
+    yhat = q Delta (Section 2.1) or code Delta + lo (Section 5.1), against the dense definition."""
+    rng = np.random.Generator(np.random.PCG64(d + bits * 3 + group + rows + int(asym)))
+    xs = rng.standard_t(3, size=(rows, d)) + (0.7 if asym else 0.0)
+    if rows > 4:
+        xs[3, :] = 0.0
+        xs[4, :] = 1.5                                    # constant row: after rotation one non-zero coordinate
+    x = torch.from_numpy(xs.astype(np.float32)).to(torch.bfloat16)
+    with Plan(d, 128, 1, bits, group, 0.9, asymmetric=asym) as plan:
+        assert plan.info.variant == 2
+        codes, scales, _ = plan.rotate_quantize(x.to(DEV))
+        for _ in range(2):
+            got32 = plan.dequantize(codes, scales, inverse=True, dtype=torch.float32)
+        got16 = plan.dequantize(codes, scales, inverse=True, dtype=torch.bfloat16)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+    sc = scales.cpu().double().numpy()
+    if asym:
+        sc = sc.reshape(rows, -1, 2)
+        yhat = oracle.dequantize_asym_rows(codes.cpu().numpy(), sc[:, :, 0], sc[:, :, 1], 128, bits, group)
+    else:
+        yhat = oracle.dequantize_rows(codes.cpu().numpy(), sc.reshape(rows, -1), 128, 128, 1, bits, group)
+    H = oracle.hadamard_full(1, 7).astype(np.float64)
+    want = (yhat @ H / np.sqrt(128.0))[:, :d]
+    g = got32.cpu().double().numpy()
+    assert g.shape == (rows, d)
+    scale_of_row = np.abs(yhat).max(axis=1, keepdims=True) * np.sqrt(128.0) + 1e-30
+    assert np.all(np.abs(g - want) <= 3e-7 * scale_of_row)
+    assert np.all(np.abs(got16.cpu().double().numpy() - want) <= 2.0 ** -8 * np.abs(want) + 3e-7 * scale_of_row)
