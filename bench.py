@@ -273,7 +273,7 @@ def main():
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-extras", action="store_true", help="skip the context legs under `also`")
     ap.add_argument("--profile", default=None, metavar="WORKLOAD[:ROWS]",
-                    help="launch one workload's kernel a few times and exit (for ncu captures), e.g. kv128:262144, "
+                    help="launch one workload's kernel a few times and exit (for ncu captures), e.g. kv128:262144, llama4096-inverse:4096, "
                          "clip:8192")
     args = ap.parse_args()
     if args.warmup < 3:
@@ -409,6 +409,9 @@ def run_profile(spec, device):
     from paper_2504_13989_b200 import Plan, synth
     name, _, rows = spec.partition(":")
     clip = name == "clip"
+    inverse = name.endswith("-inverse")               # e.g. llama4096-inverse: gbs_dequantize with inverse rotation
+    if inverse:
+        name = name[:-len("-inverse")]
     w = synth.WORKLOADS["calib4096" if clip else name]
     n = int(rows) if rows else min(w.n_rows, 8192)
     bits = w.bits[0]
@@ -416,11 +419,14 @@ def run_profile(spec, device):
     pl = Plan(w.d, w.d_pad, w.m, bits, w.group, w.alpha)
     outs = pl.alloc_outputs(n, device)
     err = torch.zeros(32, dtype=torch.float64, device=device)
+    xhat = torch.empty((n, w.d), dtype=torch.bfloat16, device=device) if inverse else None
     for _ in range(6):
         if clip:
             pl.clip_error(x, np.linspace(0.5, 1.0, 32), err_sum=err)
         else:
             pl.rotate_quantize(x, out=outs)
+            if inverse:
+                pl.dequantize(outs[0], outs[1], inverse=True, out=xhat)
     torch.cuda.synchronize()
     print(json.dumps({"profile": spec, "rows": n, "kernel_family": pl.info.variant, "status": pl.device_status()}))
 
