@@ -641,3 +641,57 @@ def test_inverse_dequantize_of_kv_rows_on_the_tensor_cores(d, bits, group, asym,
     scale_of_row = np.abs(yhat).max(axis=1, keepdims=True) * np.sqrt(128.0) + 1e-30
     assert np.all(np.abs(g - want) <= 3e-7 * scale_of_row)
     assert np.all(np.abs(got16.cpu().double().numpy() - want) <= 2.0 ** -8 * np.abs(want) + 3e-7 * scale_of_row)
+
+
+def _random_plans(n_cases: int, seed: int):
+    """Seeded draw of valid (d, d', m, bits, group, alpha, rows, dtype) over every order and kernel family."""
+    rng = np.random.Generator(np.random.PCG64(seed))
+    orders = [1, 1, 1, 12, 20, 24, 28, 44, 48, 60, 68, 72, 80, 84, 104, 108]
+    cases = []
+    while len(cases) < n_cases:
+        m = int(rng.choice(orders))
+        k = int(rng.integers(3, 14))
+        d_pad = m << k
+        if d_pad > 32768:
+            continue
+        bits = int(rng.choice([3, 4]))
+        if rng.random() < 0.5:
+            group = 0
+        else:
+            group = 1 << int(rng.integers(3, k + 1))
+        # widths: full, a multiple of 32 below d', or an arbitrary multiple of 8
+        r = rng.random()
+        if r < 0.4:
+            d = d_pad
+        elif r < 0.7 and d_pad >= 64:
+            d = int(rng.integers(1, d_pad // 32 + 1)) * 32
+        else:
+            d = int(rng.integers(1, d_pad // 8 + 1)) * 8
+        rows = int(rng.choice([1, 3, 4, 5, 33, 130, 149, 600])) if d_pad <= 8192 else int(rng.choice([1, 2, 5, 9]))
+        dtype = torch.bfloat16 if rng.random() < 0.75 else torch.float32
+        alpha = float(rng.choice([1.0, 0.9, 0.75, 0.5]))
+        cases.append((d, d_pad, m, bits, group, alpha, rows, dtype))
+    return cases
+
+
+@pytest.mark.parametrize("d,d_pad,m,bits,group,alpha,rows,dtype", _random_plans(60, 20250413))
+def test_random_plans_against_the_oracle(d, d_pad, m, bits, group, alpha, rows, dtype):
+    """Whatever family the plan picks: rotated values, scales and codes against the oracle, then the inverse
+    dequantize of the kernel's own codes."""
+    rng = np.random.Generator(np.random.PCG64(d * 31 + d_pad + m + bits + group + rows))
+    xs = rng.standard_t(3, size=(rows, d))
+    xs[:, rng.integers(0, d, 2)] *= 25
+    x = torch.from_numpy(xs.astype(np.float32)).to(dtype)
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(x), d, d_pad, m, bits, group, alpha, dense=(d_pad <= 1024))
+    with Plan(d, d_pad, m, bits, group, alpha) as plan:
+        codes, scales, y = _run_rq(plan, x.to(DEV), rows)
+        assert plan.device_status() == 0
+        compare_rotate_quantize(x, ref, codes, scales, y, bits, group, d_pad)
+        xhat = plan.dequantize(codes, scales, inverse=True)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+    wantx = oracle.dequantize_rows(codes.cpu().numpy(), scales.cpu().double().numpy(), d, d_pad, m, bits, group,
+                                   inverse=True)
+    num = np.linalg.norm(xhat.cpu().double().numpy() - wantx, axis=1)
+    den = np.linalg.norm(wantx, axis=1)
+    assert np.all(num <= TOL_ROT_L2 * den + 1e-30)
