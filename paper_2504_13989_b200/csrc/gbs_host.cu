@@ -318,6 +318,9 @@ extern "C" int gbs_clip_error(const gbs_plan_t* p, const void* x, int x_dtype, i
     else if (p->variant == GBS_VARIANT_TC_ROW && x_dtype == GBS_DTYPE_BF16)
         e = gbs_tc_row_clip_error(p, x, n_rows, x_row_stride, alphas_host, K, err_sum, err_rows_opt,
                                   static_cast<cudaStream_t>(cuda_stream));
+    else if (p->variant == GBS_VARIANT_TC_UVM && x_dtype == GBS_DTYPE_BF16)
+        e = gbs_tc_uvm_clip_error(p, x, n_rows, x_row_stride, alphas_host, K, err_sum, err_rows_opt,
+                                  static_cast<cudaStream_t>(cuda_stream));
     else
         e = gbs_generic_clip_error(p, x, x_dtype, n_rows, x_row_stride, c_scale, c_inv, K, err_sum, err_rows_opt,
                                    static_cast<cudaStream_t>(cuda_stream));

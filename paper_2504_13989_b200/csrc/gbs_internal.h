@@ -81,6 +81,8 @@ int gbs_tc_row_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int6
 int gbs_tc_uvm_glog(const gbs_plan* p);        // 0 if the family does not apply
 int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
                                float* scales, float* y_opt, cudaStream_t stream);
+int gbs_tc_uvm_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, const float* alphas, int K,
+                          double* err_sum, float* err_rows, cudaStream_t stream);
 
 // gbs_tc_row.cu
 bool gbs_tc_row_supported(const gbs_plan* p);

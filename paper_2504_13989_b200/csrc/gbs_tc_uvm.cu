@@ -45,6 +45,9 @@ struct __align__(1024) Smem {
     // GROUPED: [group][warp half w][lane u'][chunk]: max|.| of the chunk's scale group over the columns warp w
     // swept.  Written between a token's two barriers and read after the second, so one copy is enough.
     __align__(16) float gm[2][2][UMAX][8];
+    // CLIP: [group][warp of the group][candidate]: a warp's error sums over its lanes and chunks of the token.
+    // Written in sweep 3 and read after the third barrier; the next token's writes come two barriers later.
+    float cpart[2][8][GBS_MAX_CANDIDATES];
     unsigned tmem_base;
     volatile int abort_flag;
 };
@@ -66,6 +69,14 @@ struct UvmParams {
     float* scales;
     float* y_opt;
     int* status;
+    // clip-ratio scoring (the CLIP instantiations only)
+    int K;                        // candidates
+    int levels;                   // D
+    float norm2;                  // 1 / d'
+    float clip_half[GBS_MAX_CANDIDATES];    // 1 / (2 alpha_k), zero beyond K
+    float clip_scale[GBS_MAX_CANDIDATES];   // alpha_k / D,     zero beyond K
+    double* err_sum;
+    float* err_rows;
 };
 
 __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, void* bar, int c0, int c1, int c2, int c3)
@@ -150,7 +161,11 @@ __device__ __forceinline__ void tmem_ld_wait_n<32>(unsigned* r)
 // ---------------------------------------------------------------------------------------------
 // kernel
 // ---------------------------------------------------------------------------------------------
-template <int BITS, int GLOG, bool GROUPED>
+// CLIP = true: instead of quantizing, sweep 3 scores K clip ratios (Sections 2.1, 3.1) as the UV family does:
+// per value and candidate clamp (fma.sat), round half-even (magic add), residual, square-accumulate, eight
+// candidates at a time over the warp's chunks; warp sums go to shared memory, a third named barrier, and the
+// first warp of the group adds the eight parts in a fixed order (per-row output, fp64 running totals).
+template <int BITS, int GLOG, bool GROUPED, bool CLIP>
 __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant__ CUtensorMap tmap,
                                                           const __grid_constant__ UvmParams P)
 {
@@ -242,6 +257,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
         const bool quad_live = q * 32 < P.U;      // a quadrant wholly beyond U has nothing to do
         const bool lane_live = up < P.U;
         const unsigned tq = tmem_base + ((unsigned)(q * 32) << 16);
+        double dacc0 = 0.0, dacc1 = 0.0;          // CLIP, first warp of a group: totals of candidates lane, lane + 32
         int it = grp, n = 0;
         for (long long row = (long long)blockIdx.x + (long long)grp * gridDim.x; row < P.n_rows;
              row += 2ll * gridDim.x, it += 2, ++n) {
@@ -350,6 +366,63 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
                 const float4 m0 = rp[0], m1 = rp[1];
                 M = fmaxf(fmaxf(fmaxf(m0.x, m0.y), fmaxf(m0.z, m0.w)), fmaxf(fmaxf(m1.x, m1.y), fmaxf(m1.z, m1.w)));
             }
+            if constexpr (CLIP) {
+                float* part = &S->cpart[grp][ew][0];
+                if (quad_live) {
+                    tc_fence_after();
+                    const float twoD = (float)(2 * P.levels);
+                    const float MAGIC = 8388608.f;             // 2^23: w * 2D + MAGIC has rint(w * 2D) in its low bits
+                    const float mD = MAGIC + (float)P.levels;
+                    for (int k0 = 0; k0 < P.K; k0 += 8) {
+                        float acc[8];
+#pragma unroll
+                        for (int kk = 0; kk < 8; ++kk) acc[kk] = 0.f;
+#pragma unroll
+                        for (int i = 0; i < G / 2; ++i) {
+                            tmem_ld32_issue(tcol + (2 * i + w) * V, r);
+                            tmem_ld_wait(r);
+                            const float mg = GROUPED ? Ms[i] : M;
+                            const float rM = (mg > 0.f) ? (1.f / mg) : 0.f;
+                            float a1k[8], dl[8];
+#pragma unroll
+                            for (int kk = 0; kk < 8; ++kk) {
+                                a1k[kk] = P.clip_half[k0 + kk] * rM;
+                                dl[kk] = -P.clip_scale[k0 + kk] * mg;          // -Delta_k
+                            }
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) {
+                                const float y = __uint_as_float(r[e]);
+#pragma unroll
+                                for (int kk = 0; kk < 8; ++kk) {
+                                    const float wv = __saturatef(fmaf(y, a1k[kk], 0.5f));
+                                    const float qv = fmaf(wv, twoD, MAGIC) - mD;    // the code, as a float
+                                    const float err = fmaf(qv, dl[kk], y);
+                                    acc[kk] = fmaf(err, err, acc[kk]);
+                                }
+                            }
+                        }
+                        const float h1 = warp_fold8(acc, lane);
+                        const int kk = ((lane >> 4) & 1) * 4 + ((lane >> 3) & 1) * 2 + ((lane >> 2) & 1);
+                        if ((lane & 3) == 0 && k0 + kk < P.K) part[k0 + kk] = h1;
+                    }
+                    tc_fence_before();
+                } else {
+                    for (int k = lane; k < P.K; k += 32) part[k] = 0.f;
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&S->tempty[ts]);
+                asm volatile("bar.sync %0, 256;" ::"r"(1 + grp) : "memory");
+                if (ew == 0) {
+                    for (int k = lane; k < P.K; k += 32) {
+                        float rk = 0.f;
+#pragma unroll
+                        for (int e8 = 0; e8 < 8; ++e8) rk += S->cpart[grp][e8][k];
+                        if (P.err_rows) P.err_rows[row * P.K + k] = rk * P.norm2;
+                        if (k < 32) dacc0 += (double)rk; else dacc1 += (double)rk;
+                    }
+                }
+                continue;
+            }
             // sweep 3: Delta, round / clip, pack, store
             float a1 = (M > 0.f) ? __fdividef(P.c_half, M) : 0.f;
             if (quad_live) {
@@ -392,6 +465,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
             // the accumulators have been read for the last time: hand the TMEM stage back to the MMA issuer
             __syncwarp();
             if (lane == 0) mbar_arrive(&S->tempty[ts]);
+        }
+        if (CLIP && ew == 0) {
+            if (lane < P.K) atomicAdd(&P.err_sum[lane], dacc0 * (double)P.norm2);
+            if (lane + 32 < P.K) atomicAdd(&P.err_sum[lane + 32], dacc1 * (double)P.norm2);
         }
     }
 
@@ -447,8 +524,10 @@ int gbs_tc_uvm_glog(const gbs_plan* p)
     return 0;
 }
 
-int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
-                               float* scales, float* y_opt, cudaStream_t stream)
+namespace {
+
+// Tensor map of the rows and the parameters common to both uses of the kernel.
+int uvm_prepare(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, CUtensorMap* tmap_out, UvmParams* P_out)
 {
     EncodeTiledFn encode = get_encode();
     if (!encode) return (int)cudaErrorNotSupported;
@@ -456,7 +535,7 @@ int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
     const int glog = p->uvm_glog, G = 1 << glog;
     const int U = p->d_pad / (V * G);
     // dims: v (32 values), chunk c (G), u, token; one box = chunk c of one token: U rows of 32 values
-    CUtensorMap tmap;
+    CUtensorMap& tmap = *tmap_out;
     const cuuint64_t gdim[4] = {(cuuint64_t)V, (cuuint64_t)G, (cuuint64_t)(p->d / (V * G)), (cuuint64_t)n_rows};
     const cuuint64_t gstr[3] = {(cuuint64_t)(V * 2), (cuuint64_t)(V * G * 2), (cuuint64_t)(stride * 2)};
     const int Upad = (U + 15) & ~15;       // the contraction is padded to the MMA's K = 16; TMA zero-fills the rows
@@ -467,7 +546,7 @@ int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return (int)cudaErrorInvalidValue;
 
-    UvmParams P;
+    UvmParams& P = *P_out;
     memset(&P, 0, sizeof(P));
     P.n_rows = n_rows;
     P.U = U;
@@ -485,17 +564,32 @@ int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
     P.c_half = (float)(1.0 / (2.0 * (double)p->alpha));
     P.norm = p->norm;
     P.a_img = p->d_aimg;
+    P.status = p->d_status;
+    P.levels = p->levels;
+    P.norm2 = (float)(1.0 / (double)p->d_pad);
+    return 0;
+}
+
+}  // namespace
+
+int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
+                               float* scales, float* y_opt, cudaStream_t stream)
+{
+    CUtensorMap tmap;
+    UvmParams P;
+    const int rc = uvm_prepare(p, x, n_rows, stride, &tmap, &P);
+    if (rc != 0) return rc;
+    const int glog = p->uvm_glog;
     P.codes = (unsigned char*)codes;
     P.scales = scales;
     P.y_opt = y_opt;
-    P.status = p->d_status;
     const int smem = (int)sizeof(Smem) + 1024;
     const int grid = (int)(n_rows < p->sm_count ? n_rows : p->sm_count);
     const bool pdl = p->pdl != 0;
     cudaError_t e;
 #define GBS_UVM_LAUNCH(B, GL)                                                                   \
-    (p->group ? launch(k_tc_uvm_rq<B, GL, true>, grid, smem, stream, pdl, tmap, P)               \
-              : launch(k_tc_uvm_rq<B, GL, false>, grid, smem, stream, pdl, tmap, P))
+    (p->group ? launch(k_tc_uvm_rq<B, GL, true, false>, grid, smem, stream, pdl, tmap, P)        \
+              : launch(k_tc_uvm_rq<B, GL, false, false>, grid, smem, stream, pdl, tmap, P))
     if (p->bits == 3) {
         if (glog == 1) e = GBS_UVM_LAUNCH(3, 1);
         else if (glog == 2) e = GBS_UVM_LAUNCH(3, 2);
@@ -506,5 +600,35 @@ int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
         else e = GBS_UVM_LAUNCH(4, 3);
     }
 #undef GBS_UVM_LAUNCH
+    return (int)e;
+}
+
+// Clip-ratio scoring on the same front end (sweeps 1 and 2), with sweep 3 scoring instead of packing.
+int gbs_tc_uvm_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, const float* alphas, int K,
+                          double* err_sum, float* err_rows, cudaStream_t stream)
+{
+    CUtensorMap tmap;
+    UvmParams P;
+    const int rc = uvm_prepare(p, x, n_rows, stride, &tmap, &P);
+    if (rc != 0) return rc;
+    P.K = K;
+    for (int i = 0; i < K; ++i) {
+        P.clip_half[i] = (float)(1.0 / (2.0 * (double)alphas[i]));
+        P.clip_scale[i] = (float)((double)alphas[i] / (double)p->levels);
+    }
+    P.err_sum = err_sum;
+    P.err_rows = err_rows;
+    const int glog = p->uvm_glog;
+    const int smem = (int)sizeof(Smem) + 1024;
+    const int grid = (int)(n_rows < p->sm_count ? n_rows : p->sm_count);
+    const bool pdl = p->pdl != 0;
+    cudaError_t e;
+#define GBS_UVM_CLIP(GL)                                                                        \
+    (p->group ? launch(k_tc_uvm_rq<4, GL, true, true>, grid, smem, stream, pdl, tmap, P)         \
+              : launch(k_tc_uvm_rq<4, GL, false, true>, grid, smem, stream, pdl, tmap, P))
+    if (glog == 1) e = GBS_UVM_CLIP(1);
+    else if (glog == 2) e = GBS_UVM_CLIP(2);
+    else e = GBS_UVM_CLIP(3);
+#undef GBS_UVM_CLIP
     return (int)e;
 }

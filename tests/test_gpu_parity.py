@@ -306,6 +306,18 @@ def test_wide_family_shapes(d, d_pad, m, bits, alpha, rows, group):
             assert int(codes[2].max()) == 0 and float(scales[2].abs().max()) == 0.0
         codes2, scales2, _ = _run_rq(plan, x.to(DEV), rows, want_y=False)
         assert torch.equal(codes, codes2) and torch.equal(scales, scales2)
+        # clip-ratio scoring on the same front end (a third sweep that scores instead of packing)
+        K = (3, 8, 11, 33, 64)[(d + bits + group + rows) % 5]
+        alphas = np.linspace(0.3, 1.0, K)
+        nc = min(rows, 40)
+        xc = x[:nc].contiguous()
+        for _ in range(2):
+            err, erows = plan.clip_error(xc.to(DEV), alphas, want_rows=True)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+        eref, rref = oracle.clip_error_rows(synth.to_oracle_array(xc), d, d_pad, m, bits, group, alphas, want_rows=True)
+        np.testing.assert_allclose(err.cpu().numpy(), eref, rtol=TOL_CLIP)
+        np.testing.assert_allclose(erows.cpu().double().numpy(), rref, rtol=1e-4, atol=1e-12)
 
 
 ROW_SHAPES = [
