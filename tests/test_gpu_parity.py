@@ -707,3 +707,40 @@ def test_random_plans_against_the_oracle(d, d_pad, m, bits, group, alpha, rows, 
     num = np.linalg.norm(xhat.cpu().double().numpy() - wantx, axis=1)
     den = np.linalg.norm(wantx, axis=1)
     assert np.all(num <= TOL_ROT_L2 * den + 1e-30)
+
+
+@pytest.mark.parametrize("d,d_pad,m,rows", [(4096, 4096, 1, 4096), (128, 128, 1, 70000), (2560, 2560, 20, 601)])
+def test_producer_consumer_chain_without_host_synchronisation(d, d_pad, m, rows):
+    """quantize -> dequantize with inverse rotation -> quantize the result -> ... on one stream, each kernel
+    reading what the kernel before it is still writing when it becomes resident (programmatic dependent
+    launch; the quantizer also prefetches its first tile into L2 before its dependency wait).  The chain must
+    give bit-identical results with and without a host synchronisation between the calls."""
+    rng = np.random.Generator(np.random.PCG64(d + rows))
+    x0 = torch.from_numpy(rng.standard_t(3, size=(rows, d)).astype(np.float32)).to(torch.bfloat16).to(DEV)
+    with Plan(d, d_pad, m, 4, 0, 0.9) as plan:
+        def chain(sync: bool):
+            xa = x0.clone()
+            xb = torch.empty_like(xa)
+            outs = [plan.alloc_outputs(rows, DEV) for _ in range(2)]
+            torch.cuda.synchronize()
+            trace = []
+            for i in range(12):
+                o = outs[i & 1]
+                plan.rotate_quantize(xa, out=o)
+                if sync:
+                    torch.cuda.synchronize()
+                plan.dequantize(o[0], o[1], inverse=True, dtype=torch.bfloat16, out=xb)
+                if sync:
+                    torch.cuda.synchronize()
+                xa, xb = xb, xa
+                if i in (0, 5, 11):
+                    trace.append((o[0].clone(), o[1].clone()))
+            torch.cuda.synchronize()
+            return trace, xa.clone()
+        t_sync, x_sync = chain(True)
+        for _ in range(3):
+            t_free, x_free = chain(False)
+            assert torch.equal(x_sync, x_free)
+            for (c1, s1), (c2, s2) in zip(t_sync, t_free):
+                assert torch.equal(c1, c2) and torch.equal(s1, s2)
+        assert plan.device_status() == 0
