@@ -744,3 +744,40 @@ def test_producer_consumer_chain_without_host_synchronisation(d, d_pad, m, rows)
             for (c1, s1), (c2, s2) in zip(t_sync, t_free):
                 assert torch.equal(c1, c2) and torch.equal(s1, s2)
         assert plan.device_status() == 0
+
+
+def test_one_plan_from_several_streams_and_host_threads():
+    """A plan is immutable: launches from different streams and host threads at once give the same bytes."""
+    import threading
+    d, rows = 4096, 1500
+    rng = np.random.Generator(np.random.PCG64(99))
+    xs = [torch.from_numpy(rng.standard_t(3, size=(rows, d)).astype(np.float32)).to(torch.bfloat16).to(DEV)
+          for _ in range(4)]
+    with Plan(d, d, 1, 3, 0, 0.9) as plan:
+        refs = [plan.rotate_quantize(x) for x in xs]
+        torch.cuda.synchronize()
+        results = [None] * 4
+        errors = []
+
+        def worker(i):
+            try:
+                st = torch.cuda.Stream(device=DEV)
+                out = None
+                with torch.cuda.stream(st):           # allocations of this thread belong to its stream
+                    for _ in range(25):
+                        out = plan.rotate_quantize(xs[i], stream=st)
+                        plan.clip_error(xs[i], [0.8, 1.0], stream=st)
+                st.synchronize()
+                results[i] = out
+            except Exception as exc:      # surfaced below: an assertion in a thread would be lost
+                errors.append(exc)
+        threads = [threading.Thread(target=worker, args=(i,)) for i in range(4)]
+        for t in threads:
+            t.start()
+        for t in threads:
+            t.join()
+        assert not errors, errors
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+        for (c, s, _), (cr, sr, _) in zip(results, refs):
+            assert torch.equal(c, cr) and torch.equal(s, sr)
