@@ -88,6 +88,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_row_inv(const __grid_constant
         if (lane == 0) {
             constexpr unsigned IDESC = instr_desc(TILE, DP, false);
             const unsigned h_base = smem_u32(S->h);
+            const unsigned long long xd0 = smem_desc(smem_u32(S->x[0]), 16, 1024, 2);
+            const unsigned long long hd0 = smem_desc(h_base, 16, 1024, 2);
+            const unsigned xd_lo0 = (unsigned)xd0, xd_hi = (unsigned)(xd0 >> 32);
+            const unsigned hd_lo0 = (unsigned)hd0, hd_hi = (unsigned)(hd0 >> 32);
             bool ok = mbar_wait(&S->abort_flag, &S->hbar, 0, P.status, 6);
             int it = 0;
             for (long long t = blockIdx.x; ok && t < P.n_tiles; t += gridDim.x, ++it) {
@@ -96,12 +100,17 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_row_inv(const __grid_constant
                 if (!mbar_wait(&S->abort_flag, &S->full[s], ph, P.status, 2)) break;
                 if (!mbar_wait(&S->abort_flag, &S->tempty[s], ph ^ 1, P.status, 3)) break;
                 tc_fence_after();
-                const unsigned x_base = smem_u32(S->x[s]);
-                for (int ks = 0; ks < DP / 16; ++ks) {
-                    const unsigned off = (ks >> 2) * (TILE * 128) + (ks & 3) * 32;
-                    const unsigned long long ad = smem_desc(x_base + off, 16, 1024, 2);
-                    const unsigned long long bd = smem_desc(h_base + off, 16, 1024, 2);
-                    umma_f16(tmem_base + s * DP, ad, bd, IDESC, ks > 0 ? 1u : 0u);
+                // only the address fields (bytes >> 4, low words) of the two K-major descriptors change between
+                // k-steps: 32 bytes inside the 128-byte swizzled row, the second K block TILE*128 bytes further
+                unsigned x_lo = xd_lo0 + (unsigned)s * (TILE_BYTES >> 4), h_lo = hd_lo0;
+                const unsigned d_tmem = tmem_base + s * DP;
+                umma_f16_words<false>(d_tmem, x_lo, xd_hi, h_lo, hd_hi, IDESC);
+#pragma unroll
+                for (int ks = 1; ks < DP / 16; ++ks) {
+                    const unsigned step = (ks & 3) ? 2u : (unsigned)((TILE * 128 - 96) >> 4);
+                    x_lo += step;
+                    h_lo += step;
+                    umma_f16_words<true>(d_tmem, x_lo, xd_hi, h_lo, hd_hi, IDESC);
                 }
                 umma_commit(&S->empty[s]);
                 umma_commit(&S->tfull[s]);

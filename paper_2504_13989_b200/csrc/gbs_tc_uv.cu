@@ -193,6 +193,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
             constexpr unsigned IDESC = instr_desc(UMAX, STAGE_COLS);
             const unsigned a_base = smem_u32(S->a);
             const unsigned tok_bytes = (unsigned)(P.Upad * V * 2);
+            const unsigned long long ad0 = smem_desc(a_base, 16, 1024, 2);
+            const unsigned long long bd0 = smem_desc(smem_u32(S->b[0]), tok_bytes, 512, 4);
+            const unsigned ad_lo0 = (unsigned)ad0, ad_hi = (unsigned)(ad0 >> 32);
+            const unsigned bd_lo0 = (unsigned)bd0, bd_hi = (unsigned)(bd0 >> 32);
             bool ok = mbar_wait(&S->abort_flag, &S->abar, 0, P.status, 6);
             int it = 0;
             for (int g = blockIdx.x; ok && g < P.n_groups; g += gridDim.x, ++it) {
@@ -201,13 +205,17 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
                 if (!mbar_wait(&S->abort_flag, &S->full[s], ph, P.status, 2)) break;
                 if (!mbar_wait(&S->abort_flag, &S->tempty[s], ph ^ 1, P.status, 3)) break;
                 tc_fence_after();
-                const unsigned b_base = smem_u32(S->b[s]);
-                for (int ks = 0; ks < P.ksteps; ++ks) {
-                    // A: k-step ks = 32 bytes inside the 128-byte swizzled row of block ks/4; 8-row groups 1024 B apart
-                    const unsigned long long ad = smem_desc(a_base + (ks >> 2) * (UMAX * 128) + (ks & 3) * 32, 16, 1024, 2);
-                    // B: 16 u-rows of 64 bytes per k-step; 8-row groups 512 B apart; next token (N atom) U*64 B away
-                    const unsigned long long bd = smem_desc(b_base + ks * 1024, tok_bytes, 512, 4);
-                    umma_f16(tmem_base + s * STAGE_COLS, ad, bd, IDESC, ks > 0 ? 1u : 0u);
+                // A: k-step ks = 32 bytes inside the 128-byte swizzled row of block ks/4 (blocks UMAX*128 B apart);
+                // 8-row groups 1024 B apart.  B: 16 u-rows of 64 bytes per k-step (1024 B); 8-row groups 512 B
+                // apart; next token (N atom) Upad*64 B away.  Only the address fields (bytes >> 4, in the low
+                // words) change from one k-step to the next.
+                unsigned a_lo = ad_lo0, b_lo = bd_lo0 + (unsigned)s * (STAGE_BYTES_MAX >> 4);
+                const unsigned d_tmem = tmem_base + s * STAGE_COLS;
+                umma_f16_words<false>(d_tmem, a_lo, ad_hi, b_lo, bd_hi, IDESC);
+                for (int ks = 1; ks < P.ksteps; ++ks) {
+                    a_lo += (ks & 3) ? 2u : (unsigned)((UMAX * 128 - 96) >> 4);
+                    b_lo += 1024u >> 4;
+                    umma_f16_words<true>(d_tmem, a_lo, ad_hi, b_lo, bd_hi, IDESC);
                 }
                 umma_commit(&S->empty[s]);
                 umma_commit(&S->tfull[s]);

@@ -99,6 +99,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_inv(const __grid_constant_
         if (lane == 0) {
             constexpr unsigned IDESC = instr_desc(UMAX, STAGE_COLS);
             const unsigned a_base = smem_u32(S->a);
+            const unsigned long long ad0 = smem_desc(a_base, 16, 1024, 2);
+            const unsigned long long bd0 = smem_desc(smem_u32(S->b[0]), tok_bytes, 512, 4);
+            const unsigned ad_lo0 = (unsigned)ad0, ad_hi = (unsigned)(ad0 >> 32);
+            const unsigned bd_lo0 = (unsigned)bd0, bd_hi = (unsigned)(bd0 >> 32);
             bool ok = mbar_wait(&S->abort_flag, &S->abar, 0, P.status, 6);
             int it = 0;
             for (int g = blockIdx.x; ok && g < P.n_groups; g += gridDim.x, ++it) {
@@ -107,11 +111,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_inv(const __grid_constant_
                 if (!mbar_wait(&S->abort_flag, &S->full[s], ph, P.status, 2)) break;
                 if (!mbar_wait(&S->abort_flag, &S->tempty[s], ph ^ 1, P.status, 3)) break;
                 tc_fence_after();
-                const unsigned b_base = smem_u32(S->b[s]);
-                for (int ks = 0; ks < P.ksteps; ++ks) {
-                    const unsigned long long ad = smem_desc(a_base + (ks >> 2) * (UMAX * 128) + (ks & 3) * 32, 16, 1024, 2);
-                    const unsigned long long bd = smem_desc(b_base + ks * 1024, tok_bytes, 512, 4);
-                    umma_f16(tmem_base + s * STAGE_COLS, ad, bd, IDESC, ks > 0 ? 1u : 0u);
+                // only the address fields (bytes >> 4, low words) of the descriptors change between k-steps
+                unsigned a_lo = ad_lo0, b_lo = bd_lo0 + (unsigned)s * (B_STAGE_BYTES >> 4);
+                const unsigned d_tmem = tmem_base + s * STAGE_COLS;
+                umma_f16_words<false>(d_tmem, a_lo, ad_hi, b_lo, bd_hi, IDESC);
+                for (int ks = 1; ks < P.ksteps; ++ks) {
+                    a_lo += (ks & 3) ? 2u : (unsigned)((UMAX * 128 - 96) >> 4);
+                    b_lo += 1024u >> 4;
+                    umma_f16_words<true>(d_tmem, a_lo, ad_hi, b_lo, bd_hi, IDESC);
                 }
                 umma_commit(&S->empty[s]);
                 umma_commit(&S->tfull[s]);

@@ -230,6 +230,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
             constexpr unsigned IDESC = instr_desc(UMAX, NCOLS);
             const unsigned a_base = smem_u32(S->a);
             const unsigned chunk_bytes = (unsigned)(P.Upad * V * 2);  // one chunk (N atom of 32): Upad rows of 64 bytes
+            const unsigned long long ad0 = smem_desc(a_base, 16, 1024, 2);
+            const unsigned long long bd0 = smem_desc(smem_u32(S->b), chunk_bytes, 512, 4);
+            const unsigned ad_lo0 = (unsigned)ad0, ad_hi = (unsigned)(ad0 >> 32);
+            const unsigned bd_lo0 = (unsigned)bd0, bd_hi = (unsigned)(bd0 >> 32);
             bool ok = mbar_wait(&S->abort_flag, &S->abar, 0, P.status, 6);
             int it = 0;
             for (int tk = blockIdx.x; ok && tk < n_tok; tk += gridDim.x, ++it) {
@@ -237,11 +241,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
                 if (!mbar_wait(&S->abort_flag, &S->full[s], (it / nst) & 1, P.status, 2)) break;
                 if (!mbar_wait(&S->abort_flag, &S->tempty[ts], ((it / TSTAGES) & 1) ^ 1, P.status, 3)) break;
                 tc_fence_after();
-                const unsigned b_base = smem_u32(S->b + (size_t)s * P.stage_bytes);
-                for (int ks = 0; ks < P.ksteps; ++ks) {
-                    const unsigned long long ad = smem_desc(a_base + (ks >> 2) * (UMAX * 128) + (ks & 3) * 32, 16, 1024, 2);
-                    const unsigned long long bd = smem_desc(b_base + ks * 1024, chunk_bytes, 512, 4);
-                    umma_f16(tmem_base + ts * NCOLS, ad, bd, IDESC, ks > 0 ? 1u : 0u);
+                // only the address fields (bytes >> 4, low words) of the descriptors change between k-steps
+                unsigned a_lo = ad_lo0, b_lo = bd_lo0 + (unsigned)s * ((unsigned)P.stage_bytes >> 4);
+                const unsigned d_tmem = tmem_base + ts * NCOLS;
+                umma_f16_words<false>(d_tmem, a_lo, ad_hi, b_lo, bd_hi, IDESC);
+                for (int ks = 1; ks < P.ksteps; ++ks) {
+                    a_lo += (ks & 3) ? 2u : (unsigned)((UMAX * 128 - 96) >> 4);
+                    b_lo += 1024u >> 4;
+                    umma_f16_words<true>(d_tmem, a_lo, ad_hi, b_lo, bd_hi, IDESC);
                 }
                 umma_commit(&S->empty[s]);
                 umma_commit(&S->tfull[ts]);
