@@ -19,7 +19,8 @@
 //     coordinates (g <= 32 lanes) = warp shuffle only.  Delta, rounding, clipping (Section 3.1) and
 //     the 3/4-bit packing follow from registers; each thread stores 12 or 16 contiguous bytes.
 //
-// One persistent CTA per SM.  Warp 0 = TMA producer, warp 1 = MMA issuer / TMEM owner, warps 2..17 =
+// One persistent CTA per SM.  Warp 0 = TMA producer, warp 1 = MMA issuer / TMEM owner (warp 18 issues the
+// MMAs of every other tile), warps 2..17 =
 // epilogue: warp (q, t) serves TMEM lane quadrant q and token t of EVERY stage, so all sixteen work on
 // each 4-token tile and a tile's accumulators are released as soon as they are in registers.
 // The first loads are issued before the rest of the set-up.  Waiting threads sleep in the barrier
@@ -43,7 +44,13 @@ constexpr int UMAX = 128;              // largest tensor-core factor
 constexpr int STAGE_BYTES_MAX = TOK * UMAX * V * 2;   // 32 KB of bf16
 constexpr int A_BYTES = UMAX * UMAX * 2;              // 32 KB: A as bf16, two K blocks of 64
 constexpr int EPI_WARPS = 4 * TOK;
-constexpr int THREADS = 32 * (2 + EPI_WARPS);
+// Two threads issue the MMAs, on alternate tiles: in the running kernel a tcgen05.mma takes about three times
+// as long as alone on the SM and one issuing thread is busy for most of a tile's period; the second one (on
+// another scheduler) takes 1 - 3 % off the steady state.  Every stage must belong to one issuer, so that the
+// phase parities it waits for cannot alias: the count divides STAGES.
+constexpr int N_ISSUERS = 2;
+static_assert(STAGES % N_ISSUERS == 0, "a stage is served by one MMA issuer");
+constexpr int THREADS = 32 * (1 + N_ISSUERS + EPI_WARPS);   // producer, issuers (warp 1 and the last ones), epilogue
 constexpr int TMEM_COLS = 512;
 constexpr int STAGE_COLS = TOK * V;               // 128 fp32 columns per stage
 
@@ -187,8 +194,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
                 tma_load_3d(S->b[s], &tmap, &S->full[s], 0, 0, g * TOK);
             }
         }
-    } else if (warp == 1) {
-        // ------------------------------ MMA issuer ------------------------------
+    } else if (warp == 1 || warp >= 2 + EPI_WARPS) {
+        // ------------------------------ MMA issuers ------------------------------
+        const int issuer = warp == 1 ? 0 : warp - (2 + EPI_WARPS) + 1;        // takes tiles issuer, issuer + N_ISSUERS, ..
         if (lane == 0) {
             constexpr unsigned IDESC = instr_desc(UMAX, STAGE_COLS);
             const unsigned a_base = smem_u32(S->a);
@@ -198,8 +206,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
             const unsigned ad_lo0 = (unsigned)ad0, ad_hi = (unsigned)(ad0 >> 32);
             const unsigned bd_lo0 = (unsigned)bd0, bd_hi = (unsigned)(bd0 >> 32);
             bool ok = mbar_wait(&S->abort_flag, &S->abar, 0, P.status, 6);
-            int it = 0;
-            for (int g = blockIdx.x; ok && g < P.n_groups; g += gridDim.x, ++it) {
+            int it = issuer;
+            for (int g = blockIdx.x + issuer * (int)gridDim.x; ok && g < P.n_groups; g += N_ISSUERS * (int)gridDim.x, it += N_ISSUERS) {
                 const int s = it % STAGES;
                 const unsigned ph = (it / STAGES) & 1;
                 if (!mbar_wait(&S->abort_flag, &S->full[s], ph, P.status, 2)) break;
