@@ -32,7 +32,13 @@ constexpr int A_BYTES = UMAX * UMAX * 2;
 constexpr int B_BYTES = 160 * 1024;               // shared memory for the row stages
 constexpr int MAX_STAGES = 4;
 constexpr int EPI_WARPS = 16;
-constexpr int THREADS = 32 * (2 + EPI_WARPS);
+// With G = 2 a token is one 128 x 64 x K contraction and the epilogue per token is short: the thread that issues
+// the MMAs (about 200 cycles each in the running kernel) is then the bottleneck, and a second issuing thread on
+// another scheduler takes every other token (55 -> 42 us for 8192 x 8192).  With G = 4 or 8 it does not pay.
+// Every shared-memory and TMEM stage stays with one issuer (both stage counts are even), so the phase
+// parities an issuer waits for cannot alias.
+__host__ __device__ constexpr int issuers_for(int glog) { return glog == 1 ? 2 : 1; }
+__host__ __device__ constexpr int threads_for(int glog) { return 32 * (1 + issuers_for(glog) + EPI_WARPS); }
 constexpr int TMEM_COLS = 512;
 
 struct __align__(1024) Smem {
@@ -166,7 +172,7 @@ __device__ __forceinline__ void tmem_ld_wait_n<32>(unsigned* r)
 // candidates at a time over the warp's chunks; warp sums go to shared memory, a third named barrier, and the
 // first warp of the group adds the eight parts in a fixed order (per-row output, fp64 running totals).
 template <int BITS, int GLOG, bool GROUPED, bool CLIP>
-__global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant__ CUtensorMap tmap,
+__global__ void __launch_bounds__(threads_for(GLOG), 1) k_tc_uvm_rq(const __grid_constant__ CUtensorMap tmap,
                                                           const __grid_constant__ UvmParams P)
 {
     constexpr int G = 1 << GLOG;                  // chunks of 32 coordinates per TMEM lane
@@ -224,7 +230,9 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
                                 &S->full[s], 0, c, 0, tk);
             }
         }
-    } else if (warp == 1) {
+    } else if (warp == 1 || warp >= 2 + EPI_WARPS) {
+        constexpr int NISS = issuers_for(GLOG);
+        const int issuer = warp == 1 ? 0 : warp - (2 + EPI_WARPS) + 1;      // takes tokens issuer, issuer + NISS, ..
         // ------------------------------ MMA issuer ------------------------------
         if (lane == 0) {
             constexpr unsigned IDESC = instr_desc(UMAX, NCOLS);
@@ -235,8 +243,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
             const unsigned ad_lo0 = (unsigned)ad0, ad_hi = (unsigned)(ad0 >> 32);
             const unsigned bd_lo0 = (unsigned)bd0, bd_hi = (unsigned)(bd0 >> 32);
             bool ok = mbar_wait(&S->abort_flag, &S->abar, 0, P.status, 6);
-            int it = 0;
-            for (int tk = blockIdx.x; ok && tk < n_tok; tk += gridDim.x, ++it) {
+            int it = issuer;
+            for (int tk = blockIdx.x + issuer * (int)gridDim.x; ok && tk < n_tok; tk += NISS * (int)gridDim.x, it += NISS) {
                 const int s = it % nst, ts = it % TSTAGES;
                 if (!mbar_wait(&S->abort_flag, &S->full[s], (it / nst) & 1, P.status, 2)) break;
                 if (!mbar_wait(&S->abort_flag, &S->tempty[ts], ((it / TSTAGES) & 1) ^ 1, P.status, 3)) break;
@@ -489,14 +497,14 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvm_rq(const __grid_constant_
 }
 
 template <typename KernelT>
-cudaError_t launch(KernelT kernel, int grid, int smem, cudaStream_t stream, bool pdl, const CUtensorMap& tmap,
+cudaError_t launch(KernelT kernel, int threads, int grid, int smem, cudaStream_t stream, bool pdl, const CUtensorMap& tmap,
                    const UvmParams& P)
 {
     cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e != cudaSuccess) return e;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
-    cfg.blockDim = dim3(THREADS);
+    cfg.blockDim = dim3((unsigned)threads);
     cfg.dynamicSmemBytes = (size_t)smem;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -595,8 +603,8 @@ int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
     const bool pdl = p->pdl != 0;
     cudaError_t e;
 #define GBS_UVM_LAUNCH(B, GL)                                                                   \
-    (p->group ? launch(k_tc_uvm_rq<B, GL, true, false>, grid, smem, stream, pdl, tmap, P)        \
-              : launch(k_tc_uvm_rq<B, GL, false, false>, grid, smem, stream, pdl, tmap, P))
+    (p->group ? launch(k_tc_uvm_rq<B, GL, true, false>, threads_for(GL), grid, smem, stream, pdl, tmap, P)        \
+              : launch(k_tc_uvm_rq<B, GL, false, false>, threads_for(GL), grid, smem, stream, pdl, tmap, P))
     if (p->bits == 3) {
         if (glog == 1) e = GBS_UVM_LAUNCH(3, 1);
         else if (glog == 2) e = GBS_UVM_LAUNCH(3, 2);
@@ -631,8 +639,8 @@ int gbs_tc_uvm_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int6
     const bool pdl = p->pdl != 0;
     cudaError_t e;
 #define GBS_UVM_CLIP(GL)                                                                        \
-    (p->group ? launch(k_tc_uvm_rq<4, GL, true, true>, grid, smem, stream, pdl, tmap, P)         \
-              : launch(k_tc_uvm_rq<4, GL, false, true>, grid, smem, stream, pdl, tmap, P))
+    (p->group ? launch(k_tc_uvm_rq<4, GL, true, true>, threads_for(GL), grid, smem, stream, pdl, tmap, P)         \
+              : launch(k_tc_uvm_rq<4, GL, false, true>, threads_for(GL), grid, smem, stream, pdl, tmap, P))
     if (glog == 1) e = GBS_UVM_CLIP(1);
     else if (glog == 2) e = GBS_UVM_CLIP(2);
     else e = GBS_UVM_CLIP(3);
