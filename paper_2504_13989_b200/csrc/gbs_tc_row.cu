@@ -17,6 +17,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <mutex>
+
 #include "gbs_internal.h"
 #include "gbs_tc_common.cuh"
 
@@ -370,10 +372,13 @@ int row_prepare(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride
     return 0;
 }
 
-// opt in to the large dynamic shared memory once per device (not a stream operation)
+// opt in to the large dynamic shared memory once per device (not a stream operation); callable from several
+// host threads at once
 cudaError_t row_opt_in(const gbs_plan* p, int smem)
 {
+    static std::mutex mu;
     static bool attr_done[64] = {false};
+    std::lock_guard<std::mutex> lock(mu);
     if (p->device >= 0 && p->device < 64 && attr_done[p->device]) return cudaSuccess;
     cudaError_t e = cudaFuncSetAttribute(k_tc_row_rq<3, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_row_rq<4, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);

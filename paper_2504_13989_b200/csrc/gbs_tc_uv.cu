@@ -31,6 +31,7 @@
 #include <string.h>
 
 #include <mutex>
+#include <type_traits>
 
 #include "gbs_internal.h"
 #include "gbs_tc_common.cuh"
@@ -136,7 +137,8 @@ __device__ __forceinline__ void clip_score32(const unsigned r[32], float M, cons
 // ---------------------------------------------------------------------------------------------
 // GROUPED = false: one scale per token.  GROUPED = true: one scale per 2^glog adjacent lanes (32 * 2^glog
 // consecutive coordinates), 2^glog <= 32.  CLIP = true: instead of quantizing, score K clip ratios.
-template <int BITS, bool GROUPED, bool CLIP>
+// WANT_Y = true: also write the rotated normalised values (the parity output of gbs_rotate_quantize).
+template <int BITS, bool GROUPED, bool CLIP, bool WANT_Y>
 __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__ CUtensorMap tmap,
                                                          const __grid_constant__ UvParams P)
 {
@@ -235,52 +237,146 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
         const int q = warp & 3;                   // TMEM lane quadrant this warp may access
         const int up = q * 32 + lane;             // u' : this thread owns outputs [up*32, up*32+32)
         const unsigned taddr0 = tmem_base + ((unsigned)(q * 32) << 16) + t * V;
-        double dacc0 = 0.0, dacc1 = 0.0;          // CLIP, quadrant-0 warps: totals of candidates lane, lane + 32
-        // output cursors of this thread, advanced by one grid stride of token groups per iteration
-        const bool lane_live = up < P.U;
-        const long long row_step = (long long)gridDim.x * TOK;
-        long long row = (long long)blockIdx.x * TOK + t;
-        unsigned char* cptr = P.codes + row * P.code_row_bytes + up * (V * BITS / 8);
-        const long long cstep = row_step * P.code_row_bytes;
-        float* sptr = P.scales + row * P.spr + (GROUPED ? (up >> P.glog) : 0);
-        const long long sstep = row_step * P.spr;
-        const bool scale_writer = GROUPED ? ((lane & ((1 << P.glog) - 1)) == 0) : (up == 0);
-        int it = 0;
-        for (long long g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it, row += row_step, cptr += cstep, sptr += sstep) {
-            const int s = it % STAGES;
-            const unsigned ph = (it / STAGES) & 1;
-            const bool ok = mbar_wait(&S->abort_flag, &S->tfull[s], ph, P.status, 4, false);
-            if (!CLIP && GROUPED && !ok) break;
-            unsigned r[32];
-            float M = 0.f;
-            if (ok) {
+        if (!CLIP) {
+            // ---- rotate-quantize.  The loop body is kept to the arithmetic: the kernel is bound by instruction
+            // issue in these sixteen warps, so per-iteration bookkeeping is precomputed (iteration counts instead of
+            // row comparisons, one lane mask for the group maximum) or folded into the data that is exchanged anyway
+            // (a warp whose wait expired hands its token's other warps a poisoned maximum instead of a flag).
+            const int n_it = (P.n_groups - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // tiles of this CTA
+            const long long row_step = (long long)gridDim.x * TOK;
+            const long long row0 = (long long)blockIdx.x * TOK + t;
+            int n_store = 0;                      // iterations in which this thread has a row (and a live lane) to store
+            if (up < P.U && row0 < P.n_rows) n_store = (int)((P.n_rows - row0 + row_step - 1) / row_step);
+            unsigned char* cptr = P.codes + row0 * P.code_row_bytes + up * (V * BITS / 8);
+            const long long cstep = row_step * P.code_row_bytes;
+            float* sptr = P.scales + row0 * P.spr + (GROUPED ? (up >> P.glog) : 0);
+            const long long sstep = row_step * P.spr;
+            float* yptr = WANT_Y ? P.y_opt + row0 * (long long)P.d_pad + up * V : nullptr;
+            const long long ystep = row_step * P.d_pad;
+            const unsigned gl = 1u << P.glog;     // lanes per quantization group (GROUPED)
+            const bool scale_writer = GROUPED ? ((lane & (gl - 1u)) == 0) : (up == 0);
+            const bool arriver = lane == 0;
+            // one iteration on pipeline stage s (a compile-time constant: the loop below is unrolled over the
+            // stages so that barrier addresses, TMEM columns and the exchange slot are immediates); false = leave
+            auto tile = [&](auto stage, int it, unsigned ph) -> bool {
+                constexpr int s = decltype(stage)::value;
+                if (!mbar_wait(&S->abort_flag, &S->tfull[s], ph, P.status, 4, false)) {
+                    // this warp's wait expired.  With per-token scales the token's other three warps are (or will
+                    // be) waiting at the named barrier: come there once more, with a pattern no maximum of absolute
+                    // values can have (sign bit set); whoever sees it leaves too, so the four leave together.
+                    if (!GROUPED) {
+                        if (arriver) reinterpret_cast<unsigned*>(&S->red[t][s & 1][0])[q] = 0xffffffffu;
+                        asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
+                    }
+                    return false;
+                }
+                unsigned r[32];
                 tc_fence_after();
                 tmem_ld32_issue(taddr0 + s * STAGE_COLS, r);
                 tmem_ld_wait(r);
                 // the accumulators are in registers: hand the TMEM stage back to the MMA issuer
                 tc_fence_before();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&S->tempty[s]);
-                M = fwht32_absmax(r);
-            }
-            const unsigned gp = it & 1;
-            if (GROUPED) {
-                for (int o = (1 << P.glog) >> 1; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-            } else {
-                // per-token max: one warp-wide integer max (the values are non-negative floats), then the four
-                // quadrant warps of the token meet at a 128-thread named barrier.  A warp whose wait expired
-                // still comes to the barrier and raises the slot's flag first, so the four leave together.
-                const unsigned mw = __reduce_max_sync(0xffffffffu, __float_as_uint(M));
-                if (lane == 0) {
-                    S->red[t][gp][q] = __uint_as_float(mw);
-                    if (!ok) S->gabort[t][gp] = 1;
+                if (arriver) mbar_arrive(&S->tempty[s]);
+                float M = fwht32_absmax(r);
+                if (GROUPED) {
+                    // fold over the 2^glog lanes of this thread's group (a redux with one mask per group would be
+                    // issued once per distinct mask, which is slower for small groups)
+                    switch (P.glog) {
+                        case 5: M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 16));   // fall through
+                        case 4: M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 8));    // fall through
+                        case 3: M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 4));    // fall through
+                        case 2: M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 2));    // fall through
+                        case 1: M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, 1));    // fall through
+                        default: break;
+                    }
+                } else {
+                    // per-token max: a warp-wide integer max (the values are non-negative floats), then the four
+                    // quadrant warps of the token meet at a 128-thread named barrier
+                    const unsigned mw = __reduce_max_sync(0xffffffffu, __float_as_uint(M));
+                    unsigned* slot = reinterpret_cast<unsigned*>(&S->red[t][s & 1][0]);
+                    if (arriver) slot[q] = mw;
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
+                    const uint4 m4 = *reinterpret_cast<const uint4*>(slot);
+                    const unsigned mb = max(max(m4.x, m4.y), max(m4.z, m4.w));
+                    if ((int)mb < 0) return false;
+                    M = __uint_as_float(mb);
                 }
-                asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
-                const float4 m4 = *reinterpret_cast<const float4*>(&S->red[t][gp][0]);
-                M = fmaxf(fmaxf(m4.x, m4.y), fmaxf(m4.z, m4.w));
-                if (!CLIP && S->gabort[t][gp]) break;
+                // an all-zero token or group has every value at zero: any finite factor gives code 0.  Rows past
+                // the end (last tile only) and dead lanes are quantized like the rest; only the stores are guarded.
+                const float a1 = __fdividef(P.c_half, fmaxf(M, 1e-30f));
+                unsigned out[BITS];
+                quantize_pack32<BITS>(r, a1, out);
+                const bool st = it < n_store;
+                unsigned* dst = reinterpret_cast<unsigned*>(cptr);
+                if (BITS == 4) {
+                    if (st) *reinterpret_cast<uint4*>(dst) = make_uint4(out[0], out[1], out[2], out[3]);
+                } else {
+                    if (st) { dst[0] = out[0]; dst[1] = out[1]; dst[2] = out[2]; }
+                }
+                if (st && scale_writer) *sptr = P.c_scale * M;
+                if (WANT_Y) {
+                    if (st) {
+                        float4* yo = reinterpret_cast<float4*>(yptr);
+#pragma unroll
+                        for (int i = 0; i < 8; ++i)
+                            yo[i] = make_float4(__uint_as_float(r[4 * i]) * P.norm, __uint_as_float(r[4 * i + 1]) * P.norm,
+                                                __uint_as_float(r[4 * i + 2]) * P.norm, __uint_as_float(r[4 * i + 3]) * P.norm);
+                    }
+                    yptr += ystep;
+                }
+                cptr += cstep;
+                sptr += sstep;
+                return true;
+            };
+            static_assert(STAGES == 4, "the epilogue loop is unrolled over four stages");
+            unsigned ph = 0;
+            for (int it = 0;; ph ^= 1u) {
+                if (it >= n_it || !tile(std::integral_constant<int, 0>{}, it, ph)) break;
+                ++it;
+                if (it >= n_it || !tile(std::integral_constant<int, 1>{}, it, ph)) break;
+                ++it;
+                if (it >= n_it || !tile(std::integral_constant<int, 2>{}, it, ph)) break;
+                ++it;
+                if (it >= n_it || !tile(std::integral_constant<int, 3>{}, it, ph)) break;
+                ++it;
             }
-            if (CLIP) {
+        } else {
+            // ---- clip-ratio scoring
+            double dacc0 = 0.0, dacc1 = 0.0;      // quadrant-0 warps: totals of candidates lane, lane + 32
+            long long row = (long long)blockIdx.x * TOK + t;
+            const long long row_step = (long long)gridDim.x * TOK;
+            int it = 0;
+            for (long long g = blockIdx.x; g < P.n_groups; g += gridDim.x, ++it, row += row_step) {
+                const int s = it % STAGES;
+                const unsigned ph = (it / STAGES) & 1;
+                const bool ok = mbar_wait(&S->abort_flag, &S->tfull[s], ph, P.status, 4, false);
+                unsigned r[32];
+                float M = 0.f;
+                if (ok) {
+                    tc_fence_after();
+                    tmem_ld32_issue(taddr0 + s * STAGE_COLS, r);
+                    tmem_ld_wait(r);
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&S->tempty[s]);
+                    M = fwht32_absmax(r);
+                }
+                const unsigned gp = it & 1;
+                if (GROUPED) {
+                    for (int o = (1 << P.glog) >> 1; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+                } else {
+                    // per-token max: warp-wide integer max, then the token's four quadrant warps meet at a named
+                    // barrier; a warp whose wait expired still comes and raises the slot's flag first
+                    const unsigned mw = __reduce_max_sync(0xffffffffu, __float_as_uint(M));
+                    if (lane == 0) {
+                        S->red[t][gp][q] = __uint_as_float(mw);
+                        if (!ok) S->gabort[t][gp] = 1;
+                    }
+                    asm volatile("bar.sync %0, 128;" ::"r"(1 + t) : "memory");
+                    const float4 m4 = *reinterpret_cast<const float4*>(&S->red[t][gp][0]);
+                    M = fmaxf(fmaxf(m4.x, m4.y), fmaxf(m4.z, m4.w));
+                }
                 // each quadrant warp leaves its 32-lane sums in shared memory; the four meet at the token's
                 // named barrier (a warp whose wait expired comes too, flag raised), then the quadrant-0 warp
                 // adds the four parts in a fixed order: per-row output and fp64 running totals
@@ -296,31 +392,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
                         if (k < 32) dacc0 += (double)rk; else dacc1 += (double)rk;
                     }
                 }
-                continue;
             }
-            if (lane_live && row < P.n_rows) {
-                const float a1 = (M > 0.f) ? __fdividef(P.c_half, M) : 0.f;
-                unsigned out[BITS];
-                quantize_pack32<BITS>(r, a1, out);
-                unsigned* dst = reinterpret_cast<unsigned*>(cptr);
-                if (BITS == 4) {
-                    *reinterpret_cast<uint4*>(dst) = make_uint4(out[0], out[1], out[2], out[3]);
-                } else {
-                    dst[0] = out[0]; dst[1] = out[1]; dst[2] = out[2];
-                }
-                if (scale_writer) *sptr = P.c_scale * M;
-                if (P.y_opt) {
-                    float4* yo = reinterpret_cast<float4*>(P.y_opt + row * (long long)P.d_pad + up * V);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        yo[i] = make_float4(__uint_as_float(r[4 * i]) * P.norm, __uint_as_float(r[4 * i + 1]) * P.norm,
-                                            __uint_as_float(r[4 * i + 2]) * P.norm, __uint_as_float(r[4 * i + 3]) * P.norm);
-                }
+            if (q == 0) {
+                if (lane < P.K) atomicAdd(&P.err_sum[lane], dacc0 * (double)P.norm2);
+                if (lane + 32 < P.K) atomicAdd(&P.err_sum[lane + 32], dacc1 * (double)P.norm2);
             }
-        }
-        if (CLIP && q == 0) {
-            if (lane < P.K) atomicAdd(&P.err_sum[lane], dacc0 * (double)P.norm2);
-            if (lane + 32 < P.K) atomicAdd(&P.err_sum[lane + 32], dacc1 * (double)P.norm2);
         }
     }
 
@@ -441,17 +517,34 @@ int uv_prepare(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride,
     return 0;
 }
 
-// opt in to the large dynamic shared memory once per device (not a stream operation)
+// every instantiation, indexed [bits - 3][grouped][want_y] and [grouped] for the scoring form
+typedef void (*UvKernel)(const CUtensorMap, const UvParams);
+UvKernel uv_rq_kernel(int bits, bool grouped, bool want_y)
+{
+    static const UvKernel table[2][2][2] = {
+        {{k_tc_uv_rq<3, false, false, false>, k_tc_uv_rq<3, false, false, true>},
+         {k_tc_uv_rq<3, true, false, false>, k_tc_uv_rq<3, true, false, true>}},
+        {{k_tc_uv_rq<4, false, false, false>, k_tc_uv_rq<4, false, false, true>},
+         {k_tc_uv_rq<4, true, false, false>, k_tc_uv_rq<4, true, false, true>}}};
+    return table[bits - 3][grouped ? 1 : 0][want_y ? 1 : 0];
+}
+UvKernel uv_clip_kernel(bool grouped) { return grouped ? k_tc_uv_rq<4, true, true, false> : k_tc_uv_rq<4, false, true, false>; }
+
+// opt in to the large dynamic shared memory once per device (not a stream operation); callable from several
+// host threads at once
 cudaError_t uv_opt_in(const gbs_plan* p, int smem)
 {
+    static std::mutex mu;
     static bool attr_done[64] = {false};
+    std::lock_guard<std::mutex> lock(mu);
     if (p->device >= 0 && p->device < 64 && attr_done[p->device]) return cudaSuccess;
-    cudaError_t e = cudaFuncSetAttribute(k_tc_uv_rq<3, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<4, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<3, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<4, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<4, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_uv_rq<4, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    cudaError_t e = cudaSuccess;
+    for (int bits = 3; bits <= 4 && e == cudaSuccess; ++bits)
+        for (int g = 0; g < 2 && e == cudaSuccess; ++g)
+            for (int y = 0; y < 2 && e == cudaSuccess; ++y)
+                e = cudaFuncSetAttribute(uv_rq_kernel(bits, g != 0, y != 0), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+    for (int g = 0; g < 2 && e == cudaSuccess; ++g)
+        e = cudaFuncSetAttribute(uv_clip_kernel(g != 0), cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
     if (e == cudaSuccess && p->device >= 0 && p->device < 64) attr_done[p->device] = true;
     return e;
 }
@@ -473,13 +566,7 @@ int gbs_tc_uv_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, 
     cudaError_t e = uv_opt_in(p, smem);
     if (e != cudaSuccess) return (int)e;
     const bool pdl = p->pdl != 0;
-    if (p->group) {
-        if (p->bits == 3) e = launch(k_tc_uv_rq<3, true, false>, grid, smem, stream, pdl, tmap, P);
-        else e = launch(k_tc_uv_rq<4, true, false>, grid, smem, stream, pdl, tmap, P);
-    } else {
-        if (p->bits == 3) e = launch(k_tc_uv_rq<3, false, false>, grid, smem, stream, pdl, tmap, P);
-        else e = launch(k_tc_uv_rq<4, false, false>, grid, smem, stream, pdl, tmap, P);
-    }
+    e = launch(uv_rq_kernel(p->bits, p->group != 0, y_opt != nullptr), grid, smem, stream, pdl, tmap, P);
     return (int)e;
 }
 
@@ -504,8 +591,7 @@ int gbs_tc_uv_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int64
     cudaError_t e = uv_opt_in(p, smem);
     if (e != cudaSuccess) return (int)e;
     const bool pdl = p->pdl != 0;
-    if (p->group) e = launch(k_tc_uv_rq<4, true, true>, grid, smem, stream, pdl, tmap, P);
-    else e = launch(k_tc_uv_rq<4, false, true>, grid, smem, stream, pdl, tmap, P);
+    e = launch(uv_clip_kernel(p->group != 0), grid, smem, stream, pdl, tmap, P);
     return (int)e;
 }
 
