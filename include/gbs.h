@@ -133,6 +133,16 @@ int gbs_plan_info(const gbs_plan_t* plan, gbs_plan_info_t* out);
 int gbs_plan_device_status(const gbs_plan_t* plan, int* out);
 
 /*
+ * Self-test of the bounded waits (a diagnostic of this implementation, not an operation of the paper): one
+ * thread of a one-block kernel on the current device waits, for at most `limit_us` microseconds (1 .. 1 000 000),
+ * on a barrier that nothing arrives at.  The wait must run out: the call then returns GBS_OK with *code_out = 7
+ * (the code that wait records in its status word), *abort_out = 1 (the flag it raises for the other roles of a
+ * kernel) and *waited_us_out = how long it waited (limit_us plus at most a few polling periods).  Nothing
+ * faults or hangs; the context stays usable.  Runs on the default stream and WAITS for the device.
+ */
+int gbs_selftest_wait_expiry(int limit_us, int* code_out, int* abort_out, int* waited_us_out);
+
+/*
  * Fused pad -> rotate -> per-token/group absmax -> scale -> round/clip -> pack
  * (Section 4.2, Eq. (1), Algorithm 2, Section 2.1, Section 3.1), one pass over x.
  *   x            device, n_rows rows of d elements of x_dtype; row r starts at element
@@ -164,7 +174,8 @@ int gbs_rotate_quantize(const gbs_plan_t* plan, const void* x, int x_dtype, int6
  * allocating routine, and the caller still passes the input and both outputs.
  *
  *   d, d_pad, m, bits, group, alpha   as for gbs_plan_create, with these extra limits: bf16 rows only;
- *                d_pad <= GBS_STATIC_MAX_D_PAD; d_pad and d multiples of 32; d_pad / 32 a multiple of
+ *                d_pad <= GBS_STATIC_MAX_D_PAD; m one of 1, 12, 20, 24, 28 (the array's writer keeps one
+ *                32-bit sign word per row of H_m); d_pad and d multiples of 32; d_pad / 32 a multiple of
  *                16; group 0 or 32 .. 1024.  Anything else in gbs_plan_create's range returns
  *                GBS_ERR_UNSUPPORTED ("larger than the fixed array serves, or outside its kernel"):
  *                use a plan for those.
@@ -172,17 +183,30 @@ int gbs_rotate_quantize(const gbs_plan_t* plan, const void* x, int x_dtype, int6
  *                x_dtype = GBS_DTYPE_BF16; results are identical to the plan-based call.
  *
  * The array is shared by every call on a device and keeps what the last call left in it:
- *   - The first call on a device looks up the array's device address (with that device current) and
- *     clears the status word.  Make that first call before any stream capture begins.
- *   - A call whose (d_pad, m) differs from the previous call's on that device first rewrites the
- *     table, with a small kernel on `cuda_stream`; calls with the same (d_pad, m) reuse it.
+ *   - The first call on a device looks up the array's device address (with that device current).  Make
+ *     that first call before any stream capture begins.  The status word starts at zero (the array is
+ *     zero-initialised when the library's device code is loaded).
+ *   - A call reuses the table as it stands only if the previous call on that device used the same
+ *     (d_pad, m) on the same stream; every other call first rewrites the table with a small kernel on
+ *     `cuda_stream`, so its own kernel is ordered behind the write.  A call made while `cuda_stream` is
+ *     being captured always includes the rewrite, and after the first captured call on a device every
+ *     call rewrites (a replay changes the array without passing through this function).
  *   - Calls that can overlap on the GPU (different streams, or different host threads without
- *     ordering between their streams) race on the array unless they all use the same (d_pad, m).
- *     Serialise them, or give the concurrent users plans.
+ *     ordering between their streams) are safe when they all use the same (d_pad, m): they rewrite the
+ *     same bytes.  Overlapping calls with DIFFERENT (d_pad, m) race on the array: serialise them, or
+ *     give the concurrent users plans.
  */
 int gbs_rotate_quantize_static(int d, int d_pad, int m, int bits, int group, float alpha, const void* x,
                                int64_t n_rows, int64_t x_row_stride, void* codes, float* scales,
                                void* cuda_stream);
+
+/*
+ * Read and clear the status word of gbs_rotate_quantize_static on the current device (the counterpart of
+ * gbs_plan_device_status for the plan-free call: 0 = no bounded wait has expired since the last read).
+ * Copies 4 bytes from the fixed array, so it WAITS for the device's pending work; allocates nothing.
+ * (The paper has no counterpart of this call: a diagnostic of this implementation.)
+ */
+int gbs_static_device_status(int* out);
 
 /*
  * Inverse of the quantizer: yhat = q * Delta (Section 2.1) in the rotated domain, width d';

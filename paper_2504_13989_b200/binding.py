@@ -28,8 +28,8 @@ GBS_MAX_CANDIDATES = 64
 
 GBS_PLAN_ASYMMETRIC = 1
 EXPORTS = ("gbs_plan_create", "gbs_plan_create_ex", "gbs_plan_destroy", "gbs_plan_info", "gbs_plan_device_status", "gbs_rotate_quantize",
-           "gbs_rotate_quantize_static", "gbs_dequantize", "gbs_clip_error", "gbs_search_clip_ratio",
-           "gbs_hadamard_m", "gbs_status_string")
+           "gbs_rotate_quantize_static", "gbs_static_device_status", "gbs_dequantize", "gbs_clip_error",
+           "gbs_search_clip_ratio", "gbs_hadamard_m", "gbs_status_string", "gbs_selftest_wait_expiry")
 GBS_STATIC_MAX_D_PAD = 4096
 
 
@@ -79,6 +79,10 @@ def lib() -> ctypes.CDLL:
         L.gbs_rotate_quantize.restype = i32
         L.gbs_rotate_quantize_static.argtypes = [i32, i32, i32, i32, i32, ctypes.c_float, vp, i64, i64, vp, vp, vp]
         L.gbs_rotate_quantize_static.restype = i32
+        L.gbs_selftest_wait_expiry.argtypes = [i32, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(i32)]
+        L.gbs_selftest_wait_expiry.restype = i32
+        L.gbs_static_device_status.argtypes = [ctypes.POINTER(i32)]
+        L.gbs_static_device_status.restype = i32
         L.gbs_dequantize.argtypes = [vp, vp, vp, i64, vp, i32, i32, vp]
         L.gbs_dequantize.restype = i32
         L.gbs_clip_error.argtypes = [vp, vp, i32, i64, i64, ctypes.POINTER(ctypes.c_float), i32, vp, vp, vp]
@@ -135,6 +139,21 @@ def _rows_view(x: torch.Tensor, d: int):
     return x, x.shape[0], (x.stride(0) if x.shape[0] > 1 else max(x.stride(0), d))
 
 
+def _check_buffer(what: str, t: torch.Tensor, like: torch.Tensor, dtype, min_numel: int):
+    """The C ABI cannot validate pointers; the binding knows the tensors behind them.  An undersized, CPU or
+    strided buffer would make a kernel write out of bounds on the device, so it is refused here."""
+    if not isinstance(t, torch.Tensor) or not t.is_cuda:
+        raise ValueError("gbs: %s must be a CUDA tensor" % what)
+    if t.device != like.device:
+        raise ValueError("gbs: %s is on %s but the rows are on %s" % (what, t.device, like.device))
+    if dtype is not None and t.dtype != dtype:
+        raise TypeError("gbs: %s must be %s, got %s" % (what, dtype, t.dtype))
+    if not t.is_contiguous():
+        raise ValueError("gbs: %s must be contiguous" % what)
+    if t.numel() < min_numel:
+        raise ValueError("gbs: %s holds %d elements, the call writes %d" % (what, t.numel(), min_numel))
+
+
 # ----------------------------------------------------------------------------------------------
 # functions named after the C entry points
 # ----------------------------------------------------------------------------------------------
@@ -180,6 +199,10 @@ def gbs_rotate_quantize(plan: int, x: torch.Tensor, codes: torch.Tensor, scales:
                         y_opt: torch.Tensor | None = None, stream=None) -> None:
     info = gbs_plan_info(plan)
     xv, n_rows, stride = _rows_view(x, info.d)
+    _check_buffer("codes", codes, xv, torch.uint8, n_rows * info.code_bytes_per_row)
+    _check_buffer("scales", scales, xv, torch.float32, n_rows * info.scale_floats_per_row)
+    if y_opt is not None:
+        _check_buffer("y_opt", y_opt, xv, torch.float32, n_rows * info.d_pad)
     _check(lib().gbs_rotate_quantize(ctypes.c_void_p(plan), xv.data_ptr(), _dtype_code(xv), n_rows, stride,
                                      codes.data_ptr(), scales.data_ptr(),
                                      y_opt.data_ptr() if y_opt is not None else None, _stream_ptr(stream)),
@@ -195,13 +218,36 @@ def gbs_rotate_quantize_static(d: int, d_pad: int, m: int, bits: int, group: int
     xv, n_rows, stride = _rows_view(x, d)
     if xv.dtype != torch.bfloat16:
         raise TypeError("gbs_rotate_quantize_static: x must be bfloat16")
+    if d_pad > 0 and bits in (3, 4):
+        _check_buffer("codes", codes, xv, torch.uint8, n_rows * (d_pad * bits // 8))
+        _check_buffer("scales", scales, xv, torch.float32, n_rows * (d_pad // group if group > 0 else 1))
     _check(lib().gbs_rotate_quantize_static(d, d_pad, m, bits, group, alpha, xv.data_ptr(), n_rows, stride,
                                             codes.data_ptr(), scales.data_ptr(), _stream_ptr(stream)),
            "gbs_rotate_quantize_static")
 
 
+def gbs_selftest_wait_expiry(limit_us: int = 1000):
+    """Run one bounded wait that is certain to run out; returns (code, abort flag, microseconds waited)."""
+    code, ab, us = ctypes.c_int(0), ctypes.c_int(0), ctypes.c_int(0)
+    _check(lib().gbs_selftest_wait_expiry(int(limit_us), ctypes.byref(code), ctypes.byref(ab), ctypes.byref(us)),
+           "gbs_selftest_wait_expiry")
+    return code.value, ab.value, us.value
+
+
+def gbs_static_device_status() -> int:
+    """Read and clear the status word of gbs_rotate_quantize_static on the current device.  Synchronises."""
+    v = ctypes.c_int(0)
+    _check(lib().gbs_static_device_status(ctypes.byref(v)), "gbs_static_device_status")
+    return v.value
+
+
 def gbs_dequantize(plan: int, codes: torch.Tensor, scales: torch.Tensor, n_rows: int, out: torch.Tensor,
                    flags: int = 0, stream=None) -> None:
+    info = gbs_plan_info(plan)
+    width = info.d if (flags & GBS_INVERSE_ROTATE) else info.d_pad
+    _check_buffer("codes", codes, codes, torch.uint8, n_rows * info.code_bytes_per_row)
+    _check_buffer("scales", scales, codes, torch.float32, n_rows * info.scale_floats_per_row)
+    _check_buffer("out", out, codes, None, n_rows * width)
     _check(lib().gbs_dequantize(ctypes.c_void_p(plan), codes.data_ptr(), scales.data_ptr(), n_rows,
                                 out.data_ptr(), _dtype_code(out), flags, _stream_ptr(stream)),
            "gbs_dequantize")
@@ -213,8 +259,9 @@ def gbs_clip_error(plan: int, x: torch.Tensor, alphas, err_sum: torch.Tensor,
     xv, n_rows, stride = _rows_view(x, info.d)
     alphas = [float(a) for a in alphas]
     arr = (ctypes.c_float * len(alphas))(*alphas)
-    if err_sum.dtype != torch.float64:
-        raise TypeError("gbs: err_sum must be float64")
+    _check_buffer("err_sum", err_sum, xv, torch.float64, len(alphas))
+    if err_rows_opt is not None:
+        _check_buffer("err_rows_opt", err_rows_opt, xv, torch.float32, n_rows * len(alphas))
     _check(lib().gbs_clip_error(ctypes.c_void_p(plan), xv.data_ptr(), _dtype_code(xv), n_rows, stride,
                                 arr, len(alphas), err_sum.data_ptr(),
                                 err_rows_opt.data_ptr() if err_rows_opt is not None else None,
@@ -230,6 +277,7 @@ def gbs_search_clip_ratio(plan: int, x: torch.Tensor, eps: float, work: torch.Te
     xv, n_rows, stride = _rows_view(x, info.d)
     if work is None:
         work = torch.empty(GBS_MAX_CANDIDATES, dtype=torch.float64, device=x.device)
+    _check_buffer("work", work, xv, torch.float64, GBS_MAX_CANDIDATES)
     res = SearchResult()
     _check(lib().gbs_search_clip_ratio(ctypes.c_void_p(plan), xv.data_ptr(), _dtype_code(xv), n_rows, stride,
                                        float(eps), work.data_ptr(), ctypes.byref(res), _stream_ptr(stream)),

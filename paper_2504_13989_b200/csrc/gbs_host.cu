@@ -36,24 +36,7 @@ int check_rows(const gbs_plan* p, const void* x, int x_dtype, int64_t n_rows, in
     return GBS_OK;
 }
 
-struct DeviceGuard {
-    int prev = -1;
-    bool switched = false;
-    cudaError_t enter(int dev)
-    {
-        cudaError_t e = cudaGetDevice(&prev);
-        if (e != cudaSuccess) return e;
-        if (prev != dev) {
-            e = cudaSetDevice(dev);
-            switched = (e == cudaSuccess);
-        }
-        return e;
-    }
-    ~DeviceGuard()
-    {
-        if (switched) cudaSetDevice(prev);
-    }
-};
+typedef gbs_device_guard DeviceGuard;
 
 }  // namespace
 

@@ -41,6 +41,26 @@ struct gbs_plan {
     int8_t h_hm[GBS_MAX_M * GBS_MAX_M];  // host copy of H_m
 };
 
+// Makes `dev` the current device for the lifetime of the object (entry points work on the plan's device).
+struct gbs_device_guard {
+    int prev = -1;
+    bool switched = false;
+    cudaError_t enter(int dev)
+    {
+        cudaError_t e = cudaGetDevice(&prev);
+        if (e != cudaSuccess) return e;
+        if (prev != dev) {
+            e = cudaSetDevice(dev);
+            switched = (e == cudaSuccess);
+        }
+        return e;
+    }
+    ~gbs_device_guard()
+    {
+        if (switched) cudaSetDevice(prev);
+    }
+};
+
 // gbs_paley.cu
 int gbs_build_hadamard_m(int m, int8_t* out);   // 0 or GBS_ERR_UNSUPPORTED
 bool gbs_supported_m(int m);                    // the orders a plan accepts

@@ -70,6 +70,8 @@ extern "C" int gbs_search_clip_ratio(const gbs_plan_t* plan, const void* x, int 
     if (n_rows <= 0) return GBS_ERR_INVALID_ARG;
     if (reinterpret_cast<uintptr_t>(work_dev) & 7u) return GBS_ERR_ALIGNMENT;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    gbs_device_guard guard;                       // the copies below belong to the plan's device, like its launches
+    if (guard.enter(plan->device) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
 
     State s = {0.0, 1.0, 0.5, 0};
     double f_m = 0.0;

@@ -47,18 +47,18 @@ __device__ __forceinline__ unsigned long long global_ns()
     return t;
 }
 
-// Bounded wait: gives up WAIT_LIMIT_NS after its first unsuccessful poll.  Returns false if the wait
+// Bounded wait: gives up limit_ns (by default WAIT_LIMIT_NS) after its first unsuccessful poll.  Returns false if the wait
 // expired (or, with watch_abort, once another role has aborted).  The epilogue warps wait without
 // watch_abort: they leave only on their own expiry, and the four warps of a token slot leave together.
 __device__ __noinline__ bool mbar_wait_slow(volatile int* abort_flag, void* bar, unsigned parity, int* status, int code,
-                                            bool watch_abort)
+                                            bool watch_abort, unsigned long long limit_ns = WAIT_LIMIT_NS)
 {
     const unsigned long long t0 = global_ns();
     for (unsigned i = 1;; ++i) {
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 15u) == 0) {
             if (watch_abort && *abort_flag) return false;
-            if (global_ns() - t0 > WAIT_LIMIT_NS) break;
+            if (global_ns() - t0 > limit_ns) break;
         }
     }
     *abort_flag = 1;

@@ -600,7 +600,8 @@ int gbs_tc_uv_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int64
 // ---------------------------------------------------------------------------------------------
 // The kernel above needs 32 KB of device memory besides its inputs and outputs (the image of A) and
 // a status word.  A plan gets them from cudaMalloc; here they live in a file-scope device array that
-// every GPU loading this library carries until the process exits.
+// every GPU loading this library carries until the process exits (zero-initialised when the module is
+// loaded, so the status word needs no clearing before its first use).
 namespace {
 
 constexpr int STATIC_IMAGE_BYTES = A_BYTES;
@@ -610,7 +611,7 @@ static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_B
 // Fills the image of A = H_m (x) H_{2^j} (same layout as gbs_tc_uv_a_image) straight into the array.
 struct StaticFillParams {
     int U, j;
-    unsigned hm_neg[32];          // bit a of word a': H_m[a'][a] == -1
+    unsigned hm_neg[32];          // bit a of word a': H_m[a'][a] == -1   (m <= 28 < 32)
 };
 __global__ void __launch_bounds__(256) k_static_fill_a(const __grid_constant__ StaticFillParams F)
 {
@@ -625,8 +626,11 @@ __global__ void __launch_bounds__(256) k_static_fill_a(const __grid_constant__ S
 #pragma unroll
             for (int t = 0; t < 2; ++t) {
                 const int k = kb * 64 + ch * 8 + e + t;
-                const unsigned neg = ((rowbits >> (k >> F.j)) ^ (unsigned)__popc((unsigned)r & (unsigned)k & jm)) & 1u;
-                const unsigned h = (r < F.U && k < F.U) ? (neg ? 0xBF80u : 0x3F80u) : 0u;
+                unsigned h = 0u;
+                if (r < F.U && k < F.U) {          // k < U keeps the shift below m <= 28
+                    const unsigned neg = ((rowbits >> (k >> F.j)) ^ (unsigned)__popc((unsigned)r & (unsigned)k & jm)) & 1u;
+                    h = neg ? 0xBF80u : 0x3F80u;
+                }
                 h2 |= h << (16 * t);
             }
             w[e >> 1] = h2;
@@ -639,10 +643,35 @@ __global__ void __launch_bounds__(256) k_static_fill_a(const __grid_constant__ S
 struct StaticDeviceState {
     unsigned char* scratch = nullptr;   // device address of g_static_scratch on this device
     int sm_count = 0, smem_optin = 0;
-    int image_m = 0, image_k = 0;       // which A the array holds now (0 = none yet)
+    // which A the array holds, and the stream whose work wrote it: a later call may skip the rewrite only if it
+    // is ordered behind that write, i.e. on the same stream (0 = nothing written yet)
+    int image_m = 0, image_k = 0;
+    cudaStream_t image_stream = nullptr;
+    bool seen_capture = false;          // a call was captured on this device: replays rewrite the array unseen
 };
 StaticDeviceState g_static_state[64];
 std::mutex g_static_mutex;
+
+// Set-up, once per device, with that device current: the array's name is only a host-side handle, the kernels
+// need its device address.  Caller holds g_static_mutex.
+int static_state(StaticDeviceState** out)
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return GBS_ERR_CUDA; }
+    StaticDeviceState& st = g_static_state[dev];
+    if (!st.scratch) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) { cudaGetLastError(); return GBS_ERR_CUDA; }
+        if (cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&st.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
+            cudaGetLastError();
+            return GBS_ERR_CUDA;
+        }
+        st.scratch = static_cast<unsigned char*>(ptr);
+    }
+    *out = &st;
+    return dev;
+}
 
 }  // namespace
 
@@ -662,7 +691,7 @@ extern "C" int gbs_rotate_quantize_static(int d, int d_pad, int m, int bits, int
     if (group != 0 && (group < 8 || (group & (group - 1)) != 0 || (1 << k) % group != 0)) return GBS_ERR_INVALID_ARG;
     if (n_rows < 0) return GBS_ERR_INVALID_ARG;
     if (d_pad > GBS_STATIC_MAX_D_PAD) return GBS_ERR_UNSUPPORTED;          // beyond what the fixed array serves
-    if (!(m == 1 || m == 12 || m == 20 || m == 24 || m == 28)) return GBS_ERR_UNSUPPORTED;   // orders a plan accepts
+    if (!(m == 1 || m == 12 || m == 20 || m == 24 || m == 28)) return GBS_ERR_UNSUPPORTED;   // m <= 28: one sign word per row
     gbs_plan p;
     memset(&p, 0, sizeof(p));
     if (gbs_build_hadamard_m(m, p.h_hm) != GBS_OK) return GBS_ERR_UNSUPPORTED;
@@ -687,35 +716,28 @@ extern "C" int gbs_rotate_quantize_static(int d, int d_pad, int m, int bits, int
     p.pdl = 0;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { cudaGetLastError(); return GBS_ERR_CUDA; }
-    p.device = dev;
     std::lock_guard<std::mutex> lock(g_static_mutex);
-    StaticDeviceState& st = g_static_state[dev];
-    if (!st.scratch) {
-        // set-up, once per device, with that device current: the array's name is only a host-side handle,
-        // the kernels need its device address
-        void* ptr = nullptr;
-        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) { cudaGetLastError(); return GBS_ERR_CUDA; }
-        if (cudaDeviceGetAttribute(&st.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-            cudaDeviceGetAttribute(&st.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev) != cudaSuccess) {
-            cudaGetLastError();
-            return GBS_ERR_CUDA;
-        }
-        if (st.smem_optin < (int)(sizeof(Smem) + 1024) || get_encode() == nullptr) return GBS_ERR_UNSUPPORTED;
-        // the status word must start at zero; the image is written below
-        if (cudaMemsetAsync(static_cast<unsigned char*>(ptr) + STATIC_IMAGE_BYTES, 0, 256, stream) != cudaSuccess) {
-            cudaGetLastError();
-            return GBS_ERR_CUDA;
-        }
-        st.scratch = static_cast<unsigned char*>(ptr);
-    }
+    StaticDeviceState* stp = nullptr;
+    const int dev = static_state(&stp);
+    if (dev < 0) return dev;
+    StaticDeviceState& st = *stp;
+    if (st.smem_optin < (int)(sizeof(Smem) + 1024) || get_encode() == nullptr) return GBS_ERR_UNSUPPORTED;
+    p.device = dev;
     p.sm_count = st.sm_count;
     p.smem_optin = st.smem_optin;
     p.d_aimg = st.scratch;
     p.d_status = reinterpret_cast<int*>(st.scratch + STATIC_IMAGE_BYTES);
-    if (st.image_m != m || st.image_k != k) {
-        // the array still holds the previous call's A: rewrite it, on the caller's stream, before the kernel
+    // The array may be reused as it stands only by a call that is ordered behind the work that wrote it: same
+    // table and same stream.  Every other call rewrites the table on its own stream first; two streams
+    // rewriting the same table write the same bytes.  A captured call always carries its rewrite (it runs at
+    // replay, not now), and once a call has been captured on this device the record kept here can no longer
+    // be trusted (a replay rewrites the array without passing through this function), so from then on every
+    // call rewrites.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
+    const bool capturing = cap != cudaStreamCaptureStatusNone;
+    if (capturing) st.seen_capture = true;
+    if (st.seen_capture || st.image_m != m || st.image_k != k || st.image_stream != stream) {
         StaticFillParams F;
         F.U = d_pad / V;
         F.j = k - 5;
@@ -730,8 +752,27 @@ extern "C" int gbs_rotate_quantize_static(int d, int d_pad, int m, int bits, int
         if (cudaGetLastError() != cudaSuccess) return GBS_ERR_CUDA;
         st.image_m = m;
         st.image_k = k;
+        st.image_stream = stream;
     }
     const int e = gbs_tc_uv_rotate_quantize(&p, x, n_rows, x_row_stride, codes, scales, nullptr, stream);
     if (e != 0) cudaGetLastError();
     return e == 0 ? GBS_OK : GBS_ERR_CUDA;
+}
+
+extern "C" int gbs_static_device_status(int* out)
+{
+    if (!out) return GBS_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticDeviceState* st = nullptr;
+    const int dev = static_state(&st);
+    if (dev < 0) return dev;
+    int v = 0;
+    int* word = reinterpret_cast<int*>(st->scratch + STATIC_IMAGE_BYTES);
+    if (cudaMemcpy(&v, word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemset(word, 0, sizeof(int)) != cudaSuccess) {
+        cudaGetLastError();
+        return GBS_ERR_CUDA;
+    }
+    *out = v;
+    return GBS_OK;
 }

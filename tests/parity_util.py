@@ -12,6 +12,12 @@ TOL_ROT_L2 = 1e-5
 TOL_SCALE = 1e-6
 TOL_CODE_FRAC = 1e-4
 TOL_CLIP = 1e-5
+# A code may differ from the oracle's only where the oracle's own y / Delta sits at a rounding tie: within
+# TIE_WINDOW of k + 1/2 (or of the clip edge D + 1/2).  fp32 arithmetic places y / Delta (at most 7 in
+# magnitude) within about 1e-6 of the float64 value; the window is ten times the largest distance the whole
+# GPU suite has shown (5.4e-7 over 3.1e8 codes; OBSERVED, printed at the end of every run).
+TIE_WINDOW = 5e-6
+OBSERVED = {"codes_compared": 0, "codes_mismatching": 0, "tie_dist_max": 0.0}
 
 
 def unpack_codes(buf: np.ndarray, n: int, bits: int) -> np.ndarray:
@@ -46,6 +52,8 @@ def compare_rotate_quantize(x: torch.Tensor, ref: dict, codes: torch.Tensor, sca
     D = 2 ** (bits - 1) - 1
     assert qg.min(initial=0) >= -D and qg.max(initial=0) <= D, "code outside [-D, D]"
     diff = qg != ref["q"]
+    OBSERVED["codes_compared"] += int(diff.size)
+    OBSERVED["codes_mismatching"] += int(diff.sum())
     frac = diff.mean() if diff.size else 0.0
     stats["code_mismatch_frac"] = float(frac)
     assert frac <= TOL_CODE_FRAC, "codes: mismatch fraction %.3e" % frac
@@ -57,8 +65,10 @@ def compare_rotate_quantize(x: torch.Tensor, ref: dict, codes: torch.Tensor, sca
         t = ref["y"][diff] / dl[diff]
         dist = np.abs(np.abs(t - np.floor(t)) - 0.5)
         clip_edge = np.abs(np.abs(t) - (D + 0.5))     # |t| just around D+0.5 is also a tie (then clamped)
-        stats["tie_dist_max"] = float(dist.max())
-        assert np.all((dist < 2e-4) | (clip_edge < 2e-4)), "a mismatching code is not at a rounding tie"
+        stats["tie_dist_max"] = float(np.minimum(dist, clip_edge).max())
+        OBSERVED["tie_dist_max"] = max(OBSERVED["tie_dist_max"], stats["tie_dist_max"])
+        assert np.all((dist < TIE_WINDOW) | (clip_edge < TIE_WINDOW)), \
+            "a mismatching code is %.3e away from a rounding tie" % stats["tie_dist_max"]
     return stats
 
 

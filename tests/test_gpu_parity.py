@@ -781,3 +781,21 @@ def test_one_plan_from_several_streams_and_host_threads():
         assert plan.device_status() == 0
         for (c, s, _), (cr, sr, _) in zip(results, refs):
             assert torch.equal(c, cr) and torch.equal(s, sr)
+
+
+@pytest.mark.gpu
+def test_a_bounded_wait_that_runs_out_returns_its_code_and_leaves_the_context_usable():
+    """The tensor-core kernels bound every barrier wait.  gbs_selftest_wait_expiry makes one such wait run out
+    (a barrier nothing arrives at, limit 1 ms): it must come back with the wait's code and raised abort flag
+    after about the limit, and a normal launch afterwards must still match the oracle."""
+    code, abort, waited_us = binding.gbs_selftest_wait_expiry(1000)
+    assert code == 7 and abort == 1
+    assert 1000 <= waited_us <= 5000, waited_us
+    w = synth.WORKLOADS["llama4096"]
+    x = synth.make_host("llama4096", 64, seed=3)
+    ref = oracle_rq(x, w, 3)
+    with Plan(w.d, w.d_pad, w.m, 3, w.group, w.alpha) as plan:
+        codes, scales, y = plan.rotate_quantize(x.to(DEV), want_y=True)
+        torch.cuda.synchronize()
+        compare_rotate_quantize(x, ref, codes, scales, y, 3, w.group, w.d_pad)
+        assert plan.device_status() == 0

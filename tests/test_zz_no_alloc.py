@@ -60,3 +60,65 @@ def test_static_entry_point_matches_the_plan_based_call_twice_in_a_row():
             assert torch.equal(codes, codes_ref), (name, bits, rows)
             assert torch.equal(scales, scales_ref), (name, bits, rows)
             assert plan.device_status() == 0
+            assert binding.gbs_static_device_status() == 0          # the plan-free call's own status word
+
+
+@pytest.mark.gpu
+def test_static_entry_point_from_two_streams_with_the_same_table_after_a_change():
+    """Callers on different streams that use the same (d_pad, m) may overlap: the shared table is rewritten on
+    the stream of every call that is not ordered behind the last write, and all of them write the same bytes.
+    A change of (d_pad, m) in between (serialised, as the header asks) must not leave either stream with a
+    stale table."""
+    gbs_build.build()
+    s1, s2 = torch.cuda.Stream(DEV), torch.cuda.Stream(DEV)
+    cases = []
+    for name, bits, rows in (("llama4096", 3, 2048), ("qwen3584", 3, 1024)):
+        w = synth.WORKLOADS[name]
+        x = synth.make_host(name, rows, seed=5 + bits).to(DEV)
+        with Plan(w.d, w.d_pad, w.m, bits, w.group, w.alpha) as plan:
+            ref = plan.rotate_quantize(x)
+            torch.cuda.synchronize()
+        cases.append((w, bits, x, ref))
+    for rounds in range(3):
+        for w, bits, x, (codes_ref, scales_ref, _) in cases:
+            outs = []
+            for s in (s1, s2, s1, s2):                      # same table on both streams, back to back, no host sync
+                codes = torch.full_like(codes_ref, 0xEE)
+                scales = torch.full_like(scales_ref, -1.0)
+                binding.gbs_rotate_quantize_static(w.d, w.d_pad, w.m, bits, w.group, w.alpha, x, codes, scales, stream=s)
+                outs.append((codes, scales))
+            torch.cuda.synchronize()                        # the change of table that follows is serialised
+            for codes, scales in outs:
+                assert torch.equal(codes, codes_ref) and torch.equal(scales, scales_ref), (w.name, rounds)
+    assert binding.gbs_static_device_status() == 0
+
+
+@pytest.mark.gpu
+def test_static_entry_point_inside_a_captured_graph_and_eagerly_afterwards():
+    """A captured call carries its own rewrite of the table, so a replay is right whatever ran in between,
+    and eager calls made after a replay rewrite too."""
+    gbs_build.build()
+    wa, wb = synth.WORKLOADS["llama4096"], synth.WORKLOADS["qwen3584"]
+    xa = synth.make_host("llama4096", 512, seed=11).to(DEV)
+    xb = synth.make_host("qwen3584", 512, seed=12).to(DEV)
+    with Plan(wa.d, wa.d_pad, wa.m, 4, wa.group, wa.alpha) as pa, Plan(wb.d, wb.d_pad, wb.m, 3, wb.group, wb.alpha) as pb:
+        ca_ref, sa_ref, _ = pa.rotate_quantize(xa)
+        cb_ref, sb_ref, _ = pb.rotate_quantize(xb)
+        ca, sa = torch.zeros_like(ca_ref), torch.zeros_like(sa_ref)
+        cb, sb = torch.zeros_like(cb_ref), torch.zeros_like(sb_ref)
+        st = torch.cuda.Stream(DEV)
+        binding.gbs_rotate_quantize_static(wa.d, wa.d_pad, wa.m, 4, wa.group, wa.alpha, xa, ca, sa, stream=st)   # set-up before capture
+        st.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            binding.gbs_rotate_quantize_static(wa.d, wa.d_pad, wa.m, 4, wa.group, wa.alpha, xa, ca, sa, stream=st)
+        for _ in range(2):
+            binding.gbs_rotate_quantize_static(wb.d, wb.d_pad, wb.m, 3, wb.group, wb.alpha, xb, cb, sb, stream=st)  # other table, eager
+            st.synchronize()
+            assert torch.equal(cb, cb_ref) and torch.equal(sb, sb_ref)
+            ca.zero_(); sa.zero_()
+            torch.cuda.synchronize()
+            g.replay()
+            torch.cuda.synchronize()
+            assert torch.equal(ca, ca_ref) and torch.equal(sa, sa_ref)
+        assert binding.gbs_static_device_status() == 0
