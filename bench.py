@@ -38,7 +38,8 @@ HEADLINE = "llama4096"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused kernel on the headline
 # workload, from the ncu capture summarised under profiles/ (None until a capture exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = 33_608_960   # reads 33.61 MB; the codes are still in L2 when the kernel ends
+NCU_TRAFFIC_BYTES_PER_LAUNCH = None         # set from the capture of the current kernel, see profiles/
+NCU_TRAFFIC_BYTES_PER_LAUNCH_D3584 = None
 
 
 def algorithmic_bytes(n_rows: int, d: int, d_pad: int, bits: int, group: int, in_bytes: int) -> int:
@@ -114,6 +115,14 @@ class ClockSampler(threading.Thread):
 
     def stop(self):
         self._stop_evt.set()
+
+    def mark(self) -> int:
+        return len(self.samples)
+
+    def median_mhz_since(self, mark: int):
+        """Median SM clock of the samples taken since mark() while the GPU was busy (None without samples)."""
+        pool = [s[0] for s in self.samples[mark:] if s[2] > 0] or [s[0] for s in self.samples[mark:]]
+        return statistics.median(pool) if pool else None
 
     def summary(self):
         if not self.ok or not self.samples:
@@ -228,8 +237,12 @@ def capture(plan_list, sets, idx_list, stream):
     return g
 
 
-def timed_graph_loop(plan_list, sets, steps, warmup, stream, dist_ok, sampler=None):
-    """Time exactly `steps` steps replayed from CUDA graphs; returns local milliseconds."""
+MIN_TIMED_MS = 50.0      # a timed region shorter than this is repeated (whole multiples of the K steps)
+
+
+def timed_graph_loop(plan_list, sets, steps, warmup, stream, dist_ok, sampler=None, min_ms=MIN_TIMED_MS):
+    """Time `steps` steps replayed from CUDA graphs, repeated R >= 1 times so that the timed region lasts at
+    least min_ms; returns (local milliseconds, steps actually timed = R * steps)."""
     nsets = len(sets)
     with torch.cuda.stream(stream):
         for i in range(max(warmup, 3)):
@@ -238,10 +251,26 @@ def timed_graph_loop(plan_list, sets, steps, warmup, stream, dist_ok, sampler=No
     g_all = capture(plan_list, sets, list(range(nsets)), stream)
     rem = steps % nsets
     g_rem = capture(plan_list, sets, list(range(rem)), stream) if rem else None
+
+    def k_steps():
+        for _ in range(steps // nsets):
+            g_all.replay()
+        if g_rem is not None:
+            g_rem.replay()
+
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with torch.cuda.stream(stream):
         g_all.replay()
+        start.record(stream)
+        g_all.replay()
+        end.record(stream)
     stream.synchronize()
-    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    est_ms = start.elapsed_time(end) / nsets * steps             # one pass over the K steps
+    reps = max(1, int(np.ceil(min_ms / max(est_ms, 1e-6))))
+    if dist_ok:
+        r = torch.tensor([reps], dtype=torch.int64, device=sets[0][0].device)
+        torch.distributed.all_reduce(r, op=torch.distributed.ReduceOp.MAX)
+        reps = int(r.item())
     if dist_ok:
         torch.distributed.barrier()
     torch.cuda.synchronize()
@@ -249,17 +278,55 @@ def timed_graph_loop(plan_list, sets, steps, warmup, stream, dist_ok, sampler=No
         sampler.in_timed = True
     with torch.cuda.stream(stream):
         start.record(stream)
-        for _ in range(steps // nsets):
-            g_all.replay()
-        if g_rem is not None:
-            g_rem.replay()
+        for _ in range(reps):
+            k_steps()
         end.record(stream)
     if dist_ok:
         torch.distributed.barrier()
     torch.cuda.synchronize()
     if sampler:
         sampler.in_timed = False
-    return start.elapsed_time(end)
+    return start.elapsed_time(end), steps * reps
+
+
+def plain_traffic(stream, device, read_bytes, write_bytes, min_ms=20.0):
+    """Size-matched denominators under the same protocol (graph replay, buffers rotating through > 4x L2):
+    a plain device copy that moves read_bytes + write_bytes in total (half of it read, half written), and a
+    plain fill of write_bytes.  Returns (copy GB/s of bytes read + written, fill GB/s)."""
+    out = []
+    for kind, nbytes in (("copy", (read_bytes + write_bytes) // 2), ("fill", write_bytes)):
+        nbytes = max(1024, nbytes // 16 * 16)
+        nsets = max(2, min(32, int(4 * 126e6 / nbytes) + 1))
+        src = [torch.empty(nbytes, dtype=torch.uint8, device=device).fill_(i) for i in range(nsets)] if kind == "copy" else None
+        dst = [torch.empty(nbytes, dtype=torch.uint8, device=device) for _ in range(nsets)]
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(stream):
+            for i in range(min(3, nsets)):
+                dst[i].copy_(src[i]) if kind == "copy" else dst[i].fill_(7)
+        stream.synchronize()
+        with torch.cuda.graph(g, stream=stream):
+            for i in range(nsets):
+                dst[i].copy_(src[(i + nsets // 2) % nsets]) if kind == "copy" else dst[i].fill_(7)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            g.replay()
+            a.record(stream)
+            g.replay()
+            b.record(stream)
+        stream.synchronize()
+        reps = max(1, int(np.ceil(min_ms / max(a.elapsed_time(b), 1e-6))))
+        with torch.cuda.stream(stream):
+            a.record(stream)
+            for _ in range(reps):
+                g.replay()
+            b.record(stream)
+        stream.synchronize()
+        ms = a.elapsed_time(b) / (reps * nsets)
+        moved = 2 * nbytes if kind == "copy" else nbytes
+        out.append(moved / ms / 1e6)
+        del src, dst, g
+        torch.cuda.empty_cache()
+    return out[0], out[1]
 
 
 def main():
@@ -307,7 +374,7 @@ def main():
         run_profile(args.profile, device)
         return
 
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(local_rank, period_s=0.005)
     sampler.start()
 
     w = synth.WORKLOADS[HEADLINE]
@@ -319,20 +386,45 @@ def main():
     step_tokens = len(w.bits) * w.n_rows
     launches_per_step = len(w.bits)
 
-    local_ms = timed_graph_loop(plans, sets, args.steps, args.warmup, stream, dist_ok, sampler)
-    total_ms, total_bytes = aggregate(local_ms, step_bytes * args.steps, dist_ok, device)
-    _, total_tokens = aggregate(local_ms, step_tokens * args.steps, dist_ok, device)
-    ms_per_step = total_ms / args.steps
+    local_ms, steps_timed = timed_graph_loop(plans, sets, args.steps, args.warmup, stream, dist_ok, sampler)
+    total_ms, total_bytes = aggregate(local_ms, step_bytes * steps_timed, dist_ok, device)
+    _, total_tokens = aggregate(local_ms, step_tokens * steps_timed, dist_ok, device)
+    ms_per_step = total_ms / steps_timed
     value = total_bytes / (total_ms * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
 
     # roofline of the fused kernel on this rank: algorithmic bytes per launch / mean launch duration
-    launch_ms = local_ms / (args.steps * launches_per_step)
+    launch_ms = local_ms / (steps_timed * launches_per_step)
     achieved = (step_bytes / launches_per_step) / (launch_ms * 1e-3) / 1e9
+    del sets
+    torch.cuda.empty_cache()
+    copy_gbs, _ = plain_traffic(stream, device, w.n_rows * w.d * 2, step_bytes // launches_per_step - w.n_rows * w.d * 2)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                 "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH, "peak_kind": "of " + peak_kind,
-                "kernel": "fused rotate-quantize, mean of the b=3 and b=4 launches",
-                "frac_of_8000_nominal": achieved / 8000.0}
+                "kernel": "fused rotate-quantize at d=4096, mean of the b=3 and b=4 launches",
+                "frac_of_8000_nominal": achieved / 8000.0,
+                "copy_same_size_gbs": copy_gbs,
+                "copy_same_size_note": "plain device copy moving the same %.1f MB per launch (read + written), same "
+                                       "graph-replay protocol; context beside `peak`, not a replacement" %
+                                       (step_bytes / launches_per_step / 1e6)}
+
+    # the metric's second width, d = 3584 (H_28 (x) H_128, groups of 128): its own timed loop and roofline object
+    w2 = synth.WORKLOADS["qwen3584"]
+    plans2 = [Plan(w2.d, w2.d_pad, w2.m, b, w2.group, w2.alpha) for b in w2.bits]
+    bytes2 = sum(algorithmic_bytes(w2.n_rows, w2.d, w2.d_pad, b, w2.group, 2) for b in w2.bits)
+    sets2 = build_sets(plans2, synth.make_host("qwen3584"), 8, device)
+    steps2 = max(8, args.steps // 2 // 8 * 8)
+    ms2, timed2 = timed_graph_loop(plans2, sets2, steps2, 3, stream, False)
+    del sets2
+    torch.cuda.empty_cache()
+    ach2 = bytes2 / (ms2 / timed2 * 1e-3) / 1e9
+    copy2, _ = plain_traffic(stream, device, w2.n_rows * w2.d * 2, bytes2 - w2.n_rows * w2.d * 2)
+    roofline_d3584 = {"bound": "hbm", "achieved": ach2, "peak": peak, "unit": "GB/s", "frac": ach2 / peak,
+                      "traffic": NCU_TRAFFIC_BYTES_PER_LAUNCH_D3584, "peak_kind": "of " + peak_kind,
+                      "kernel": "fused rotate-quantize at d=3584 (8192 tokens, b=3, groups of 128)",
+                      "us_per_launch": ms2 / timed2 * 1e3, "steps_timed": timed2,
+                      "mtokens_per_s": w2.n_rows / (ms2 / timed2) / 1e3,
+                      "frac_of_8000_nominal": ach2 / 8000.0, "copy_same_size_gbs": copy2}
 
     # ---- end to end through the public API with host buffers (copies inside the timed region)
     x_pin = x_base.pin_memory()
@@ -340,7 +432,7 @@ def main():
     for pl in plans:
         host_outs.append((torch.empty((w.n_rows, pl.info.code_bytes_per_row), dtype=torch.uint8).pin_memory(),
                           torch.empty((w.n_rows, pl.info.scales_per_row), dtype=torch.float32).pin_memory()))
-    e2e_steps = max(3, min(args.steps, 20))
+    e2e_steps = max(3, min(args.steps, 60))
 
     pipe = HostPipeline(plans, w.n_rows, device=device, chunks=args.e2e_chunks)
 
@@ -367,7 +459,7 @@ def main():
     # ---- context legs (outside the K timed steps)
     also = {}
     if not args.no_extras and rank == 0:
-        also = extras(device, stream, args, peak)
+        also = extras(device, stream, args, peak, sampler)
 
     sampler.stop()
     clocks = sampler.summary()
@@ -385,6 +477,7 @@ def main():
     if rank == 0:
         line = {
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "steps_timed": steps_timed,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": "%s: %d tokens x d=%d bf16, H_%d, b=3 and b=4 (one launch each per step), "
@@ -392,11 +485,13 @@ def main():
                        "replicas": world, "l2": "inputs rotate over %d buffer sets (%.0f MB > 4x L2); the b=3 and b=4 launches of a step read "
                        "different copies" %
                        (args.nsets, args.nsets * (step_bytes + w.n_rows * w.d * 2) / 1e6),
-                       "launch": "CUDA graph replay", "levels": "D=2^(b-1)-1"},
+                       "launch": "CUDA graph replay", "levels": "D=2^(b-1)-1",
+                       "timed_region": "the K steps repeated %d time(s): at least %.0f ms on the device" %
+                                       (steps_timed // args.steps, MIN_TIMED_MS)},
             "mtokens_per_s": total_tokens / (total_ms * 1e-3) / 1e6,
             "hbm_frac_of_measured": value / world / peak, "hbm_frac_of_8000": value / world / 8000.0,
-            "roofline": roofline, "cpu_baseline": cpu_baseline, "e2e": e2e, "clocks": clocks,
-            "gpu_launches": args.steps * launches_per_step, "also": also,
+            "roofline": roofline, "roofline_d3584": roofline_d3584, "cpu_baseline": cpu_baseline, "e2e": e2e, "clocks": clocks,
+            "gpu_launches": steps_timed * launches_per_step, "also": also,
         }
         print(json.dumps(line))
     if dist_ok:
@@ -412,6 +507,9 @@ def run_profile(spec, device):
     inverse = name.endswith("-inverse")               # e.g. llama4096-inverse: gbs_dequantize with inverse rotation
     if inverse:
         name = name[:-len("-inverse")]
+    plain_dq = name.endswith("-dequantize")           # e.g. llama4096-dequantize: gbs_dequantize, rotated domain
+    if plain_dq:
+        name = name[:-len("-dequantize")]
     w = synth.WORKLOADS["calib4096" if clip else name]
     n = int(rows) if rows else min(w.n_rows, 8192)
     bits = w.bits[0]
@@ -420,6 +518,7 @@ def run_profile(spec, device):
     outs = pl.alloc_outputs(n, device)
     err = torch.zeros(32, dtype=torch.float64, device=device)
     xhat = torch.empty((n, w.d), dtype=torch.bfloat16, device=device) if inverse else None
+    yhat = torch.empty((n, w.d_pad), dtype=torch.bfloat16, device=device) if plain_dq else None
     for _ in range(6):
         if clip:
             pl.clip_error(x, np.linspace(0.5, 1.0, 32), err_sum=err)
@@ -427,45 +526,69 @@ def run_profile(spec, device):
             pl.rotate_quantize(x, out=outs)
             if inverse:
                 pl.dequantize(outs[0], outs[1], inverse=True, out=xhat)
+            if plain_dq:
+                pl.dequantize(outs[0], outs[1], out=yhat)
     torch.cuda.synchronize()
     print(json.dumps({"profile": spec, "rows": n, "kernel_family": pl.info.variant, "status": pl.device_status()}))
 
 
-def extras(device, stream, args, peak):
+def extras(device, stream, args, peak, sampler=None):
     """Context figures for the other workloads / entry points (not part of the K timed steps)."""
     from paper_2504_13989_b200 import Plan, synth
     out = {}
 
-    def time_loop(fn, iters):
+    def time_loop(fn, iters, min_ms=20.0):
+        """Mean milliseconds per call of fn(i), i < iters, replayed from a CUDA graph (no host launch cost in
+        the figure) for at least min_ms."""
         with torch.cuda.stream(stream):
             for _ in range(3):
                 fn(0)
         stream.synchronize()
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        with torch.cuda.stream(stream):
-            a.record(stream)
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=stream):
             for i in range(iters):
                 fn(i)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        with torch.cuda.stream(stream):
+            g.replay()
+            a.record(stream)
+            g.replay()
             b.record(stream)
         stream.synchronize()
-        return a.elapsed_time(b) / iters
+        reps = max(1, int(np.ceil(min_ms / max(a.elapsed_time(b), 1e-6))))
+        with torch.cuda.stream(stream):
+            a.record(stream)
+            for _ in range(reps):
+                g.replay()
+            b.record(stream)
+        stream.synchronize()
+        return a.elapsed_time(b) / (iters * reps)
 
-    # per-bit figures of every rotate-quantize workload (graph replay, rotating buffer sets > 4x L2)
+    def rq_leg(name, bits, n_rows=None, xb=None, min_ms=20.0):
+        """One rotate-quantize workload: graph replay over buffer sets > 4x L2, at least min_ms timed."""
+        w = synth.WORKLOADS[name]
+        if xb is None:
+            xb = synth.make_host(name) if name != "kv128" else synth.make_device(name, device=str(device))
+        n = xb.shape[0]
+        pl = Plan(w.d, w.d_pad, w.m, bits, w.group, w.alpha)
+        nbytes = algorithmic_bytes(n, w.d, w.d_pad, bits, w.group, 2)
+        nsets = max(2, min(16, int(4 * 126e6 / (nbytes + 1)) + 1))
+        sets = build_sets([pl], xb, nsets, device)
+        ms, timed = timed_graph_loop([pl], sets, nsets, 3, stream, False, min_ms=min_ms)
+        ms /= timed
+        rec = {"us_per_launch": ms * 1e3, "gbs": nbytes / ms / 1e6, "frac_of_measured": nbytes / ms / 1e6 / peak,
+               "frac_of_8000": nbytes / ms / 1e6 / 8000.0, "mrows_per_s": n / ms / 1e3,
+               "kernel_family": pl.info.variant, "launches_timed": timed}
+        del sets, pl
+        torch.cuda.empty_cache()
+        return rec
+
+    # per-bit figures of every rotate-quantize workload
     for name in ("llama4096", "qwen3584", "mlp18944", "kv128"):
         w = synth.WORKLOADS[name]
         xb = synth.make_host(name) if name != "kv128" else synth.make_device(name, device=str(device))
         for b in w.bits:
-            pl = Plan(w.d, w.d_pad, w.m, b, w.group, w.alpha)
-            nbytes = algorithmic_bytes(w.n_rows, w.d, w.d_pad, b, w.group, 2)
-            nsets = max(2, min(16, int(4 * 126e6 / (nbytes + 1)) + 1))
-            sets = build_sets([pl], xb, nsets, device)
-            iters = max(2 * nsets, min(20 * nsets, int(20e-3 / (nbytes / 5e12)) // nsets * nsets))
-            ms = timed_graph_loop([pl], sets, iters, 3, stream, False) / iters
-            out["%s_b%d" % (name, b)] = {"us_per_launch": ms * 1e3, "gbs": nbytes / ms / 1e6,
-                                         "frac_of_measured": nbytes / ms / 1e6 / peak,
-                                         "frac_of_8000": nbytes / ms / 1e6 / 8000.0,
-                                         "mrows_per_s": w.n_rows / ms / 1e3, "kernel_family": pl.info.variant}
-            del sets, pl
+            out["%s_b%d" % (name, b)] = rq_leg(name, b, xb=xb)
         del xb
         torch.cuda.empty_cache()
     # the asymmetric KV quantizer (group 128 = one row) on the same KV tensor
@@ -474,59 +597,81 @@ def extras(device, stream, args, peak):
     pl = Plan(w.d, w.d_pad, w.m, 3, 128, 1.0, asymmetric=True)
     nbytes = w.n_rows * (w.d * 2 + w.d_pad * 3 // 8 + 8)
     sets = build_sets([pl], xb, 2, device)
-    ms = timed_graph_loop([pl], sets, 40, 3, stream, False) / 40
+    ms, timed = timed_graph_loop([pl], sets, 2, 3, stream, False, min_ms=20.0)
+    ms /= timed
     out["kv128_b3_asymmetric_group128"] = {"us_per_launch": ms * 1e3, "gbs": nbytes / ms / 1e6,
                                            "frac_of_measured": nbytes / ms / 1e6 / peak}
     del sets, pl, xb
     torch.cuda.empty_cache()
-    # steady state of the d=4096 kernel: 65536 tokens per launch (the batch tiled 16 times)
-    w = synth.WORKLOADS["llama4096"]
-    xb = synth.make_host("llama4096").repeat(16, 1)
-    pl = Plan(w.d, w.d_pad, w.m, 3, w.group, w.alpha)
-    nbytes = algorithmic_bytes(xb.shape[0], w.d, w.d_pad, 3, w.group, 2)
-    sets = build_sets([pl], xb, 2, device)
-    ms = timed_graph_loop([pl], sets, 20, 3, stream, False) / 20
-    out["llama4096_b3_65536rows"] = {"us_per_launch": ms * 1e3, "gbs": nbytes / ms / 1e6,
-                                     "frac_of_measured": nbytes / ms / 1e6 / peak}
-    del sets, pl, xb
-    torch.cuda.empty_cache()
-    # dequantize and clip-error on the headline workload
+    # steady state of the two widths of the metric: 65536 tokens per launch (the batch tiled)
+    for name, reps in (("llama4096", 16), ("qwen3584", 8)):
+        xb = synth.make_host(name).repeat(reps, 1)
+        out["%s_b3_65536rows" % name] = rq_leg(name, 3, xb=xb)
+        del xb
+    # dequantize on the headline workload, with the plain fill of the same output bytes beside it
     w = synth.WORKLOADS["llama4096"]
     x = synth.make_host("llama4096").to(device)
     pl = Plan(w.d, w.d_pad, w.m, 3, w.group, w.alpha)
     codes, scales, _ = pl.rotate_quantize(x)
-    yhat = torch.empty((w.n_rows, w.d_pad), dtype=torch.bfloat16, device=device)
-    ms = time_loop(lambda i: pl.dequantize(codes, scales, out=yhat, stream=stream), 50)
-    dq_bytes = w.n_rows * (w.d_pad * 3 // 8 + 4 + w.d_pad * 2)
-    out["dequantize_b3_bf16"] = {"us_per_launch": ms * 1e3, "gbs": dq_bytes / ms / 1e6}
-    xhat = torch.empty((w.n_rows, w.d), dtype=torch.bfloat16, device=device)
-    ms = time_loop(lambda i: pl.dequantize(codes, scales, inverse=True, out=xhat, stream=stream), 50)
+    yhat = [torch.empty((w.n_rows, w.d_pad), dtype=torch.bfloat16, device=device) for _ in range(16)]
+    ms = time_loop(lambda i: pl.dequantize(codes, scales, out=yhat[i % 16], stream=stream), 48)
+    dq_in, dq_out = w.n_rows * (w.d_pad * 3 // 8 + 4), w.n_rows * w.d_pad * 2
+    copy_gbs, fill_gbs = plain_traffic(stream, device, dq_in, dq_out)
+    fill_us = dq_out / fill_gbs / 1e3
+    out["dequantize_b3_bf16"] = {"us_per_launch": ms * 1e3, "gbs": (dq_in + dq_out) / ms / 1e6,
+                                 "frac_of_measured": (dq_in + dq_out) / ms / 1e6 / peak,
+                                 "fill_same_output_bytes_us": fill_us, "fill_same_output_bytes_gbs": fill_gbs,
+                                 "copy_same_size_gbs": copy_gbs,
+                                 "note": "write-bound: %.1f of its %.1f MB are output; a plain fill of that output alone "
+                                         "takes the time beside it" % (dq_out / 1e6, (dq_in + dq_out) / 1e6)}
+    xhat = yhat
+    ms = time_loop(lambda i: pl.dequantize(codes, scales, inverse=True, out=xhat[i % 16], stream=stream), 48)
     out["dequantize_inverse_rotate_b3_bf16"] = {"us_per_launch": ms * 1e3,
                                                 "gbs": w.n_rows * (w.d_pad * 3 // 8 + 4 + w.d * 2) / ms / 1e6}
-    del xhat
-    # clip-ratio scoring, K = 32, on a 32768-token sample of one calibration layer (262144 tokens x 4096)
-    del x, codes, scales, yhat
+    del xhat, x, codes, scales, yhat
+    torch.cuda.empty_cache()
+    # clip-ratio scoring at the calibration size: K = 32 candidates over one full layer of 128 sequences x 2048
+    # tokens x d = 4096 per launch, for each of 32 layers (its own seeded tensor each: seed 5 + layer)
     wc = synth.WORKLOADS["calib4096"]
-    xc = synth.make_device("calib4096", 32768, device=str(device))
     alphas = np.linspace(0.5, 1.0, 32)
-    err = torch.zeros(32, dtype=torch.float64, device=device)
-    ms = time_loop(lambda i: pl.clip_error(xc, alphas, err_sum=err, stream=stream), 5)
-    evals = 32768 * wc.d_pad * 32
-    sm_clock_hz = 1.965e9
-    alu_peak = 148 * 128 * sm_clock_hz                  # fp32 lanes x clock: lane-operations per second
-    out["clip_error_K32"] = {"us_per_launch": ms * 1e3, "gevals_per_s": evals / ms / 1e6,
-                             "ms_per_layer_262144_tokens": ms * 8, "mtokens_per_s": 32768 / ms / 1e3,
+    layer_ms = []
+    mark = sampler.mark() if sampler else 0
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for layer in range(32):
+        xc = synth.make_device("calib4096", wc.n_rows, seed=wc.seed + layer, device=str(device))
+        err = torch.zeros(32, dtype=torch.float64, device=device)
+        if layer == 0:
+            pl.clip_error(xc[:4096], alphas, err_sum=err, stream=stream)          # warm-up launch
+            err.zero_()
+        stream.synchronize()
+        torch.cuda.synchronize()
+        with torch.cuda.stream(stream):
+            a.record(stream)
+            pl.clip_error(xc, alphas, err_sum=err, stream=stream)
+            b.record(stream)
+        stream.synchronize()
+        layer_ms.append(a.elapsed_time(b))
+        if layer == 31:
+            t0 = time.perf_counter()
+            res = pl.search_clip_ratio(xc, 1.0 / 64, stream=stream)
+            dt = time.perf_counter() - t0
+        del xc, err
+    sm_mhz = (sampler.median_mhz_since(mark) if sampler else None) or 1965.0
+    ms = statistics.median(layer_ms)
+    evals = wc.n_rows * wc.d_pad * 32
+    alu_peak = 148 * 128 * sm_mhz * 1e6                   # fp32 lanes x sampled SM clock: lane-operations per second
+    out["clip_error_K32"] = {"ms_per_layer_262144_tokens": ms, "ms_32_layers": sum(layer_ms),
+                             "ms_per_layer_min_max": [min(layer_ms), max(layer_ms)],
+                             "gevals_per_s": evals / ms / 1e6, "mtokens_per_s": wc.n_rows / ms / 1e3,
+                             "hbm_gbs": wc.n_rows * wc.d * 2 / ms / 1e6,
                              "roofline": {"bound": "alu", "unit": "Glane-op/s", "achieved": 5 * evals / ms / 1e6,
                                           "peak": alu_peak / 1e9, "frac": 5 * evals / ms / 1e6 / (alu_peak / 1e9),
+                                          "sm_mhz_sampled": sm_mhz,
                                           "note": "5 fp32 operations per value and candidate; peak = 148 SMs x 128 "
-                                                  "lanes x 1.965 GHz"}}
-    # Algorithm 1's bracket search on the same sample (eps = 1/64): rounds of <= 31 probes, blocking
-    t0 = time.perf_counter()
-    res = pl.search_clip_ratio(xc, 1.0 / 64, stream=stream)
-    dt = time.perf_counter() - t0
+                                                  "lanes x the SM clock sampled during these launches"}}
+    # Algorithm 1's bracket search on the last layer's tensor (eps = 1/64): rounds of <= 31 probes, blocking
     out["search_clip_ratio_eps_1_64"] = {"alpha": res.alpha, "iterations": res.iterations, "rounds": res.rounds,
-                                         "evaluations": res.evaluations, "wall_ms": dt * 1e3,
-                                         "wall_ms_per_layer_262144_tokens": dt * 8e3}
+                                         "evaluations": res.evaluations, "wall_ms_per_layer_262144_tokens": dt * 1e3}
     return out
 
 

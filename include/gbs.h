@@ -269,6 +269,61 @@ int gbs_search_clip_ratio(const gbs_plan_t* plan, const void* x, int x_dtype, in
                           void* cuda_stream);
 
 /*
+ * State of one projection's search (Algorithm 1), a handful of numbers: plain data that may be copied, stored
+ * and handed back later to resume the search where it stopped (gbs_search_state_init gives the algorithm's
+ * start a = 0, b = 1, m = 1/2).
+ */
+typedef struct gbs_search_state {
+    double a, b, m;     /* the bracket and the kept point                                        */
+    double f_m;         /* the objective at m (valid once have_fm is set)                       */
+    int iteration;      /* passes through the loop body so far                                   */
+    int evaluations;    /* objective values consumed so far                                      */
+    int have_fm;        /* f(m) of the start point has been evaluated                            */
+    int done;           /* b - a <= eps was reached (set by the search calls)                    */
+} gbs_search_state_t;
+
+int gbs_search_state_init(gbs_search_state_t* state);
+
+/*
+ * Algorithm 1's loop for one projection with the CALLER's objective, e.g. the perplexity the paper minimises
+ * (Sections 3.1, 4.1): f(alpha, ctx) is called once per pass, in the order of the algorithm as printed, plus
+ * once for the start point.  Runs until b - a <= eps, or for at most max_iterations passes when that is > 0;
+ * `state` (in/out) then resumes.  Host only: touches no device.
+ */
+typedef double (*gbs_objective_fn)(float alpha, void* ctx);
+int gbs_search_clip_ratio_fn(gbs_objective_fn f, void* ctx, float eps, gbs_search_state_t* state,
+                             int max_iterations);
+
+/*
+ * Algorithm 1's loop for n_tasks projections at once with the quantization error as objective.  The paper walks
+ * the projections one after the other because its objective, the model's perplexity, couples them; the
+ * quantization error of one projection's input does not depend on the others, so here every round scores the
+ * pending probes (the next five iterations' decision tree, at most 31 clip ratios, as in gbs_search_clip_ratio)
+ * of EVERY unfinished projection, one gbs_clip_error launch per projection enqueued back to back, and waits once
+ * per round.  Each projection visits exactly the states its own gbs_search_clip_ratio call would visit.
+ *   tasks       host array: plan, rows (device), dtype, n_rows >= 1 and row stride of each projection; all plans on
+ *               one device; n_tasks 1 .. GBS_MAX_SEARCH_TASKS
+ *   eps         0 < eps < 1
+ *   states      host array, in/out: start from gbs_search_state_init, or resume earlier states
+ *   max_rounds  0 = run until every projection is done; otherwise stop after that many rounds (resumable)
+ *   work_dev    device, n_tasks * GBS_MAX_CANDIDATES doubles, 8-byte aligned, overwritten
+ *   alphas_out  NULL, or host array of n_tasks floats: the list L of Algorithm 1 (the kept point of each projection)
+ *   rounds_out  NULL, or the number of rounds this call ran
+ * BLOCKS: once per round the call waits for `cuda_stream`.
+ */
+#define GBS_MAX_SEARCH_TASKS 4096
+typedef struct gbs_search_task {
+    const gbs_plan_t* plan;
+    const void* x;
+    int x_dtype;
+    int64_t n_rows;
+    int64_t x_row_stride;
+} gbs_search_task_t;
+int gbs_search_clip_ratio_batch(const gbs_search_task_t* tasks, int n_tasks, float eps, gbs_search_state_t* states,
+                                int max_rounds, double* work_dev, float* alphas_out, int* rounds_out,
+                                void* cuda_stream);
+
+/*
  * Host-only helper: write the m x m sign matrix H_m (row-major, +1 / -1) the plans use
  * (Algorithm 2).  `out_host` must hold m*m bytes.  Needs no device.
  */

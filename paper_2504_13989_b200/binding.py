@@ -29,7 +29,8 @@ GBS_MAX_CANDIDATES = 64
 GBS_PLAN_ASYMMETRIC = 1
 EXPORTS = ("gbs_plan_create", "gbs_plan_create_ex", "gbs_plan_destroy", "gbs_plan_info", "gbs_plan_device_status", "gbs_rotate_quantize",
            "gbs_rotate_quantize_static", "gbs_static_device_status", "gbs_dequantize", "gbs_clip_error",
-           "gbs_search_clip_ratio", "gbs_hadamard_m", "gbs_status_string", "gbs_selftest_wait_expiry")
+           "gbs_search_clip_ratio", "gbs_search_state_init", "gbs_search_clip_ratio_fn", "gbs_search_clip_ratio_batch",
+           "gbs_hadamard_m", "gbs_status_string", "gbs_selftest_wait_expiry")
 GBS_STATIC_MAX_D_PAD = 4096
 
 
@@ -52,6 +53,21 @@ class SearchResult(ctypes.Structure):
     _fields_ = [("alpha", ctypes.c_float), ("a", ctypes.c_float), ("b", ctypes.c_float), ("err", ctypes.c_double),
                 ("iterations", ctypes.c_int), ("evaluations", ctypes.c_int), ("rounds", ctypes.c_int)]
 
+
+class SearchState(ctypes.Structure):
+    """gbs_search_state_t: the resumable state of one projection's search (plain data; bytes(state) stores it)."""
+    _fields_ = [("a", ctypes.c_double), ("b", ctypes.c_double), ("m", ctypes.c_double), ("f_m", ctypes.c_double),
+                ("iteration", ctypes.c_int), ("evaluations", ctypes.c_int), ("have_fm", ctypes.c_int),
+                ("done", ctypes.c_int)]
+
+
+class SearchTask(ctypes.Structure):
+    _fields_ = [("plan", ctypes.c_void_p), ("x", ctypes.c_void_p), ("x_dtype", ctypes.c_int),
+                ("n_rows", ctypes.c_int64), ("x_row_stride", ctypes.c_int64)]
+
+
+OBJECTIVE_FN = ctypes.CFUNCTYPE(ctypes.c_double, ctypes.c_float, ctypes.c_void_p)
+GBS_MAX_SEARCH_TASKS = 4096
 
 _lib = None
 
@@ -89,6 +105,14 @@ def lib() -> ctypes.CDLL:
         L.gbs_clip_error.restype = i32
         L.gbs_search_clip_ratio.argtypes = [vp, vp, i32, i64, i64, ctypes.c_float, vp, ctypes.POINTER(SearchResult), vp]
         L.gbs_search_clip_ratio.restype = i32
+        L.gbs_search_state_init.argtypes = [ctypes.POINTER(SearchState)]
+        L.gbs_search_state_init.restype = i32
+        L.gbs_search_clip_ratio_fn.argtypes = [OBJECTIVE_FN, vp, ctypes.c_float, ctypes.POINTER(SearchState), i32]
+        L.gbs_search_clip_ratio_fn.restype = i32
+        L.gbs_search_clip_ratio_batch.argtypes = [ctypes.POINTER(SearchTask), i32, ctypes.c_float,
+                                                  ctypes.POINTER(SearchState), i32, vp, ctypes.POINTER(ctypes.c_float),
+                                                  ctypes.POINTER(i32), vp]
+        L.gbs_search_clip_ratio_batch.restype = i32
         L.gbs_hadamard_m.argtypes = [i32, vp]
         L.gbs_hadamard_m.restype = i32
         L.gbs_status_string.argtypes = [i32]
@@ -283,6 +307,51 @@ def gbs_search_clip_ratio(plan: int, x: torch.Tensor, eps: float, work: torch.Te
                                        float(eps), work.data_ptr(), ctypes.byref(res), _stream_ptr(stream)),
            "gbs_search_clip_ratio")
     return res
+
+
+def gbs_search_state_init() -> SearchState:
+    st = SearchState()
+    _check(lib().gbs_search_state_init(ctypes.byref(st)), "gbs_search_state_init")
+    return st
+
+
+def gbs_search_clip_ratio_fn(objective, eps: float, state: SearchState | None = None,
+                             max_iterations: int = 0) -> SearchState:
+    """Algorithm 1's loop for one projection with a Python objective `objective(alpha) -> float` (e.g. a model's
+    perplexity).  Host only.  Returns the state (done = 1 when b - a <= eps); pass it back to resume."""
+    st = state if state is not None else gbs_search_state_init()
+    cb = OBJECTIVE_FN(lambda alpha, _ctx: float(objective(float(alpha))))
+    _check(lib().gbs_search_clip_ratio_fn(cb, None, float(eps), ctypes.byref(st), int(max_iterations)),
+           "gbs_search_clip_ratio_fn")
+    return st
+
+
+def gbs_search_clip_ratio_batch(plans, xs, eps: float, states=None, max_rounds: int = 0, work: torch.Tensor | None = None,
+                                stream=None):
+    """Algorithm 1's loop for several projections at once (plan i scores rows xs[i]); one wait per round.
+    Returns (alphas: the list L, states, rounds).  `plans` are plan handles (ints)."""
+    n = len(plans)
+    if n < 1 or n != len(xs):
+        raise ValueError("gbs_search_clip_ratio_batch: one tensor per plan")
+    tasks = (SearchTask * n)()
+    keep = []
+    for i, (pl, x) in enumerate(zip(plans, xs)):
+        info = gbs_plan_info(pl)
+        xv, n_rows, stride = _rows_view(x, info.d)
+        keep.append(xv)
+        tasks[i] = SearchTask(pl, xv.data_ptr(), _dtype_code(xv), n_rows, stride)
+    sts = (SearchState * n)()
+    for i in range(n):
+        sts[i] = states[i] if states is not None else gbs_search_state_init()
+    if work is None:
+        work = torch.empty(n * GBS_MAX_CANDIDATES, dtype=torch.float64, device=keep[0].device)
+    _check_buffer("work", work, keep[0], torch.float64, n * GBS_MAX_CANDIDATES)
+    alphas = (ctypes.c_float * n)()
+    rounds = ctypes.c_int(0)
+    _check(lib().gbs_search_clip_ratio_batch(tasks, n, float(eps), sts, int(max_rounds), work.data_ptr(), alphas,
+                                             ctypes.byref(rounds), _stream_ptr(stream)),
+           "gbs_search_clip_ratio_batch")
+    return [float(a) for a in alphas], [sts[i] for i in range(n)], rounds.value
 
 
 # ----------------------------------------------------------------------------------------------

@@ -503,6 +503,117 @@ __global__ void __launch_bounds__(NT) k_dequantize_plain(int d_pad, int G, int s
     }
 }
 
+// The same for rows whose width is a multiple of 256 (or is 128), warp-cooperative: one warp item is 256 consecutive
+// codes of the flat code stream (96 or 128 bytes, read as coalesced 32-bit words) and 512 or 1024 contiguous output
+// bytes, and every store instruction of the warp covers 512 contiguous bytes.  Lane l turns codes [8l, 8l+8) of the
+// item into bf16, or codes [4l, 4l+4) and [128+4l, 128+4l+4) into fp32.  The kernel is bound by the device's write
+// bandwidth (the output is 5 to 11 times the size of the input).
+template <typename OutT, int BITS>
+__global__ void __launch_bounds__(NT) k_dequantize_stream(int d_pad, int glog, int spr, int asym, long long total_codes,
+                                                          const unsigned* __restrict__ words,
+                                                          const float* __restrict__ scales, OutT* __restrict__ out)
+{
+    constexpr bool WIDE = sizeof(OutT) == 4;        // fp32 output: two groups of four codes per lane
+    constexpr int PER = WIDE ? 4 : 8;               // codes per lane and store
+    constexpr int NST = WIDE ? 2 : 1;               // groups (= stores) per lane and item
+    constexpr int UNR = 4;                          // items per warp and pass: all their loads are issued first
+    const int lane = threadIdx.x & 31;
+    const long long n_items = (total_codes + 255) >> 8;
+    const long long last_word = (total_codes * BITS >> 5) - 1;
+    const long long stride = (long long)gridDim.x * (NT / 32) * UNR;
+    long long item0 = ((long long)blockIdx.x * (NT / 32) + (threadIdx.x >> 5)) * UNR;
+    // position of the pass's first code, kept up to date without a division per item
+    long long row = (item0 << 8) / d_pad;
+    int col = (int)((item0 << 8) - row * d_pad);
+    const long long row_step = (stride << 8) / d_pad;
+    const int col_step = (int)((stride << 8) - row_step * d_pad);
+    // per-lane constants: where this lane's group starts inside an item (codes, words, bit shift), and whether its
+    // field runs into a second word
+    int c_of[NST], w_of[NST], sh_of[NST];
+    bool two[NST];
+#pragma unroll
+    for (int h = 0; h < NST; ++h) {
+        c_of[h] = WIDE ? 128 * h + 4 * lane : 8 * lane;
+        w_of[h] = (c_of[h] * BITS) >> 5;
+        sh_of[h] = (c_of[h] * BITS) & 31;
+        two[h] = sh_of[h] + PER * BITS > 32;
+    }
+    const int amul = asym ? 2 : 1;
+    for (; item0 < n_items; item0 += stride) {
+        // every item of the pass complete and not the buffer's last: no bound checks on the loads and stores
+        const bool inner = item0 + UNR < n_items;
+        const unsigned* wp = words + item0 * (8 * BITS);
+        OutT* op = out + (item0 << 8);
+        unsigned field[UNR][NST];
+        float delta[UNR][NST], zero[UNR][NST];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+#pragma unroll
+            for (int h = 0; h < NST; ++h) {
+                field[u][h] = 0u; delta[u][h] = 0.f; zero[u][h] = 0.f;
+                const int widx = u * (8 * BITS) + w_of[h];
+                if (inner || ((item0 + u) << 8) + c_of[h] < total_codes) {
+                    const unsigned lo = __ldg(wp + widx);
+                    unsigned hi = 0u;
+                    if (two[h] && (inner || item0 * (8 * BITS) + widx < last_word)) hi = __ldg(wp + widx + 1);
+                    field[u][h] = __funnelshift_r(lo, hi, sh_of[h]);
+                    // the group's row and scale (rows of 128 codes: an item spans two rows)
+                    int cc = col + 256 * u + c_of[h];
+                    long long r = row;
+                    while (cc >= d_pad) { cc -= d_pad; ++r; }
+                    const float* sp = scales + (r * spr + (cc >> glog)) * amul;
+                    delta[u][h] = __ldg(sp);
+                    if (asym) zero[u][h] = __ldg(sp + 1);
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+#pragma unroll
+            for (int h = 0; h < NST; ++h) {
+                if (!inner && !(((item0 + u) << 8) + c_of[h] < total_codes)) continue;
+                // Fields -> floats without integer conversions: the group's fields are spread to one per nibble
+                // (3-bit fields by three mask-and-shift steps), symmetric codes turned into offset binary by one XOR
+                // of every sign bit, each nibble dropped into the mantissa of 2^23 by a byte permute, and the
+                // offset removed by an exact subtraction:  2^23 + (q + off)  -  (2^23 + off)  =  q.
+                unsigned nib = field[u][h];
+                if (BITS == 3) {
+                    nib = (nib & 0x00000fffu) | ((nib & 0x00fff000u) << 4);       // 12 bits per half-word
+                    nib = (nib & 0x003f003fu) | ((nib & 0x0fc00fc0u) << 2);       // 6 bits per byte
+                    nib = (nib & 0x07070707u) | ((nib & 0x38383838u) << 1);       // 3 bits per nibble
+                }
+                constexpr unsigned SIGNS = BITS == 3 ? 0x44444444u : 0x88888888u;
+                constexpr float OFF = BITS == 3 ? 4.f : 8.f;
+                if (!asym) nib ^= SIGNS;
+                const unsigned even = nib & 0x0f0f0f0fu, odd = (nib >> 4) & 0x0f0f0f0fu;
+                const float bias = 8388608.f + (asym ? 0.f : OFF);
+                float v[PER];
+#pragma unroll
+                for (int e = 0; e < PER; ++e) {
+                    // byte e/2 of the even or odd word, below the three upper bytes of 2^23 (0x4B000000)
+                    const unsigned fb = __byte_perm((e & 1) ? odd : even, 0x4B000000u, 0x7440u + (unsigned)(e >> 1));
+                    v[e] = fmaf(__uint_as_float(fb) - bias, delta[u][h], zero[u][h]);
+                }
+                OutT* dst = op + 256 * u + c_of[h];
+                if (WIDE) {
+                    *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+                } else {
+                    unsigned o[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+                        o[e] = *reinterpret_cast<unsigned*>(&b2);
+                    }
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+                }
+            }
+        }
+        row += row_step;
+        col += col_step;
+        if (col >= d_pad) { col -= d_pad; ++row; }
+    }
+}
+
 // xhat = (H^T yhat / sqrt(d'))[0:d]: same shared-memory machinery with the transposed H_m.
 template <typename OutT, int BITS, bool WIDE>
 __global__ void __launch_bounds__(NT) k_dequantize_inverse(GenericParams P, const unsigned char* __restrict__ codes,
@@ -685,6 +796,28 @@ int gbs_generic_dequantize(const gbs_plan* p, const void* codes, const float* sc
     GenericParams P;
     fill_params(p, P, n_rows, 0, inverse != 0);
     cudaError_t e = cudaSuccess;
+    if (!inverse && (P.d_pad % 256 == 0 || P.d_pad == 128)) {
+        // warp-cooperative streaming form; a quantization group (a power of two >= 8) never splits a lane's codes
+        const long long total = (long long)n_rows * P.d_pad;
+        const long long items = (total + 255) >> 8;
+        long long blocks = (items + (NT / 32) * 4 - 1) / ((NT / 32) * 4);        // four items per warp and pass
+        // the kernel is bound by the latency of its (small) loads under the pressure of its own stores, i.e. by the
+        // bytes in flight: measured best with four resident blocks per SM for 2-byte outputs, eight for 4-byte ones
+        const long long cap = (long long)p->sm_count * (out_dtype == GBS_DTYPE_F32 ? 8 : 4);
+        const int grid = (int)(blocks < cap ? blocks : cap);
+        int glog = 31;                               // one scale per row: every column maps to scale 0
+        if (p->group) { glog = 0; while ((1 << glog) < p->group) ++glog; }
+#define LAUNCH_DS(T, B)                                                                            \
+    do {                                                                                           \
+        k_dequantize_stream<T, B><<<grid, NT, 0, stream>>>(P.d_pad, glog, P.spr, P.asym, total,     \
+                                                           (const unsigned*)codes, scales, (T*)out); \
+        e = cudaGetLastError();                                                                    \
+    } while (0)
+        if (out_dtype == GBS_DTYPE_F32) { if (p->bits == 3) LAUNCH_DS(float, 3); else LAUNCH_DS(float, 4); }
+        else { if (p->bits == 3) LAUNCH_DS(__nv_bfloat16, 3); else LAUNCH_DS(__nv_bfloat16, 4); }
+#undef LAUNCH_DS
+        return (int)e;
+    }
     if (!inverse) {
         const long long n_chunks = (long long)n_rows * P.chunks;
         long long blocks = (n_chunks + NT - 1) / NT;

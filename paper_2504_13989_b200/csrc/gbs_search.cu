@@ -11,6 +11,8 @@
 #include <math.h>
 #include <string.h>
 
+#include <new>
+
 #include "gbs_internal.h"
 
 namespace {
@@ -59,58 +61,163 @@ int find(const float* alphas, int K, float v)
     return -1;
 }
 
+// Algorithm 1's start: a = 0, b = 1, m = 1/2, nothing evaluated yet.
+void reset(gbs_search_state_t* st)
+{
+    st->a = 0.0; st->b = 1.0; st->m = 0.5; st->f_m = 0.0;
+    st->iteration = 0; st->evaluations = 0; st->have_fm = 0; st->done = 0;
+}
+
+State load(const gbs_search_state_t& st) { return State{st.a, st.b, st.m, st.iteration}; }
+
+bool state_valid(const gbs_search_state_t& st)
+{
+    return st.a >= 0.0 && st.b <= 1.0 && st.a <= st.m && st.m <= st.b && st.iteration >= 0 && st.evaluations >= 0;
+}
+
+// One pass through the loop body with the objective value f_x of this state's probe.
+void advance(gbs_search_state_t* st, double x, double f_x)
+{
+    const State s = load(*st);
+    const bool improved = f_x < st->f_m;
+    const State n = next_state(s, x, improved);
+    st->a = n.a; st->b = n.b; st->m = n.m; st->iteration = n.iteration;
+    if (improved) st->f_m = f_x;
+    st->evaluations += 1;
+}
+
 }  // namespace
+
+extern "C" int gbs_search_state_init(gbs_search_state_t* state)
+{
+    if (!state) return GBS_ERR_INVALID_ARG;
+    reset(state);
+    return GBS_OK;
+}
+
+// Algorithm 1's loop for one projection with the caller's objective (the paper's is perplexity): one evaluation
+// per pass, exactly in the printed order; stops at b - a <= eps or after max_iterations passes (> 0), leaving the
+// state resumable.
+extern "C" int gbs_search_clip_ratio_fn(gbs_objective_fn f, void* ctx, float eps, gbs_search_state_t* st,
+                                        int max_iterations)
+{
+    if (!f || !st) return GBS_ERR_INVALID_ARG;
+    if (!(eps > 0.f) || !(eps < 1.f) || max_iterations < 0) return GBS_ERR_INVALID_ARG;
+    if (!state_valid(*st)) return GBS_ERR_INVALID_ARG;
+    if (!st->have_fm) {
+        st->f_m = f((float)st->m, ctx);
+        st->have_fm = 1;
+        st->evaluations += 1;
+    }
+    int passes = 0;
+    while (st->b - st->a > (double)eps && (max_iterations == 0 || passes < max_iterations)) {
+        const double x = probe_of(load(*st));
+        advance(st, x, f((float)x, ctx));
+        ++passes;
+    }
+    st->done = !(st->b - st->a > (double)eps);
+    return GBS_OK;
+}
+
+// Algorithm 1's loop for P projections at once, with the quantization error as the objective.  With that
+// objective the projections do not depend on one another (the paper's perplexity couples them, which is why it
+// walks them one after the other), so every round scores, for EVERY unfinished projection, the probes of its next
+// five iterations' decision tree -- one gbs_clip_error launch per projection, enqueued back to back -- and the
+// host waits ONCE per round for all the sums.
+extern "C" int gbs_search_clip_ratio_batch(const gbs_search_task_t* tasks, int n_tasks, float eps,
+                                           gbs_search_state_t* states, int max_rounds, double* work_dev,
+                                           float* alphas_out, int* rounds_out, void* cuda_stream)
+{
+    if (!tasks || !states || !work_dev || n_tasks < 1 || n_tasks > GBS_MAX_SEARCH_TASKS) return GBS_ERR_INVALID_ARG;
+    if (!(eps > 0.f) || !(eps < 1.f) || max_rounds < 0) return GBS_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(work_dev) & 7u) return GBS_ERR_ALIGNMENT;
+    int device = -1;
+    for (int i = 0; i < n_tasks; ++i) {
+        if (!tasks[i].plan || tasks[i].n_rows <= 0 || !state_valid(states[i])) return GBS_ERR_INVALID_ARG;
+        if (i == 0) device = tasks[i].plan->device;
+        else if (tasks[i].plan->device != device) return GBS_ERR_INVALID_ARG;     // one stream, one device
+        states[i].done = !(states[i].b - states[i].a > (double)eps);
+    }
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    gbs_device_guard guard;
+    if (guard.enter(device) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
+
+    float* alphas = new (std::nothrow) float[(size_t)n_tasks * GBS_MAX_CANDIDATES];
+    double* sums = new (std::nothrow) double[(size_t)n_tasks * GBS_MAX_CANDIDATES];
+    int* K = new (std::nothrow) int[n_tasks];
+    int rc = (alphas && sums && K) ? GBS_OK : GBS_ERR_ALLOC;
+    int rounds = 0;
+    while (rc == GBS_OK && (max_rounds == 0 || rounds < max_rounds)) {
+        int pending = 0;
+        for (int i = 0; i < n_tasks; ++i) pending += states[i].done ? 0 : 1;
+        if (!pending) break;
+        if (cudaMemsetAsync(work_dev, 0, sizeof(double) * GBS_MAX_CANDIDATES * (size_t)n_tasks, stream) != cudaSuccess) {
+            cudaGetLastError();
+            rc = GBS_ERR_CUDA;
+            break;
+        }
+        for (int i = 0; i < n_tasks && rc == GBS_OK; ++i) {
+            K[i] = 0;
+            if (states[i].done) continue;
+            float* al = alphas + (size_t)i * GBS_MAX_CANDIDATES;
+            if (!states[i].have_fm) al[K[i]++] = (float)states[i].m;
+            collect(load(states[i]), (double)eps, DEPTH, al, &K[i]);
+            rc = gbs_clip_error(tasks[i].plan, tasks[i].x, tasks[i].x_dtype, tasks[i].n_rows, tasks[i].x_row_stride, al,
+                                K[i], work_dev + (size_t)i * GBS_MAX_CANDIDATES, nullptr, cuda_stream);
+        }
+        if (rc != GBS_OK) break;
+        if (cudaMemcpyAsync(sums, work_dev, sizeof(double) * GBS_MAX_CANDIDATES * (size_t)n_tasks, cudaMemcpyDeviceToHost,
+                            stream) != cudaSuccess ||
+            cudaStreamSynchronize(stream) != cudaSuccess) {
+            cudaGetLastError();
+            rc = GBS_ERR_CUDA;
+            break;
+        }
+        ++rounds;
+        for (int i = 0; i < n_tasks; ++i) {
+            if (states[i].done) continue;
+            const float* al = alphas + (size_t)i * GBS_MAX_CANDIDATES;
+            const double* sm = sums + (size_t)i * GBS_MAX_CANDIDATES;
+            gbs_search_state_t* st = &states[i];
+            if (!st->have_fm) { st->f_m = sm[0]; st->have_fm = 1; st->evaluations += 1; }
+            // walk the tree along the outcomes that occurred
+            for (int level = 0; level < DEPTH && st->b - st->a > (double)eps; ++level) {
+                const double xp = probe_of(load(*st));
+                const int j = find(al, K[i], (float)xp);
+                if (j < 0) break;
+                advance(st, xp, sm[j]);
+            }
+            st->done = !(st->b - st->a > (double)eps);
+        }
+    }
+    delete[] alphas;
+    delete[] sums;
+    delete[] K;
+    if (rc != GBS_OK) return rc;
+    if (alphas_out)
+        for (int i = 0; i < n_tasks; ++i) alphas_out[i] = (float)states[i].m;     // the list L of Algorithm 1
+    if (rounds_out) *rounds_out = rounds;
+    return GBS_OK;
+}
 
 extern "C" int gbs_search_clip_ratio(const gbs_plan_t* plan, const void* x, int x_dtype, int64_t n_rows,
                                      int64_t x_row_stride, float eps, double* work_dev,
                                      gbs_search_result_t* out_host, void* cuda_stream)
 {
     if (!plan || !out_host || !work_dev) return GBS_ERR_INVALID_ARG;
-    if (!(eps > 0.f) || !(eps < 1.f)) return GBS_ERR_INVALID_ARG;
     if (n_rows <= 0) return GBS_ERR_INVALID_ARG;
-    if (reinterpret_cast<uintptr_t>(work_dev) & 7u) return GBS_ERR_ALIGNMENT;
-    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    gbs_device_guard guard;                       // the copies below belong to the plan's device, like its launches
-    if (guard.enter(plan->device) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
-
-    State s = {0.0, 1.0, 0.5, 0};
-    double f_m = 0.0;
-    bool have_fm = false;
-    int evaluations = 0, rounds = 0;
-    float alphas[GBS_MAX_CANDIDATES];
-    double sums[GBS_MAX_CANDIDATES];
-    while (s.b - s.a > (double)eps) {
-        int K = 0;
-        if (!have_fm) alphas[K++] = (float)s.m;
-        collect(s, (double)eps, DEPTH, alphas, &K);
-        if (cudaMemsetAsync(work_dev, 0, sizeof(double) * K, stream) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
-        const int rc = gbs_clip_error(plan, x, x_dtype, n_rows, x_row_stride, alphas, K, work_dev, nullptr, cuda_stream);
-        if (rc != GBS_OK) return rc;
-        if (cudaMemcpyAsync(sums, work_dev, sizeof(double) * K, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-            cudaStreamSynchronize(stream) != cudaSuccess) {
-            cudaGetLastError();
-            return GBS_ERR_CUDA;
-        }
-        ++rounds;
-        if (!have_fm) { f_m = sums[0]; have_fm = true; ++evaluations; }
-        // walk the tree along the outcomes that occurred
-        for (int level = 0; level < DEPTH && s.b - s.a > (double)eps; ++level) {
-            const double xp = probe_of(s);
-            const int i = find(alphas, K, (float)xp);
-            if (i < 0) break;                         // not scored in this round (cannot happen below 64 probes)
-            const double f_x = sums[i];
-            ++evaluations;
-            const bool improved = f_x < f_m;
-            s = next_state(s, xp, improved);
-            if (improved) f_m = f_x;
-        }
-    }
-    out_host->alpha = (float)s.m;
-    out_host->a = (float)s.a;
-    out_host->b = (float)s.b;
-    out_host->err = f_m;
-    out_host->iterations = s.iteration;
-    out_host->evaluations = evaluations;
+    gbs_search_task_t task = {plan, x, x_dtype, n_rows, x_row_stride};
+    gbs_search_state_t st;
+    reset(&st);
+    int rounds = 0;
+    const int rc = gbs_search_clip_ratio_batch(&task, 1, eps, &st, 0, work_dev, nullptr, &rounds, cuda_stream);
+    if (rc != GBS_OK) return rc;
+    out_host->alpha = (float)st.m;
+    out_host->a = (float)st.a;
+    out_host->b = (float)st.b;
+    out_host->err = st.f_m;
+    out_host->iterations = st.iteration;
+    out_host->evaluations = st.evaluations;
     out_host->rounds = rounds;
     return GBS_OK;
 }

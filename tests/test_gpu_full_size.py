@@ -60,18 +60,21 @@ def test_kv_tensor_sampled_rows_and_code_range():
         assert bool((scales >= 0).all())
 
 
-def test_calibration_layer_clip_error_sampled_rows():
-    """One calibration layer's scoring call at K = 32 on 65 536 tokens of the layer; per-row errors of
-    sampled rows against the oracle, and the fp64 totals against the sum of the kernel's own rows."""
+@pytest.mark.parametrize("layer", [0, 31])
+def test_calibration_layer_clip_error_sampled_rows(layer):
+    """One whole calibration layer (128 sequences x 2048 tokens = 262 144 rows of d = 4096, seed 5 + layer) in
+    ONE scoring call at K = 32, the launch configuration the benchmark times; per-row errors of sampled rows
+    against the oracle, and the fp64 totals against the sum of the kernel's own rows."""
     w = synth.WORKLOADS["calib4096"]
-    n = 65536
-    x = synth.make_device("calib4096", n, device=DEV)
+    n = w.n_rows
+    assert n == 128 * 2048
+    x = synth.make_device("calib4096", n, seed=w.seed + layer, device=DEV)
     alphas = np.linspace(0.5, 1.0, 32)
     with Plan(w.d, w.d_pad, w.m, 3, w.group, w.alpha) as plan:
         err, rows = plan.clip_error(x, alphas, want_rows=True)
         torch.cuda.synchronize()
         assert plan.device_status() == 0
-        idx = torch.arange(0, n, 331)
+        idx = torch.arange(0, n, 1021)
         xs = x[idx.to(DEV)].cpu()
         eref, rref = oracle.clip_error_rows(synth.to_oracle_array(xs), w.d, w.d_pad, w.m, 3, w.group, alphas,
                                             want_rows=True)

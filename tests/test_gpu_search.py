@@ -60,3 +60,39 @@ def test_search_argument_errors():
         for eps in (0.0, 1.0, -0.5, float("nan")):
             with pytest.raises(binding.GbsError):
                 plan.search_clip_ratio(x, eps)
+
+
+def test_batched_search_equals_independent_searches_and_resumes():
+    """P projections of different shapes searched together visit, each, the states of its own single search;
+    stopping after every round and resuming from the stored states gives the same list L."""
+    gbs_build.build()
+    specs = [("llama4096", 96, 3), ("qwen3584", 64, 3), ("kv128", 1000, 3), ("llama4096", 33, 4), ("mlp18944", 8, 4),
+             ("tiny", 64, 4)]
+    eps = 1 / 64
+    plans, xs, singles = [], [], []
+    for name, rows, bits in specs:
+        w = synth.WORKLOADS[name]
+        pl = Plan(w.d, w.d_pad, w.m, bits, w.group, w.alpha)
+        x = synth.make_host(name, rows).to(DEV)
+        plans.append(pl)
+        xs.append(x)
+        singles.append(pl.search_clip_ratio(x, eps))
+    alphas, states, rounds = binding.gbs_search_clip_ratio_batch([p.handle for p in plans], xs, eps)
+    assert rounds == max(s.rounds for s in singles)               # one wait per round, not per projection
+    for a, st, s in zip(alphas, states, singles):
+        assert st.done == 1 and a == s.alpha and st.iteration == s.iterations and st.evaluations == s.evaluations
+        # the K sums are accumulated with fp64 atomics across CTAs: equal up to summation order
+        assert np.isclose(st.f_m, s.err, rtol=1e-9) and (np.float32(st.a), np.float32(st.b)) == (np.float32(s.a), np.float32(s.b))
+    # resumable: one round per call, states copied through bytes in between
+    sts, total = None, 0
+    while True:
+        al2, sts, r = binding.gbs_search_clip_ratio_batch([p.handle for p in plans], xs, eps, states=sts, max_rounds=1)
+        sts = [binding.SearchState.from_buffer_copy(bytes(s)) for s in sts]
+        total += r
+        if all(s.done for s in sts):
+            break
+        assert total < 20
+    assert al2 == alphas and total == rounds
+    for p in plans:
+        assert p.device_status() == 0
+        p.close()
