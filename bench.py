@@ -57,6 +57,16 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def measured_bf16_tflops():
+    """Dense bf16 tensor throughput measured on this machine (burst figure: for a kernel timed alone)."""
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["bf16_tflops"]), "measured"
+    except Exception:
+        return 1590.0, "fallback"
+
+
 def aggregate(local_ms: float, local_units: float, dist_ok: bool, device=None):
     """Whole-job figures: time = max over ranks, units = sum over ranks (replicas are independent)."""
     if not dist_ok:
@@ -629,6 +639,30 @@ def extras(device, stream, args, peak, sampler=None):
     out["dequantize_inverse_rotate_b3_bf16"] = {"us_per_launch": ms * 1e3,
                                                 "gbs": w.n_rows * (w.d_pad * 3 // 8 + 4 + w.d * 2) / ms / 1e6}
     del xhat, x, codes, scales, yhat
+    torch.cuda.empty_cache()
+    # the consumer of the codes: the layer's output from the packed codes of activations and weights (int8 x int8
+    # -> int32 on the tensor cores), 4096 tokens x 4096 output channels x d' = 4096
+    bf16_tf, bf16_kind = measured_bf16_tflops()
+    i8_peak = 2.0 * bf16_tf                      # nominal dense int8 : bf16 ratio of the part (4.5 : 2.25 PFLOP/s)
+    xq = synth.make_host("llama4096").to(device)
+    wq = (torch.randn((4096, w.d), generator=torch.Generator().manual_seed(7)) / 64.0).to(torch.bfloat16).to(device)
+    for bx, bw in ((4, 4), (3, 3)):
+        px, pw = Plan(w.d, w.d_pad, w.m, bx, 0, w.alpha), Plan(w.d, w.d_pad, w.m, bw, 0, 1.0)
+        cx, sx, _ = px.rotate_quantize(xq)
+        cw, sw = pw.weight_rotate_quantize(wq)
+        outm = torch.empty((xq.shape[0], wq.shape[0]), dtype=torch.bfloat16, device=device)
+        ms = time_loop(lambda i: px.quantized_matmul(cx, sx, pw, cw, sw, out=outm, stream=stream), 8)
+        tops = 2.0 * xq.shape[0] * wq.shape[0] * w.d_pad / ms / 1e9
+        out["quantized_matmul_x%d_w%d_4096x4096x4096" % (bx, bw)] = {
+            "us_per_launch": ms * 1e3, "tops": tops,
+            "roofline": {"bound": "tensor", "unit": "TOP/s", "achieved": tops, "peak": i8_peak, "frac": tops / i8_peak,
+                         "note": "int8 peak = 2 x the %s bf16 figure (nominal int8 : bf16 ratio); the kernel is bound by "
+                                 "unpacking the codes to int8, not by the tensor pipe" % bf16_kind}}
+        del px, pw, cx, sx, cw, sw, outm
+    ms = time_loop(lambda i: torch.matmul(xq, wq.t()), 8)
+    out["bf16_matmul_of_the_unquantized_operands_4096x4096x4096"] = {"us_per_launch": ms * 1e3,
+                                                                     "note": "library GEMM, context only"}
+    del xq, wq
     torch.cuda.empty_cache()
     # clip-ratio scoring at the calibration size: K = 32 candidates over one full layer of 128 sequences x 2048
     # tokens x d = 4096 per launch, for each of 32 layers (its own seeded tensor each: seed 5 + layer)

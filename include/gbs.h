@@ -269,6 +269,36 @@ int gbs_search_clip_ratio(const gbs_plan_t* plan, const void* x, int x_dtype, in
                           void* cuda_stream);
 
 /*
+ * Weight side of the expansion (Section 4.2, Eq. (2)): the rows of W (one per output channel, width d) are
+ * zero-padded to d', rotated by the same H_{d'} / sqrt(d') as the activations and quantized round-to-nearest with
+ * the plan's bits, group and alpha -- exactly gbs_rotate_quantize applied to the rows of W, which is what makes
+ * (H x_pad)^T (H w_pad) / d' = x^T w hold code for code.  With group = 0 there is one scale per output channel, the
+ * form gbs_quantized_matmul consumes.  Done once, offline.
+ *   w, w_dtype, n_out, w_row_stride   the weight matrix [n_out, d] (device), as x / x_dtype / n_rows / x_row_stride
+ *   codes, scales                     as for gbs_rotate_quantize
+ */
+int gbs_weight_rotate_quantize(const gbs_plan_t* plan, const void* w, int w_dtype, int64_t n_out, int64_t w_row_stride,
+                               void* codes, float* scales, void* cuda_stream);
+
+/*
+ * The layer's output straight from the packed codes of both sides (Eq. (2); Section 2.3.1 on keeping the inverse
+ * rotation out of the online path): out[t][o] = Delta_x[t] * Delta_w[o] * sum_j q_x[t][j] * q_w[o][j], j over the
+ * d' rotated coordinates -- the product of the dequantized rotated activation and the dequantized rotated weight,
+ * which equals x^T w up to the two quantization errors.  The sum is an int8 x int8 -> int32 contraction on the
+ * tensor cores (exact); the rotated activation is never materialised as floats.
+ *   plan_x, codes_x, scales_x, n_tokens   activations as written by gbs_rotate_quantize
+ *   plan_w, codes_w, scales_w, n_out      weights as written by gbs_weight_rotate_quantize
+ *   out, out_dtype, out_row_stride        device, [n_tokens, n_out] fp32 or bf16, row stride in elements (>= n_out);
+ *                                         rows that start on 16-byte boundaries get vector stores
+ * Limits: both plans on one device with the same d, d' and m, symmetric, group 0 (one scale per token and per
+ * output channel, so the scales leave the sum), d' a multiple of 128; bits may differ (3 or 4 each).  Other plans
+ * return GBS_ERR_UNSUPPORTED.
+ */
+int gbs_quantized_matmul(const gbs_plan_t* plan_x, const void* codes_x, const float* scales_x, int64_t n_tokens,
+                         const gbs_plan_t* plan_w, const void* codes_w, const float* scales_w, int64_t n_out,
+                         void* out, int out_dtype, int64_t out_row_stride, void* cuda_stream);
+
+/*
  * State of one projection's search (Algorithm 1), a handful of numbers: plain data that may be copied, stored
  * and handed back later to resume the search where it stopped (gbs_search_state_init gives the algorithm's
  * start a = 0, b = 1, m = 1/2).

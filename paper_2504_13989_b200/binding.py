@@ -30,7 +30,8 @@ GBS_PLAN_ASYMMETRIC = 1
 EXPORTS = ("gbs_plan_create", "gbs_plan_create_ex", "gbs_plan_destroy", "gbs_plan_info", "gbs_plan_device_status", "gbs_rotate_quantize",
            "gbs_rotate_quantize_static", "gbs_static_device_status", "gbs_dequantize", "gbs_clip_error",
            "gbs_search_clip_ratio", "gbs_search_state_init", "gbs_search_clip_ratio_fn", "gbs_search_clip_ratio_batch",
-           "gbs_hadamard_m", "gbs_status_string", "gbs_selftest_wait_expiry")
+           "gbs_hadamard_m", "gbs_status_string", "gbs_selftest_wait_expiry", "gbs_weight_rotate_quantize",
+           "gbs_quantized_matmul")
 GBS_STATIC_MAX_D_PAD = 4096
 
 
@@ -113,6 +114,10 @@ def lib() -> ctypes.CDLL:
                                                   ctypes.POINTER(SearchState), i32, vp, ctypes.POINTER(ctypes.c_float),
                                                   ctypes.POINTER(i32), vp]
         L.gbs_search_clip_ratio_batch.restype = i32
+        L.gbs_weight_rotate_quantize.argtypes = [vp, vp, i32, i64, i64, vp, vp, vp]
+        L.gbs_weight_rotate_quantize.restype = i32
+        L.gbs_quantized_matmul.argtypes = [vp, vp, vp, i64, vp, vp, vp, i64, vp, i32, i64, vp]
+        L.gbs_quantized_matmul.restype = i32
         L.gbs_hadamard_m.argtypes = [i32, vp]
         L.gbs_hadamard_m.restype = i32
         L.gbs_status_string.argtypes = [i32]
@@ -309,6 +314,35 @@ def gbs_search_clip_ratio(plan: int, x: torch.Tensor, eps: float, work: torch.Te
     return res
 
 
+def gbs_weight_rotate_quantize(plan: int, w: torch.Tensor, codes: torch.Tensor, scales: torch.Tensor, stream=None) -> None:
+    """Rows of the weight matrix [n_out, d] through the activation path's rotation and quantizer (Eq. (2))."""
+    info = gbs_plan_info(plan)
+    wv, n_out, stride = _rows_view(w, info.d)
+    _check_buffer("codes", codes, wv, torch.uint8, n_out * info.code_bytes_per_row)
+    _check_buffer("scales", scales, wv, torch.float32, n_out * info.scale_floats_per_row)
+    _check(lib().gbs_weight_rotate_quantize(ctypes.c_void_p(plan), wv.data_ptr(), _dtype_code(wv), n_out, stride,
+                                            codes.data_ptr(), scales.data_ptr(), _stream_ptr(stream)),
+           "gbs_weight_rotate_quantize")
+
+
+def gbs_quantized_matmul(plan_x: int, codes_x: torch.Tensor, scales_x: torch.Tensor, plan_w: int, codes_w: torch.Tensor,
+                         scales_w: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+    """out[t, o] = Delta_x[t] * Delta_w[o] * sum_j q_x[t, j] * q_w[o, j] from the packed codes of both sides."""
+    ix, iw = gbs_plan_info(plan_x), gbs_plan_info(plan_w)
+    n_tok, n_out = codes_x.shape[0], codes_w.shape[0]
+    _check_buffer("codes_x", codes_x, codes_x, torch.uint8, n_tok * ix.code_bytes_per_row)
+    _check_buffer("scales_x", scales_x, codes_x, torch.float32, n_tok * ix.scale_floats_per_row)
+    _check_buffer("codes_w", codes_w, codes_x, torch.uint8, n_out * iw.code_bytes_per_row)
+    _check_buffer("scales_w", scales_w, codes_x, torch.float32, n_out * iw.scale_floats_per_row)
+    if out.dim() != 2 or out.shape[0] != n_tok or out.shape[1] != n_out or out.stride(1) != 1 or not out.is_cuda \
+            or out.device != codes_x.device:
+        raise ValueError("gbs_quantized_matmul: out must be a CUDA [n_tokens, n_out] tensor with contiguous rows")
+    _check(lib().gbs_quantized_matmul(ctypes.c_void_p(plan_x), codes_x.data_ptr(), scales_x.data_ptr(), n_tok,
+                                      ctypes.c_void_p(plan_w), codes_w.data_ptr(), scales_w.data_ptr(), n_out,
+                                      out.data_ptr(), _dtype_code(out), out.stride(0), _stream_ptr(stream)),
+           "gbs_quantized_matmul")
+
+
 def gbs_search_state_init() -> SearchState:
     st = SearchState()
     _check(lib().gbs_search_state_init(ctypes.byref(st)), "gbs_search_state_init")
@@ -415,6 +449,21 @@ class Plan:
         rows = torch.empty((n_rows, K), dtype=torch.float32, device=x.device) if want_rows else None
         gbs_clip_error(self.handle, x, alphas, err_sum, rows, stream)
         return (err_sum, rows) if want_rows else err_sum
+
+    def weight_rotate_quantize(self, w: torch.Tensor, out=None, stream=None):
+        """Quantize the rows of a weight matrix [n_out, d] (Eq. (2)); returns (codes, scales)."""
+        n_out = w.numel() // self.info.d
+        codes, scales, _ = out if out is not None else self.alloc_outputs(n_out, w.device)
+        gbs_weight_rotate_quantize(self.handle, w, codes, scales, stream)
+        return codes, scales
+
+    def quantized_matmul(self, codes_x, scales_x, plan_w: "Plan", codes_w, scales_w, dtype=torch.float32, out=None,
+                         stream=None) -> torch.Tensor:
+        """The layer's output from the packed codes of activations (this plan) and weights (plan_w)."""
+        if out is None:
+            out = torch.empty((codes_x.shape[0], codes_w.shape[0]), dtype=dtype, device=codes_x.device)
+        gbs_quantized_matmul(self.handle, codes_x, scales_x, plan_w.handle, codes_w, scales_w, out, stream)
+        return out
 
     def search_clip_ratio(self, x: torch.Tensor, eps: float = 1.0 / 64, stream=None) -> SearchResult:
         return gbs_search_clip_ratio(self.handle, x, eps, stream=stream)
