@@ -81,7 +81,8 @@ typedef struct gbs_plan_info {
                                       d % 32 == 0 and group in {0, 32 .. 1024}, 2 = tensor-core path for
                                       d' = 128 rows (m = 1, group in {0, 32, 64, 128}), 3 = tensor-core path for
                                       4096 < d' = 32 * G * U <= 32768 (G in {2, 4, 8}, U as above, per-token
-                                      scales, d a multiple of 32 * G) (set GBS_FORCE_GENERIC=1 in the
+                                      scales, d a multiple of 32 * G), 4 = dense tensor-core contraction with the full
+                                      Paley matrix (d' = m) (set GBS_FORCE_GENERIC=1 in the
                                       environment before gbs_plan_create to force 0; GBS_NO_PDL=1 launches it
                                       without programmatic stream serialization) */
 } gbs_plan_info_t;
@@ -94,6 +95,11 @@ typedef struct gbs_plan_info {
  *   m       1 (pure Sylvester); 12, 20, 24, 44, 48, 60, 68, 72, 80, 84, 104 or 108 (Algorithm 2 with the
  *           prime p = m-1 = 3 mod 4); or 28 (Algorithm 2 over GF(27) = GF(3)[x]/(x^3+2x+1), elements
  *           indexed c0 + 3 c1 + 9 c2).  Other orders return GBS_ERR_UNSUPPORTED.
+ *           Full orders: d_pad = m (2^k = 1) is accepted when m - 1 is a prime = 3 mod 4, m a multiple of 8 and
+ *           128 <= m <= 4096 -- the rotation is then the Paley matrix H_m itself, e.g. d = 1536, d_pad = m = 1544
+ *           (Section 5.2.2).  Such plans take bf16 rows with d a multiple of 8 and group = 0, run as a dense
+ *           tensor-core contraction, and support gbs_rotate_quantize and gbs_dequantize without inverse rotation;
+ *           the other calls return GBS_ERR_UNSUPPORTED for them.
  *   bits    3 or 4
  *   group   0, or a power of two >= 8 dividing 2^k (so a group never straddles a block of H_m)
  *   alpha   0 < alpha <= 1

@@ -43,7 +43,7 @@ typedef gbs_device_guard DeviceGuard;
 extern "C" int gbs_hadamard_m(int m, int8_t* out_host)
 {
     if (!out_host || m < 1) return GBS_ERR_INVALID_ARG;
-    if (!supported_m(m)) return GBS_ERR_UNSUPPORTED;
+    if (!supported_m(m) && !gbs_supported_full_m(m)) return GBS_ERR_UNSUPPORTED;
     return gbs_build_hadamard_m(m, out_host);
 }
 
@@ -75,12 +75,14 @@ extern "C" int gbs_plan_create_ex(gbs_plan_t** out, int d, int d_pad, int m, int
     if (!(alpha > 0.f) || !(alpha <= 1.f)) return GBS_ERR_INVALID_ARG;     // also rejects NaN
     if (d_pad % m != 0) return GBS_ERR_INVALID_ARG;
     const int k = log2_exact(d_pad / m);
-    if (k < 3) return GBS_ERR_INVALID_ARG;                                  // 2^k >= 8
+    const bool full = (k == 0 && gbs_supported_full_m(m));                  // d' = m: the rotation is H_m itself
+    if (k < 3 && !full) return GBS_ERR_INVALID_ARG;                         // 2^k >= 8
     if (group != 0) {
         if (group < 8 || log2_exact(group) < 0 || (1 << k) % group != 0) return GBS_ERR_INVALID_ARG;
     }
-    if (!supported_m(m)) return GBS_ERR_UNSUPPORTED;
+    if (!full && !supported_m(m)) return GBS_ERR_UNSUPPORTED;
     if (d_pad > GBS_MAX_D_PAD) return GBS_ERR_UNSUPPORTED;
+    if (full && (group != 0 || (flags & GBS_PLAN_ASYMMETRIC) || d % 8 != 0)) return GBS_ERR_UNSUPPORTED;
     if ((flags & GBS_PLAN_ASYMMETRIC) &&
         !(d_pad == 128 && m == 1 && (group == 0 || group == 32 || group == 64 || group == 128)))
         return GBS_ERR_UNSUPPORTED;
@@ -96,7 +98,7 @@ extern "C" int gbs_plan_create_ex(gbs_plan_t** out, int d, int d_pad, int m, int
     p->c_inv = (float)((double)p->levels / (double)alpha);
     p->variant = GBS_VARIANT_GENERIC;
     p->asym = (flags & GBS_PLAN_ASYMMETRIC) ? 1 : 0;
-    int rc = gbs_build_hadamard_m(m, p->h_hm);
+    int rc = full ? GBS_OK : gbs_build_hadamard_m(m, p->h_hm);          // a full order has no small factor to keep
     if (rc != GBS_OK) { delete p; return rc; }
 
     cudaError_t e = cudaGetDevice(&p->device);
@@ -104,11 +106,36 @@ extern "C" int gbs_plan_create_ex(gbs_plan_t** out, int d, int d_pad, int m, int
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, p->device);
     if (e != cudaSuccess) { cudaGetLastError(); delete p; return GBS_ERR_CUDA; }
 
-    if (gbs_generic_smem_bytes(p, nullptr) > (size_t)p->smem_optin) { delete p; return GBS_ERR_UNSUPPORTED; }
+    if (!full && gbs_generic_smem_bytes(p, nullptr) > (size_t)p->smem_optin) { delete p; return GBS_ERR_UNSUPPORTED; }
 
     e = cudaMalloc(&p->d_status, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(p->d_status, 0, sizeof(int));
     if (e != cudaSuccess) { cudaGetLastError(); if (p->d_status) cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC; }
+    if (full) {
+        // the only family for a full order: the bf16 image of H_m (m * m * 2 bytes) is the plan's one table
+        if (!gbs_tc_dense_supported(p)) { cudaFree(p->d_status); delete p; return GBS_ERR_UNSUPPORTED; }
+        int8_t* hm = (int8_t*)malloc((size_t)m * m);
+        unsigned short* img = (unsigned short*)malloc((size_t)m * m * 2);
+        rc = (hm && img) ? gbs_build_hadamard_m(m, hm) : GBS_ERR_ALLOC;
+        if (rc == GBS_OK) {
+            gbs_tc_dense_image(hm, m, img);
+            e = cudaMalloc(&p->d_aimg, (size_t)m * m * 2);
+            if (e == cudaSuccess) e = cudaMemcpy(p->d_aimg, img, (size_t)m * m * 2, cudaMemcpyHostToDevice);
+            if (e != cudaSuccess) { cudaGetLastError(); rc = GBS_ERR_ALLOC; }
+        }
+        free(hm);
+        free(img);
+        if (rc != GBS_OK) {
+            if (p->d_aimg) cudaFree(p->d_aimg);
+            cudaFree(p->d_status);
+            delete p;
+            return rc;
+        }
+        p->variant = GBS_VARIANT_TC_DENSE;
+        p->pdl = 0;
+        *out = p;
+        return GBS_OK;
+    }
     const char* force = getenv("GBS_FORCE_GENERIC");
     const bool want_tc = !(force && force[0] == '1');
     const bool tc_uv = want_tc && gbs_tc_uv_supported(p);
@@ -232,11 +259,14 @@ extern "C" int gbs_rotate_quantize(const gbs_plan_t* p, const void* x, int x_dty
     if (!aligned16(codes) || (y_opt && !aligned16(y_opt)) || (reinterpret_cast<uintptr_t>(scales) & 3u))
         return GBS_ERR_ALIGNMENT;
     if (p->asym && !(p->variant == GBS_VARIANT_TC_ROW && x_dtype == GBS_DTYPE_BF16)) return GBS_ERR_UNSUPPORTED;
+    if (p->variant == GBS_VARIANT_TC_DENSE && x_dtype != GBS_DTYPE_BF16) return GBS_ERR_UNSUPPORTED;   // bf16 rows only
     DeviceGuard g;
     if (g.enter(p->device) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     int e;
-    if (p->variant == GBS_VARIANT_TC_UV && x_dtype == GBS_DTYPE_BF16)
+    if (p->variant == GBS_VARIANT_TC_DENSE)
+        e = gbs_tc_dense_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
+    else if (p->variant == GBS_VARIANT_TC_UV && x_dtype == GBS_DTYPE_BF16)
         e = gbs_tc_uv_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
     else if (p->variant == GBS_VARIANT_TC_UVM && x_dtype == GBS_DTYPE_BF16)
         e = gbs_tc_uvm_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
@@ -255,6 +285,7 @@ extern "C" int gbs_dequantize(const gbs_plan_t* p, const void* codes, const floa
     if (out_dtype != GBS_DTYPE_F32 && out_dtype != GBS_DTYPE_BF16) return GBS_ERR_INVALID_ARG;
     if (flags & ~GBS_INVERSE_ROTATE) return GBS_ERR_INVALID_ARG;
     if (n_rows < 0) return GBS_ERR_INVALID_ARG;
+    if ((flags & GBS_INVERSE_ROTATE) && p->variant == GBS_VARIANT_TC_DENSE) return GBS_ERR_UNSUPPORTED;
     if (n_rows == 0) return GBS_OK;
     if (!codes || !scales || !out) return GBS_ERR_INVALID_ARG;
     if (!aligned16(codes) || !aligned16(out) || (reinterpret_cast<uintptr_t>(scales) & 3u))
@@ -279,7 +310,7 @@ extern "C" int gbs_clip_error(const gbs_plan_t* p, const void* x, int x_dtype, i
     int rc = check_rows(p, x, x_dtype, n_rows, x_row_stride);
     if (rc != GBS_OK) return rc;
     if (K < 1 || K > GBS_MAX_CANDIDATES || !alphas_host) return GBS_ERR_INVALID_ARG;
-    if (p->asym) return GBS_ERR_UNSUPPORTED;
+    if (p->asym || p->variant == GBS_VARIANT_TC_DENSE) return GBS_ERR_UNSUPPORTED;
     float c_scale[GBS_MAX_CANDIDATES], c_inv[GBS_MAX_CANDIDATES];
     const double rootn = sqrt((double)p->d_pad);
     for (int i = 0; i < K; ++i) {

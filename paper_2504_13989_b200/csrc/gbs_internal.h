@@ -14,6 +14,7 @@ enum gbs_variant {
     GBS_VARIANT_GENERIC = 0,   // shared-memory FWHT on the plain ALUs; any supported (m, k), any dtype
     GBS_VARIANT_TC_UVM = 3,    // 4096 < d' = 32*G*U <= 32768, G in {2,4,8}: tensor cores + two register sweeps over TMEM
     GBS_VARIANT_TC_ROW = 2,    // d' = 128 (KV rows): X * H_128 on tcgen05 tensor cores, one thread owns one row
+    GBS_VARIANT_TC_DENSE = 4,  // d' = m, a full Paley order (k = 0): X * H_m^T as a dense tcgen05 contraction, two sweeps
     GBS_VARIANT_TC_UV = 1,     // d' = U*32, U = m*2^j <= 128: (H_m (x) H_{2^j}) on tcgen05 tensor cores + H_32 in
                                // registers (bf16 rows)
 };
@@ -63,7 +64,8 @@ struct gbs_device_guard {
 
 // gbs_paley.cu
 int gbs_build_hadamard_m(int m, int8_t* out);   // 0 or GBS_ERR_UNSUPPORTED
-bool gbs_supported_m(int m);                    // the orders a plan accepts
+bool gbs_supported_m(int m);                    // the orders a plan accepts as the factor of H_m (x) H_{2^k}
+bool gbs_supported_full_m(int m);               // the orders a plan accepts as the whole rotation (d' = m, k = 0)
 
 // gbs_generic.cu : launches on `stream`; return a cudaError_t cast to int (0 = success)
 int gbs_generic_rotate_quantize(const gbs_plan* p, const void* x, int x_dtype, int64_t n_rows,
@@ -103,6 +105,12 @@ int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
                                float* scales, float* y_opt, cudaStream_t stream);
 int gbs_tc_uvm_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, const float* alphas, int K,
                           double* err_sum, float* err_rows, cudaStream_t stream);
+
+// gbs_tc_dense.cu
+bool gbs_tc_dense_supported(const gbs_plan* p);
+void gbs_tc_dense_image(const int8_t* hm, int m, unsigned short* img);
+int gbs_tc_dense_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
+                                 float* scales, float* y_opt, cudaStream_t stream);
 
 // gbs_tc_row.cu
 bool gbs_tc_row_supported(const gbs_plan* p);

@@ -77,6 +77,13 @@ bool gbs_supported_m(int m)
     return false;
 }
 
+// Full orders (the whole rotation is H_m, Section 5.2.2): p = m - 1 prime, p = 3 (mod 4), m a multiple of 8 so that
+// packed rows are whole bytes, large enough to be worth a dense tensor-core contraction and small enough for its image.
+bool gbs_supported_full_m(int m)
+{
+    return m >= 128 && m <= 4096 && m % 8 == 0 && prime_3_mod_4(m - 1);
+}
+
 int gbs_build_hadamard_m(int m, int8_t* H)
 {
     if (m == 1) { H[0] = 1; return GBS_OK; }

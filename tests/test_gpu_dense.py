@@ -1,0 +1,61 @@
+"""The full Paley order (Section 5.2.2): width 1536 expanded by 8 to d' = m = 1544 = 1543 + 1, the rotation being
+Algorithm 2's matrix itself, run as a dense tensor-core contraction; against the oracle's dense definition."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2504_13989_b200 import Plan, binding, synth
+from paper_2504_13989_b200 import build as gbs_build
+from parity_util import compare_rotate_quantize, unpack_codes
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+D, M = 1536, 1544
+
+
+def _rows(n, seed):
+    rng = np.random.Generator(np.random.PCG64(seed))
+    x = 0.5 * rng.standard_t(3.0, size=(n, D))
+    x[:, rng.choice(D, 8, replace=False)] *= 50.0
+    x[rng.choice(n, max(1, n // 100), replace=False)] *= 20.0
+    return torch.from_numpy(x.astype(np.float32)).to(torch.bfloat16)
+
+
+@pytest.mark.parametrize("bits,rows,alpha", [(3, 130, 0.9), (4, 1, 1.0)])
+def test_full_paley_1544_against_the_dense_definition(bits, rows, alpha):
+    gbs_build.build()
+    x = _rows(rows, 40 + rows)
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(x), D, M, M, bits, 0, alpha, dense=True)
+    with Plan(D, M, M, bits, 0, alpha) as plan:
+        assert plan.info.variant == 4 and plan.info.k == 0 and plan.info.code_bytes_per_row == M * bits // 8
+        codes, scales, y = plan.rotate_quantize(x.to(DEV), want_y=True)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+        compare_rotate_quantize(x, ref, codes, scales, y, bits, 0, M, alpha)
+        # rotated-domain dequantize of these codes
+        yhat = plan.dequantize(codes, scales)
+        q = unpack_codes(codes.cpu().numpy(), M, bits)
+        np.testing.assert_allclose(yhat.cpu().double().numpy(), q * scales.cpu().double().numpy(), rtol=2e-7, atol=0)
+        # what this family does not serve is refused, not faulted
+        for call in (lambda: plan.clip_error(x.to(DEV), [0.5, 1.0]), lambda: plan.dequantize(codes, scales, inverse=True)):
+            with pytest.raises(binding.GbsError) as e:
+                call()
+            assert e.value.status == binding.GBS_ERR_UNSUPPORTED
+
+
+def test_full_order_plans_are_validated_on_the_host():
+    gbs_build.build()
+    lib = binding.lib()
+    import ctypes
+    h = ctypes.c_void_p()
+    # 1545 - 1 is not a prime = 3 mod 4; 1544 with a group; fp32 rows
+    assert lib.gbs_plan_create(ctypes.byref(h), 1536, 1545, 1545, 3, 0, 0.9) in (binding.GBS_ERR_INVALID_ARG, binding.GBS_ERR_UNSUPPORTED)
+    assert lib.gbs_plan_create(ctypes.byref(h), 1536, 1544, 1544, 3, 8, 0.9) == binding.GBS_ERR_INVALID_ARG
+    with Plan(D, M, M, 3, 0, 0.9) as plan:
+        x = torch.zeros((4, D), dtype=torch.float32, device=DEV)
+        with pytest.raises(binding.GbsError) as e:
+            plan.rotate_quantize(x)
+        assert e.value.status == binding.GBS_ERR_UNSUPPORTED
+    hm = binding.gbs_hadamard_m(M).to(torch.int64)
+    assert torch.equal(hm @ hm.T, M * torch.eye(M, dtype=torch.int64))
