@@ -38,8 +38,8 @@ HEADLINE = "llama4096"
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused kernel on the headline
 # workload, from the ncu capture summarised under profiles/ (None until a capture exists).
-NCU_TRAFFIC_BYTES_PER_LAUNCH = None         # set from the capture of the current kernel, see profiles/
-NCU_TRAFFIC_BYTES_PER_LAUNCH_D3584 = None
+NCU_TRAFFIC_BYTES_PER_LAUNCH = 33_624_064   # dram reads 33.62 MB + writes 0 (codes still in L2 at kernel end); profiles/uv_rq_llama4096.md
+NCU_TRAFFIC_BYTES_PER_LAUNCH_D3584 = 59_470_592   # 58.79 MB read + 0.68 MB written; profiles/uv_rq_qwen3584.md
 
 
 def algorithmic_bytes(n_rows: int, d: int, d_pad: int, bits: int, group: int, in_bytes: int) -> int:
@@ -349,6 +349,8 @@ def main():
     ap.add_argument("--e2e-chunks", type=int, default=4, help="row chunks of the host-buffer pipeline (copies overlap)")
     ap.add_argument("--cpu-seconds", type=float, default=10.0)
     ap.add_argument("--no-extras", action="store_true", help="skip the context legs under `also`")
+    ap.add_argument("--min-ms", type=float, default=MIN_TIMED_MS,
+                    help="the K steps are repeated until the timed region lasts this long (0: exactly K steps)")
     ap.add_argument("--profile", default=None, metavar="WORKLOAD[:ROWS]",
                     help="launch one workload's kernel a few times and exit (for ncu captures), e.g. kv128:262144, llama4096-inverse:4096, "
                          "clip:8192")
@@ -396,7 +398,8 @@ def main():
     step_tokens = len(w.bits) * w.n_rows
     launches_per_step = len(w.bits)
 
-    local_ms, steps_timed = timed_graph_loop(plans, sets, args.steps, args.warmup, stream, dist_ok, sampler)
+    local_ms, steps_timed = timed_graph_loop(plans, sets, args.steps, args.warmup, stream, dist_ok, sampler,
+                                             min_ms=args.min_ms)
     total_ms, total_bytes = aggregate(local_ms, step_bytes * steps_timed, dist_ok, device)
     _, total_tokens = aggregate(local_ms, step_tokens * steps_timed, dist_ok, device)
     ms_per_step = total_ms / steps_timed
@@ -424,7 +427,7 @@ def main():
     bytes2 = sum(algorithmic_bytes(w2.n_rows, w2.d, w2.d_pad, b, w2.group, 2) for b in w2.bits)
     sets2 = build_sets(plans2, synth.make_host("qwen3584"), 8, device)
     steps2 = max(8, args.steps // 2 // 8 * 8)
-    ms2, timed2 = timed_graph_loop(plans2, sets2, steps2, 3, stream, False)
+    ms2, timed2 = timed_graph_loop(plans2, sets2, steps2, 3, stream, False, min_ms=args.min_ms)
     del sets2
     torch.cuda.empty_cache()
     ach2 = bytes2 / (ms2 / timed2 * 1e-3) / 1e9
@@ -497,7 +500,7 @@ def main():
                        (args.nsets, args.nsets * (step_bytes + w.n_rows * w.d * 2) / 1e6),
                        "launch": "CUDA graph replay", "levels": "D=2^(b-1)-1",
                        "timed_region": "the K steps repeated %d time(s): at least %.0f ms on the device" %
-                                       (steps_timed // args.steps, MIN_TIMED_MS)},
+                                       (steps_timed // args.steps, args.min_ms)},
             "mtokens_per_s": total_tokens / (total_ms * 1e-3) / 1e6,
             "hbm_frac_of_measured": value / world / peak, "hbm_frac_of_8000": value / world / 8000.0,
             "roofline": roofline, "roofline_d3584": roofline_d3584, "cpu_baseline": cpu_baseline, "e2e": e2e, "clocks": clocks,
@@ -513,6 +516,28 @@ def run_profile(spec, device):
     """A few launches of one kernel on a small case, for an ncu capture (prints nothing a result line would)."""
     from paper_2504_13989_b200 import Plan, synth
     name, _, rows = spec.partition(":")
+    if name in ("matmul", "dense1544"):
+        n = int(rows) if rows else 4096
+        if name == "matmul":          # the consumer: 4-bit codes x 4-bit codes, n tokens x n output channels x 4096
+            px, pw = Plan(4096, 4096, 1, 4, 0, 0.9), Plan(4096, 4096, 1, 4, 0, 1.0)
+            xq = synth.make_device("llama4096", n, device=str(device))
+            wq = (torch.randn((n, 4096), device=device) / 64).to(torch.bfloat16)
+            cx, sx, _ = px.rotate_quantize(xq)
+            cw, sw = pw.weight_rotate_quantize(wq)
+            out = torch.empty((n, n), dtype=torch.bfloat16, device=device)
+            for _ in range(4):
+                px.quantized_matmul(cx, sx, pw, cw, sw, out=out)
+            torch.cuda.synchronize()
+            print(json.dumps({"profile": spec, "rows": n, "status": px.device_status()}))
+        else:                         # the full Paley order: width 1536 -> d' = m = 1544
+            pl = Plan(1536, 1544, 1544, 3, 0, 0.9)
+            xq = (torch.randn((n, 1536), device=device) * 0.5).to(torch.bfloat16)
+            outs = pl.alloc_outputs(n, device)
+            for _ in range(4):
+                pl.rotate_quantize(xq, out=outs)
+            torch.cuda.synchronize()
+            print(json.dumps({"profile": spec, "rows": n, "kernel_family": pl.info.variant, "status": pl.device_status()}))
+        return
     clip = name == "clip"
     inverse = name.endswith("-inverse")               # e.g. llama4096-inverse: gbs_dequantize with inverse rotation
     if inverse:
