@@ -14,14 +14,15 @@
 //   * One CTA per 128 x 256 tile of the output (tokens x output channels); the contraction runs over blocks of 128
 //     codes through a ring of shared-memory stages.
 //   * Sixteen warps unpack: each thread fetches the packed 3- or 4-bit codes of its slice of the next block straight
-//     from global memory (one block ahead, held in registers), sign-extends them to int8 with byte-wise logic (a
-//     byte permute replicates every field's sign bit), and writes 16-byte chunks into the K-major, 128-byte-swizzled
-//     operand tiles the tensor cores read.  Both operands use the same order of the codes inside a chunk (even
+//     from global memory (whole lines: 256 codes of a row per eight threads, two such super-blocks ahead, held in
+//     registers), turns them into int8 with byte-wise logic (a field moved to the top bits of its byte IS the int8
+//     q * 2^(8-b); the epilogue removes the power of two), and writes 16-byte chunks into the K-major,
+//     128-byte-swizzled operand tiles the tensor cores read.  Both operands use the same order of the codes inside a chunk (even
 //     fields first, then odd), which a dot product does not see.
 //   * One thread issues tcgen05.mma kind::i8 (int8 x int8 -> int32, 128 x 256 x 32 per instruction), accumulators
 //     in TMEM; tcgen05.commit hands the stage back to the unpackers.
-//   * After the last block the sixteen warps read the int32 sums from TMEM (exact: at most 49 * d' < 2^24 in
-//     magnitude), convert, scale by Delta_x[t] * Delta_w[o] and store fp32 or bf16.
+//   * After the last block the sixteen warps read the int32 sums from TMEM (exact), convert (a multiple of
+//     2^(16-bx-bw) whose quotient is below 2^24: exact in fp32), scale by Delta_x[t] * Delta_w[o], store fp32 or bf16.
 // Every wait is bounded; an expired wait records a code in the activation plan's status word.
 #include <math.h>
 #include <string.h>
@@ -87,32 +88,25 @@ __device__ __forceinline__ void st_shared_v4(unsigned addr, uint4 v)
     asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 
-// 0x00 or 0xFF per byte of x, by that byte's top bit: prmt with the sign-replication bit set in every selector
-// (the __byte_perm intrinsic keeps only three selector bits, so the instruction is written out).
-__device__ __forceinline__ unsigned byte_signs(unsigned x)
-{
-    unsigned d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(x), "r"(0u), "r"(0xBA98u));
-    return d;
-}
-
 // Eight two's-complement fields (24 or 32 bits) -> two words of four int8 each: the even fields, the odd fields.
-// The fields are spread to one per nibble; a byte permute in sign-replication mode turns the byte whose top bit is a
-// field's sign bit into 0x00 or 0xFF, which supplies the upper bits of the int8.
+// No sign extension is computed: a field moved to the TOP bits of its byte is the int8 value q * 2^(8 - BITS) (the
+// field's sign bit becomes the byte's), products are then scaled by a power of two that the epilogue's scale factor
+// takes out exactly, and the int32 sums stay far below 2^31 (49 * d' * 2^10 at most).  Four-bit fields already sit in
+// nibbles: one mask for the odd ones, a shift and a mask for the even ones.  Three-bit fields are first spread to one
+// per nibble by three mask-and-shift steps.
 template <int BITS>
 __device__ __forceinline__ void fields_to_int8(unsigned f, unsigned& even, unsigned& odd)
 {
-    if (BITS == 3) {
+    if (BITS == 4) {
+        odd = f & 0xf0f0f0f0u;
+        even = (f << 4) & 0xf0f0f0f0u;
+    } else {
         f = (f & 0x00000fffu) | ((f & 0x00fff000u) << 4);       // 12 bits per half-word
         f = (f & 0x003f003fu) | ((f & 0x0fc00fc0u) << 2);       // 6 bits per byte
         f = (f & 0x07070707u) | ((f & 0x38383838u) << 1);       // 3 bits per nibble (bit 3 of every nibble clear)
+        odd = (f << 1) & 0xe0e0e0e0u;
+        even = (f << 5) & 0xe0e0e0e0u;
     }
-    constexpr unsigned LOW = BITS == 3 ? 0x07070707u : 0x0f0f0f0fu;     // value bits below the sign extension
-    constexpr int UP = BITS == 3 ? 5 : 4;                                // even field's sign bit -> bit 7 of its byte
-    const unsigned se = byte_signs(f << UP);                             // 0xFF where the even field is negative
-    const unsigned so = byte_signs(f << (UP - 4));                       // the same for the odd fields
-    even = (f & LOW) | (se & ~LOW);
-    odd = ((f >> 4) & LOW) | (so & ~LOW);
 }
 
 // NF fields of a row slice, from its packed words (3 words per 4 fields at 3 bits, 1 word per field at 4 bits).
@@ -212,40 +206,75 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_qgemm(const __grid_constant__
     } else {
         // ------------------------------ unpack, then epilogue ------------------------------
         const int ut = threadIdx.x - 32;              // 0 .. 511
-        // activation tile: 128 rows x 128 codes, four threads per row, 32 codes (two chunks) each
-        const int ar = ut >> 2, ap = ut & 3;
-        // weight tile: 256 rows x 128 codes, two threads per row, 64 codes (four chunks) each
-        const int br = ut >> 1, bp = ut & 1;
-        const bool a_live = tok0 + ar < P.n_tok, b_live = out0 + br < P.n_out;
-        const unsigned char* ax = P.cx + (tok0 + ar) * (long long)P.rbx + ap * (32 * XBITS / 8);
-        const unsigned char* bw = P.cw + (out0 + br) * (long long)P.rbw + bp * (64 * WBITS / 8);
-        // The packed codes of the next PF blocks are in flight (in registers) while one block is unpacked: a block is
-        // consumed in a few hundred cycles, a global load takes a few thousand.
-        constexpr int PF = 3;
-        unsigned ra[PF][4], rb[PF][8];
+        // Work is cut into SUPER-BLOCKS of 256 codes per row (two stages) so that the global loads are whole lines: an
+        // item is 32 codes (four fields, 16 or 12 bytes) of one row; the eight threads ut & 7 = 0..7 take the eight
+        // items of a row's 256 codes (128 or 96 contiguous bytes), so a warp's load instruction covers four rows'
+        // full lines.  (Loading per 128-code block, with two or four threads per row, asked the L1 for 32 sectors per
+        // request and kept it 89 % busy: that, not the arithmetic or shared memory, bound the kernel.)
+        // A thread's item position seg is fixed: stage half h = seg >> 2, chunks 2 (seg & 3) and + 1 of the row; its
+        // rows are r0 + 64 i: two of the activation tile, four of the weight tile.
+        // Lane bits, low to high: part (2), row bit 0, half, row bit 1.  A 16-byte shared-memory store is served eight
+        // lanes at a time: eight consecutive lanes then hold two rows x four parts of ONE stage, whose swizzled chunk
+        // positions are all different (both halves of a row would collide: same banks, other stage).
+        const int part = lane & 3, half = (lane >> 3) & 1, seg = 4 * half + part;
+        const int r0 = (ut >> 5) * 4 + ((lane >> 4) & 1) * 2 + ((lane >> 2) & 1);
+        constexpr int NA = TM / 64, NB = TN / 64;
+        constexpr int XSB = 256 * XBITS / 8, WSB = 256 * WBITS / 8;        // bytes of a super-block per row
+        const unsigned char* ax = P.cx + (tok0 + r0) * (long long)P.rbx + seg * (32 * XBITS / 8);
+        const unsigned char* bw = P.cw + (out0 + r0) * (long long)P.rbw + seg * (32 * WBITS / 8);
+        bool a_live[NA], b_live[NB];
 #pragma unroll
-        for (int j = 0; j < PF; ++j) {
-            const bool in = j < P.kblocks;
-            load_raw<XBITS, 4>(ax + (long long)j * (KB * XBITS / 8), a_live && in, ra[j]);
-            load_raw<WBITS, 8>(bw + (long long)j * (KB * WBITS / 8), b_live && in, rb[j]);
-        }
+        for (int i = 0; i < NA; ++i) a_live[i] = tok0 + r0 + 64 * i < P.n_tok;
+#pragma unroll
+        for (int i = 0; i < NB; ++i) b_live[i] = out0 + r0 + 64 * i < P.n_out;
+        const int n_sb = (P.kblocks + 1) >> 1;
+        // the packed codes of the next PF super-blocks are in flight (in registers) while one is unpacked
+        constexpr int PF = 2;
+        unsigned ra[PF][NA][4], rb[PF][NB][4];
+        auto load_sb = [&](int sb, unsigned (&qa)[NA][4], unsigned (&qb)[NB][4]) {
+            const bool in = 2 * sb + half < P.kblocks;                  // an odd number of blocks: no second half
+#pragma unroll
+            for (int i = 0; i < NA; ++i)
+                load_raw<XBITS, 4>(ax + (long long)sb * XSB + (long long)(64 * i) * P.rbx, in && a_live[i], qa[i]);
+#pragma unroll
+            for (int i = 0; i < NB; ++i)
+                load_raw<WBITS, 4>(bw + (long long)sb * WSB + (long long)(64 * i) * P.rbw, in && b_live[i], qb[i]);
+        };
+#pragma unroll
+        for (int j = 0; j < PF; ++j) load_sb(j, ra[j], rb[j]);
         bool alive = true;
-        for (int kb0 = 0; alive && kb0 < P.kblocks; kb0 += PF) {
+        for (int sb0 = 0; alive && sb0 < n_sb; sb0 += PF) {
 #pragma unroll
             for (int j = 0; j < PF; ++j) {
-                const int kb = kb0 + j;
-                if (kb >= P.kblocks) break;
+                const int sb = sb0 + j;
+                if (sb >= n_sb) break;
+                const int kb = 2 * sb + half;                           // the block this thread's items belong to
+                const bool mine = kb < P.kblocks;
                 const int s = kb % STAGES;
-                if (!mbar_wait(&S->abort_flag, &S->empty[s], ((kb / STAGES) & 1) ^ 1, P.status, 1)) { alive = false; break; }
-                unpack_store<XBITS, 4>(ra[j], smem_u32(S->a[s]) + (unsigned)ar * 128u, 2 * ap, ar & 7);
-                unpack_store<WBITS, 8>(rb[j], smem_u32(S->b[s]) + (unsigned)br * 128u, 4 * bp, br & 7);
-                const bool in = kb + PF < P.kblocks;
-                load_raw<XBITS, 4>(ax + (long long)(kb + PF) * (KB * XBITS / 8), a_live && in, ra[j]);
-                load_raw<WBITS, 8>(bw + (long long)(kb + PF) * (KB * WBITS / 8), b_live && in, rb[j]);
-                // make the generic-proxy writes visible to the tensor cores' (async proxy) reads, then signal
+                bool ok = true;
+                if (mine) ok = mbar_wait(&S->abort_flag, &S->empty[s], ((kb / STAGES) & 1) ^ 1, P.status, 1);
+                if (!__all_sync(0xffffffffu, ok)) { alive = false; break; }       // the warp leaves as one
+                if (mine) {
+#pragma unroll
+                    for (int i = 0; i < NA; ++i) {
+                        const int r = r0 + 64 * i;
+                        unpack_store<XBITS, 4>(ra[j][i], smem_u32(S->a[s]) + (unsigned)r * 128u, 2 * part, r & 7);
+                    }
+#pragma unroll
+                    for (int i = 0; i < NB; ++i) {
+                        const int r = r0 + 64 * i;
+                        unpack_store<WBITS, 4>(rb[j][i], smem_u32(S->b[s]) + (unsigned)r * 128u, 2 * part, r & 7);
+                    }
+                }
+                if (sb + PF < n_sb) load_sb(sb + PF, ra[j], rb[j]);
+                // make the generic-proxy writes visible to the tensor cores' (async proxy) reads, then signal: a warp
+                // holds items of both halves, so it reports to both stages of the super-block
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&S->full[s]);
+                if (lane == 0) {
+                    mbar_arrive(&S->full[(2 * sb) % STAGES]);
+                    if (2 * sb + 1 < P.kblocks) mbar_arrive(&S->full[(2 * sb + 1) % STAGES]);
+                }
             }
         }
         if (alive && mbar_wait(&S->abort_flag, &S->tfull, 0, P.status, 4)) {
@@ -253,7 +282,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_qgemm(const __grid_constant__
             const int q = warp & 3;                    // TMEM lane quadrant this warp may access
             const int cb = (warp - 1) >> 2;            // 64-column block of the tile
             const long long tok = tok0 + q * 32 + lane;
-            const float dx = tok < P.n_tok ? __ldg(P.sx + tok) : 0.f;
+            // the int8 operands were q * 2^(8 - bits): take the two powers of two out again (exact)
+            const float dx = tok < P.n_tok ? __ldg(P.sx + tok) * (1.f / (float)(1 << (16 - XBITS - WBITS))) : 0.f;
             OutT* orow = reinterpret_cast<OutT*>(P.out) + tok * P.out_stride + out0;
 #pragma unroll 1
             for (int h = 0; h < 2; ++h) {
