@@ -14,6 +14,8 @@
 // fp32 inputs.
 #include <cuda_bf16.h>
 
+#include <stdlib.h>
+
 #include "gbs_internal.h"
 
 namespace {
@@ -614,6 +616,139 @@ __global__ void __launch_bounds__(NT) k_dequantize_stream(int d_pad, int glog, i
     }
 }
 
+// The same work with the codes staged through shared memory: a CTA takes tiles of 64 items (16 384 codes, 6 or 8 KB
+// of packed bytes), brought in by 16-byte asynchronous copies three tiles ahead of their use, so that the unpacking
+// threads read their fields from shared memory and never wait on a global load (the direct-load form above is bound
+// by exactly that wait).  The scales (one load per lane and item) are fetched one tile ahead into registers.
+constexpr int DQ_TILE_ITEMS = 64;
+constexpr int DQ_STAGES = 4;
+#ifndef DQ_BLOCKS_PER_SM
+#define DQ_BLOCKS_PER_SM 4
+#endif
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((unsigned)__cvta_generic_to_shared(smem_dst)), "l"(gsrc)
+                 : "memory");
+}
+
+template <typename OutT, int BITS>
+__global__ void __launch_bounds__(NT) k_dequantize_staged(int d_pad, int glog, int spr, int asym, long long total_codes,
+                                                          const unsigned* __restrict__ words,
+                                                          const float* __restrict__ scales, OutT* __restrict__ out)
+{
+    constexpr bool WIDE = sizeof(OutT) == 4;
+    constexpr int PER = WIDE ? 4 : 8;
+    constexpr int NST = WIDE ? 2 : 1;
+    constexpr int IPW = DQ_TILE_ITEMS / (NT / 32);           // items per warp and tile: 8
+    constexpr int TILE_WORDS = DQ_TILE_ITEMS * 8 * BITS;     // 32-bit words of packed codes per tile
+    __shared__ __align__(16) unsigned stage[DQ_STAGES][TILE_WORDS];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const long long n_items = (total_codes + 255) >> 8;
+    const long long n_tiles = (n_items + DQ_TILE_ITEMS - 1) / DQ_TILE_ITEMS;
+    const long long total_chunks = (total_codes * BITS) >> 7;            // 16-byte pieces of the code stream
+    const int amul = asym ? 2 : 1;
+
+    int c_of[NST], w_of[NST], sh_of[NST];
+#pragma unroll
+    for (int h = 0; h < NST; ++h) {
+        c_of[h] = WIDE ? 128 * h + 4 * lane : 8 * lane;
+        w_of[h] = (c_of[h] * BITS) >> 5;
+        sh_of[h] = (c_of[h] * BITS) & 31;
+    }
+    auto fetch = [&](long long tile, int slot) {                          // all threads: the tile's packed bytes
+        if (tile < n_tiles) {
+            const long long chunk0 = tile * (TILE_WORDS / 4);
+            for (int i = threadIdx.x; i < TILE_WORDS / 4; i += NT)
+                if (chunk0 + i < total_chunks) cp_async16(&stage[slot][4 * i], words + 4 * (chunk0 + i));
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    // scale (and zero point) of every group this lane will unpack in a tile: one division per tile, then the
+    // items' rows follow by counting (rows are a whole number of items, or half an item when 128 wide)
+    const int ipr = d_pad >> 8;                                            // items per row (0 for 128-wide rows)
+    auto fetch_scales = [&](long long tile, float (&dl)[IPW][NST], float (&zr)[IPW][NST]) {
+        const long long item0 = tile * DQ_TILE_ITEMS + warp * IPW;
+        long long r = ipr ? item0 / ipr : 2 * item0;
+        int ci = ipr ? (int)(item0 - r * ipr) : 0;
+#pragma unroll
+        for (int u = 0; u < IPW; ++u) {
+#pragma unroll
+            for (int h = 0; h < NST; ++h) {
+                dl[u][h] = 0.f; zr[u][h] = 0.f;
+                if (tile < n_tiles && ((item0 + u) << 8) + c_of[h] < total_codes) {
+                    const long long rr = ipr ? r : r + (c_of[h] >> 7);
+                    const int cc = ipr ? (ci << 8) + c_of[h] : (c_of[h] & 127);
+                    const float* sp = scales + (rr * spr + (cc >> glog)) * amul;
+                    dl[u][h] = __ldg(sp);
+                    if (asym) zr[u][h] = __ldg(sp + 1);
+                }
+            }
+            if (ipr) { if (++ci == ipr) { ci = 0; ++r; } } else r += 2;
+        }
+    };
+
+    long long tile = blockIdx.x;
+    const long long tstride = gridDim.x;
+#pragma unroll
+    for (int j = 0; j < DQ_STAGES - 1; ++j) fetch(tile + j * tstride, j);
+    float dl[IPW][NST], zr[IPW][NST], dl_n[IPW][NST], zr_n[IPW][NST];
+    fetch_scales(tile, dl, zr);
+    for (int it = 0; tile < n_tiles; tile += tstride, ++it) {
+        fetch(tile + (DQ_STAGES - 1) * tstride, (it + DQ_STAGES - 1) % DQ_STAGES);
+        fetch_scales(tile + tstride, dl_n, zr_n);
+        asm volatile("cp.async.wait_group %0;" ::"n"(DQ_STAGES - 1) : "memory");
+        __syncthreads();
+        const unsigned* sw = stage[it % DQ_STAGES];
+#pragma unroll
+        for (int u = 0; u < IPW; ++u) {
+            const long long item = tile * DQ_TILE_ITEMS + warp * IPW + u;
+#pragma unroll
+            for (int h = 0; h < NST; ++h) {
+                if ((item << 8) + c_of[h] >= total_codes) continue;
+                const int widx = (warp * IPW + u) * (8 * BITS) + w_of[h];
+                const unsigned lo = sw[widx];
+                const unsigned hi = sw[widx + 1 < TILE_WORDS ? widx + 1 : widx];
+                unsigned nib = __funnelshift_r(lo, hi, sh_of[h]);
+                if (BITS == 3) {
+                    nib = (nib & 0x00000fffu) | ((nib & 0x00fff000u) << 4);
+                    nib = (nib & 0x003f003fu) | ((nib & 0x0fc00fc0u) << 2);
+                    nib = (nib & 0x07070707u) | ((nib & 0x38383838u) << 1);
+                }
+                constexpr unsigned SIGNS = BITS == 3 ? 0x44444444u : 0x88888888u;
+                constexpr float OFF = BITS == 3 ? 4.f : 8.f;
+                if (!asym) nib ^= SIGNS;
+                const unsigned even = nib & 0x0f0f0f0fu, odd = (nib >> 4) & 0x0f0f0f0fu;
+                const float bias = 8388608.f + (asym ? 0.f : OFF);
+                float v[PER];
+#pragma unroll
+                for (int e = 0; e < PER; ++e) {
+                    const unsigned fb = __byte_perm((e & 1) ? odd : even, 0x4B000000u, 0x7440u + (unsigned)(e >> 1));
+                    v[e] = fmaf(__uint_as_float(fb) - bias, dl[u][h], zr[u][h]);
+                }
+                OutT* dst = out + (item << 8) + c_of[h];
+                if (WIDE) {
+                    *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+                } else {
+                    unsigned o[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        __nv_bfloat162 b2 = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+                        o[e] = *reinterpret_cast<unsigned*>(&b2);
+                    }
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(o[0], o[1], o[2], o[3]);
+                }
+            }
+        }
+        __syncthreads();                                  // the slot refilled next is the one just read
+#pragma unroll
+        for (int u = 0; u < IPW; ++u)
+#pragma unroll
+            for (int h = 0; h < NST; ++h) { dl[u][h] = dl_n[u][h]; zr[u][h] = zr_n[u][h]; }
+    }
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
 // xhat = (H^T yhat / sqrt(d'))[0:d]: same shared-memory machinery with the transposed H_m.
 template <typename OutT, int BITS, bool WIDE>
 __global__ void __launch_bounds__(NT) k_dequantize_inverse(GenericParams P, const unsigned char* __restrict__ codes,
@@ -807,8 +942,18 @@ int gbs_generic_dequantize(const gbs_plan* p, const void* codes, const float* sc
         const int grid = (int)(blocks < cap ? blocks : cap);
         int glog = 31;                               // one scale per row: every column maps to scale 0
         if (p->group) { glog = 0; while ((1 << glog) < p->group) ++glog; }
+        const long long tiles = (items + DQ_TILE_ITEMS - 1) / DQ_TILE_ITEMS;
+        const long long cap2 = (long long)p->sm_count * DQ_BLOCKS_PER_SM;
+        const int grid2 = (int)(tiles < cap2 ? tiles : cap2);
+        // the staged form pays a three-tile prologue per block: it wins once a block has a few tiles to work through
+        // (and always for 4-byte outputs, where the direct form holds too few bytes in flight); measured crossover
+        const bool staged = out_dtype == GBS_DTYPE_F32 || 2 * tiles >= 5 * cap2;
 #define LAUNCH_DS(T, B)                                                                            \
     do {                                                                                           \
+        if (staged)                                                                                \
+            k_dequantize_staged<T, B><<<grid2, NT, 0, stream>>>(P.d_pad, glog, P.spr, P.asym, total,\
+                                                               (const unsigned*)codes, scales, (T*)out); \
+        else                                                                                       \
         k_dequantize_stream<T, B><<<grid, NT, 0, stream>>>(P.d_pad, glog, P.spr, P.asym, total,     \
                                                            (const unsigned*)codes, scales, (T*)out); \
         e = cudaGetLastError();                                                                    \

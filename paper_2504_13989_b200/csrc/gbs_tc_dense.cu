@@ -275,11 +275,16 @@ int gbs_tc_dense_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_row
     P.status = p->d_status;
     const int smem = (int)sizeof(Smem) + 1024;
     {
+        // opt in to the large dynamic shared memory once per device (not a stream operation)
         static std::mutex mu;
+        static bool done[64] = {false};
         std::lock_guard<std::mutex> lock(mu);
-        cudaError_t e = cudaFuncSetAttribute(k_tc_dense_rq<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_dense_rq<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return (int)e;
+        if (!(p->device >= 0 && p->device < 64 && done[p->device])) {
+            cudaError_t e = cudaFuncSetAttribute(k_tc_dense_rq<3>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            if (e == cudaSuccess) e = cudaFuncSetAttribute(k_tc_dense_rq<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+            if (e != cudaSuccess) return (int)e;
+            if (p->device >= 0 && p->device < 64) done[p->device] = true;
+        }
     }
     const int grid = P.n_tiles < p->sm_count ? P.n_tiles : p->sm_count;
     if (p->bits == 3) k_tc_dense_rq<3><<<grid, THREADS, smem, stream>>>(xmap, hmap, P);

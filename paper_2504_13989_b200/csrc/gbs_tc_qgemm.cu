@@ -382,11 +382,17 @@ extern "C" int gbs_quantized_matmul(const gbs_plan_t* px, const void* codes_x, c
     const int smem = (int)sizeof(Smem) + 1024;
     QgemmKernel kernel = pick(px->bits, pw->bits, out_dtype);
     {
+        // opt in to the large dynamic shared memory once per device and instantiation (not a stream operation)
         static std::mutex mu;
+        static bool done[64][8] = {{false}};
+        const int ki = (px->bits - 3) * 4 + (pw->bits - 3) * 2 + (out_dtype == GBS_DTYPE_F32 ? 0 : 1);
         std::lock_guard<std::mutex> lock(mu);
-        if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
-            cudaGetLastError();
-            return GBS_ERR_CUDA;
+        if (!(px->device >= 0 && px->device < 64 && done[px->device][ki])) {
+            if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) {
+                cudaGetLastError();
+                return GBS_ERR_CUDA;
+            }
+            if (px->device >= 0 && px->device < 64) done[px->device][ki] = true;
         }
     }
     const dim3 grid((unsigned)((n_out + TN - 1) / TN), (unsigned)((n_tokens + TM - 1) / TM));
