@@ -82,3 +82,40 @@ def test_calibration_layer_clip_error_sampled_rows(layer):
         np.testing.assert_allclose(err.cpu().numpy(), rows.double().sum(dim=0).cpu().numpy(), rtol=TOL_CLIP)
         # the sampled rows' totals agree with the oracle's totals to the tolerance of the sums
         np.testing.assert_allclose(rows[idx.to(DEV)].double().sum(dim=0).cpu().numpy(), eref, rtol=TOL_CLIP)
+
+
+@pytest.mark.parametrize("name,rows,bits,asym,dtype", [
+    ("llama4096", 20000, 3, False, torch.bfloat16),      # large enough for the shared-memory-staged form, ragged tile
+    ("llama4096", 20000, 4, False, torch.float32),
+    ("kv128", 300001, 3, True, torch.bfloat16),          # 128-wide rows (an item spans two rows), odd row count
+    ("qwen3584", 9000, 3, False, torch.bfloat16),        # per-group scales, width not a power of two
+    ("llama4096", 300, 3, False, torch.bfloat16),        # small launch: the direct form
+])
+def test_rotated_domain_dequantize_at_launch_sizes_of_both_forms(name, rows, bits, asym, dtype):
+    """gbs_dequantize without inverse rotation, yhat = q * Delta (+ lo), at sizes that take the staged form and the
+    direct form of the streaming kernel: every element against the codes and scales unpacked independently."""
+    w = synth.WORKLOADS[name]
+    x = synth.make_device(name, rows, device=DEV)
+    group = 128 if asym else w.group
+    with Plan(w.d, w.d_pad, w.m, bits, group, w.alpha, asymmetric=asym) as plan:
+        codes, scales, _ = plan.rotate_quantize(x)
+        out = torch.full((rows + 1, w.d_pad), float("nan"), dtype=dtype, device=DEV)
+        plan.dequantize(codes, scales, out=out[:rows])
+        torch.cuda.synchronize()
+        assert bool(torch.isnan(out[rows]).all()), "wrote past the last row"
+        g = group or w.d_pad
+        step = 7 if rows > 1000 else 1                      # every seventh row, plus the last rows (the ragged tail)
+        idx = torch.unique(torch.cat([torch.arange(0, rows, step), torch.arange(max(0, rows - 70), rows)])).to(DEV)
+        cb = codes[idx].cpu().numpy()
+        bitsarr = np.unpackbits(cb, axis=1, bitorder="little")[:, : w.d_pad * bits].reshape(len(idx), w.d_pad, bits)
+        f = (bitsarr.astype(np.int32) * (1 << np.arange(bits))).sum(axis=2)
+        sc = scales[idx].cpu().double().numpy()
+        if asym:
+            sc = sc.reshape(len(idx), -1, 2)
+            want = f * np.repeat(sc[:, :, 0], g, axis=1) + np.repeat(sc[:, :, 1], g, axis=1)
+        else:
+            q = np.where(f >= (1 << (bits - 1)), f - (1 << bits), f)
+            want = q * np.repeat(sc, g, axis=1)
+        got = out[idx].cpu().double().numpy()
+        tol = 2e-7 if dtype == torch.float32 else 2.0 ** -8
+        np.testing.assert_allclose(got, want, rtol=tol, atol=1e-30 if not asym else 1e-6 * np.abs(want).max())
