@@ -7,12 +7,14 @@ One STEP = one pass of the fused path over one batch of the headline workload: t
 d=4096 bf16 activation batch, quantized at b=3 and at b=4 (two launches of the fused kernel, as the
 workload names both bit-widths).  Inputs are synthetic, resident in HBM before the timed region; the
 launches rotate over NSETS distinct buffer sets whose footprint exceeds 4x the L2 so every launch
-reads from HBM.  The timed K steps are replayed from CUDA graphs, bracketed by a barrier and a
-device synchronise, timed with CUDA events on the launching stream, max over ranks.
+reads from HBM.  The K steps are replayed from CUDA graphs, bracketed by a barrier and a device
+synchronise, timed with CUDA events on the launching stream, max over ranks; they are repeated whole
+times until the timed region lasts --min-ms (50 ms by default; `steps_timed` says how many ran).
 
 Prints ONE JSON line.  `value` is GB/s of algorithmic bytes (row in, packed codes + scales out).
-Extra keys: `roofline`, `cpu_baseline`, `e2e`, `clocks`, `gpu_launches`, and `also` (the d=3584
-workload and the other entry points, timed outside the K steps, for context).
+Extra keys: `roofline` (d=4096) and `roofline_d3584` (the metric's second width, its own timed loop), each
+with the size-matched plain copy beside the measured peak, `cpu_baseline`, `e2e`, `clocks`, `gpu_launches`,
+and `also` (every other workload and entry point, timed outside the K steps, for context).
 
 The path does not shard: with --gpus N every rank runs an independent replica on its own GPU.
 """
