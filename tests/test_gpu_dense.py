@@ -44,6 +44,27 @@ def test_full_paley_1544_against_the_dense_definition(bits, rows, alpha):
             assert e.value.status == binding.GBS_ERR_UNSUPPORTED
 
 
+def test_full_paley_1544_with_256_token_tiles_sampled_rows():
+    """A batch large enough for the kernel's 256-token tiles (two sub-tiles sharing each chunk of H), with a ragged last
+    tile; sampled rows (first, last, across sub-tile and tile borders) against the oracle's dense definition."""
+    gbs_build.build()
+    rows, bits, alpha = 19000 + 37, 3, 0.9
+    x = _rows(rows, 7)
+    idx = np.unique(np.concatenate([np.arange(0, 6), np.arange(125, 131), np.arange(253, 259), np.arange(9000, 9004),
+                                    np.arange(rows - 40, rows)]))
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(x[idx]), D, M, M, bits, 0, alpha, dense=True)
+    with Plan(D, M, M, bits, 0, alpha) as plan:
+        codes = torch.full((rows + 1, M * bits // 8), 0xEE, dtype=torch.uint8, device=DEV)
+        scales = torch.full((rows + 1, 1), -1.0, dtype=torch.float32, device=DEV)
+        y = torch.empty((rows, M), dtype=torch.float32, device=DEV)
+        binding.gbs_rotate_quantize(plan.handle, x.to(DEV), codes[:rows], scales[:rows], y)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+        assert bool((codes[rows] == 0xEE).all()) and float(scales[rows, 0]) == -1.0, "wrote past the last row"
+        t = torch.from_numpy(idx).to(DEV)
+        compare_rotate_quantize(x[idx], ref, codes[t], scales[t], y[t], bits, 0, M, alpha)
+
+
 def test_full_order_plans_are_validated_on_the_host():
     gbs_build.build()
     lib = binding.lib()
