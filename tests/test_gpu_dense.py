@@ -44,6 +44,22 @@ def test_full_paley_1544_against_the_dense_definition(bits, rows, alpha):
             assert e.value.status == binding.GBS_ERR_UNSUPPORTED
 
 
+@pytest.mark.parametrize("d,m,bits,rows", [(256, 264, 3, 300), (120, 128, 4, 77), (368, 368, 4, 129)])
+def test_other_full_orders_against_the_dense_definition(d, m, bits, rows):
+    """Smaller full orders (263, 127 and 367 are primes = 3 mod 4): a last block of 8 coordinates, a single block, an
+    order without expansion; every row against the oracle's dense definition."""
+    gbs_build.build()
+    rng = np.random.Generator(np.random.PCG64(d + m))
+    x = torch.from_numpy((0.5 * rng.standard_t(3.0, size=(rows, d))).astype(np.float32)).to(torch.bfloat16)
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(x), d, m, m, bits, 0, 0.9, dense=True)
+    with Plan(d, m, m, bits, 0, 0.9) as plan:
+        assert plan.info.variant == 4
+        codes, scales, y = plan.rotate_quantize(x.to(DEV), want_y=True)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+        compare_rotate_quantize(x, ref, codes, scales, y, bits, 0, m, 0.9)
+
+
 def test_full_paley_1544_with_256_token_tiles_sampled_rows():
     """A batch large enough for the kernel's 256-token tiles (two sub-tiles sharing each chunk of H), with a ragged last
     tile; sampled rows (first, last, across sub-tile and tile borders) against the oracle's dense definition."""
