@@ -664,27 +664,35 @@ __global__ void __launch_bounds__(NT) k_dequantize_staged(int d_pad, int glog, i
         }
         asm volatile("cp.async.commit_group;" ::: "memory");
     };
-    // scale (and zero point) of every group this lane will unpack in a tile: one division per tile, then the
-    // items' rows follow by counting (rows are a whole number of items, or half an item when 128 wide)
+    // scale (and zero point) of every group this lane will unpack in a tile.  Rows are contiguous and a group divides a
+    // row, so with groups the scale index is simply (flat code index) >> log2(group); with one scale per row it is the
+    // row, found by one division per tile and counting from there (rows are a whole number of items, or half an item
+    // when 128 wide).
     const int ipr = d_pad >> 8;                                            // items per row (0 for 128-wide rows)
+    const bool per_row = glog >= 31;
     auto fetch_scales = [&](long long tile, float (&dl)[IPW][NST], float (&zr)[IPW][NST]) {
         const long long item0 = tile * DQ_TILE_ITEMS + warp * IPW;
-        long long r = ipr ? item0 / ipr : 2 * item0;
-        int ci = ipr ? (int)(item0 - r * ipr) : 0;
+        const bool whole = (tile + 1) * ((long long)DQ_TILE_ITEMS << 8) <= total_codes;     // no ragged end in this tile
+        long long r = 0;
+        int ci = 0;
+        if (per_row) {
+            r = ipr ? item0 / ipr : 2 * item0;
+            ci = ipr ? (int)(item0 - r * ipr) : 0;
+        }
 #pragma unroll
         for (int u = 0; u < IPW; ++u) {
 #pragma unroll
             for (int h = 0; h < NST; ++h) {
                 dl[u][h] = 0.f; zr[u][h] = 0.f;
-                if (tile < n_tiles && ((item0 + u) << 8) + c_of[h] < total_codes) {
-                    const long long rr = ipr ? r : r + (c_of[h] >> 7);
-                    const int cc = ipr ? (ci << 8) + c_of[h] : (c_of[h] & 127);
-                    const float* sp = scales + (rr * spr + (cc >> glog)) * amul;
+                const long long code = ((item0 + u) << 8) + c_of[h];
+                if (whole || (tile < n_tiles && code < total_codes)) {
+                    const long long si = per_row ? (ipr ? r : r + (c_of[h] >> 7)) : (code >> glog);
+                    const float* sp = scales + si * amul;
                     dl[u][h] = __ldg(sp);
                     if (asym) zr[u][h] = __ldg(sp + 1);
                 }
             }
-            if (ipr) { if (++ci == ipr) { ci = 0; ++r; } } else r += 2;
+            if (per_row) { if (ipr) { if (++ci == ipr) { ci = 0; ++r; } } else r += 2; }
         }
     };
 
@@ -700,12 +708,13 @@ __global__ void __launch_bounds__(NT) k_dequantize_staged(int d_pad, int glog, i
         asm volatile("cp.async.wait_group %0;" ::"n"(DQ_STAGES - 1) : "memory");
         __syncthreads();
         const unsigned* sw = stage[it % DQ_STAGES];
+        const bool whole = (tile + 1) * ((long long)DQ_TILE_ITEMS << 8) <= total_codes;
 #pragma unroll
         for (int u = 0; u < IPW; ++u) {
             const long long item = tile * DQ_TILE_ITEMS + warp * IPW + u;
 #pragma unroll
             for (int h = 0; h < NST; ++h) {
-                if ((item << 8) + c_of[h] >= total_codes) continue;
+                if (!whole && (item << 8) + c_of[h] >= total_codes) continue;
                 const int widx = (warp * IPW + u) * (8 * BITS) + w_of[h];
                 const unsigned lo = sw[widx];
                 const unsigned hi = sw[widx + 1 < TILE_WORDS ? widx + 1 : widx];
