@@ -507,21 +507,35 @@ class HostPipeline:
         self.copy_stream = torch.cuda.Stream(device=device)
         self.ev_in = [torch.cuda.Event() for _ in self.ranges]
         self.ev_start = torch.cuda.Event()
+        # views of the staging buffers and the marshalled arguments of every launch, made once: the per-call host
+        # work is what bounds a pipeline of short launches
+        self.x_views = [self.x_dev[r0:r1] for r0, r1 in self.ranges]
+        self.calls = []
+        dt = _dtype_code(self.x_dev)
+        for (r0, r1), xv in zip(self.ranges, self.x_views):
+            per_plan = []
+            for p, (codes, scales, _) in zip(self.plans, self.outs):
+                cv, sv = codes[r0:r1], scales[r0:r1]
+                per_plan.append((ctypes.c_void_p(p.handle), xv.data_ptr(), dt, r1 - r0, xv.stride(0) if r1 - r0 > 1 else d,
+                                 cv.data_ptr(), sv.data_ptr(), cv, sv))
+            self.calls.append(per_plan)
 
     def run(self, x_host: torch.Tensor, outs_host, stream=None):
         """outs_host: one (codes_host, scales_host) pair per plan.  Work is enqueued on `stream` (and the
         internal copy stream, joined to it); the caller synchronises `stream`."""
         s = stream or torch.cuda.current_stream()
+        sp = int(s.cuda_stream)
+        rq = lib().gbs_rotate_quantize
         self.ev_start.record(s)
         self.copy_stream.wait_event(self.ev_start)          # staging buffers of the previous call are free
         for i, (r0, r1) in enumerate(self.ranges):
             with torch.cuda.stream(self.copy_stream):
-                self.x_dev[r0:r1].copy_(x_host[r0:r1], non_blocking=True)
+                self.x_views[i].copy_(x_host[r0:r1], non_blocking=True)
                 self.ev_in[i].record(self.copy_stream)
             with torch.cuda.stream(s):
                 s.wait_event(self.ev_in[i])
-                for p, (codes, scales, _), (ch, sh) in zip(self.plans, self.outs, outs_host):
-                    gbs_rotate_quantize(p.handle, self.x_dev[r0:r1], codes[r0:r1], scales[r0:r1], None, s)
-                    ch[r0:r1].copy_(codes[r0:r1], non_blocking=True)
-                    sh[r0:r1].copy_(scales[r0:r1], non_blocking=True)
+                for (h, xp, dt, n, stride, cp, scp, cv, sv), (ch, sh) in zip(self.calls[i], outs_host):
+                    _check(rq(h, xp, dt, n, stride, cp, scp, None, sp), "gbs_rotate_quantize")
+                    ch[r0:r1].copy_(cv, non_blocking=True)
+                    sh[r0:r1].copy_(sv, non_blocking=True)
         return outs_host
