@@ -98,8 +98,9 @@ typedef struct gbs_plan_info {
  *           Full orders: d_pad = m (2^k = 1) is accepted when m - 1 is a prime = 3 mod 4, m a multiple of 8 and
  *           128 <= m <= 4096 -- the rotation is then the Paley matrix H_m itself, e.g. d = 1536, d_pad = m = 1544
  *           (Section 5.2.2).  Such plans take bf16 rows with d a multiple of 8 and group = 0, run as a dense
- *           tensor-core contraction, and support gbs_rotate_quantize and gbs_dequantize without inverse rotation;
- *           the other calls return GBS_ERR_UNSUPPORTED for them.
+ *           tensor-core contraction, and support gbs_rotate_quantize and gbs_dequantize (both forms; the inverse
+ *           rotation is a dense contraction too); gbs_clip_error and the searches return GBS_ERR_UNSUPPORTED
+ *           for them.
  *   bits    3 or 4
  *   group   0, or a power of two >= 8 dividing 2^k (so a group never straddles a block of H_m)
  *   alpha   0 < alpha <= 1

@@ -285,7 +285,7 @@ extern "C" int gbs_dequantize(const gbs_plan_t* p, const void* codes, const floa
     if (out_dtype != GBS_DTYPE_F32 && out_dtype != GBS_DTYPE_BF16) return GBS_ERR_INVALID_ARG;
     if (flags & ~GBS_INVERSE_ROTATE) return GBS_ERR_INVALID_ARG;
     if (n_rows < 0) return GBS_ERR_INVALID_ARG;
-    if ((flags & GBS_INVERSE_ROTATE) && p->variant == GBS_VARIANT_TC_DENSE) return GBS_ERR_UNSUPPORTED;
+    if ((flags & GBS_INVERSE_ROTATE) && p->variant == GBS_VARIANT_TC_DENSE && !gbs_tc_denseinv_supported(p)) return GBS_ERR_UNSUPPORTED;
     if (n_rows == 0) return GBS_OK;
     if (!codes || !scales || !out) return GBS_ERR_INVALID_ARG;
     if (!aligned16(codes) || !aligned16(out) || (reinterpret_cast<uintptr_t>(scales) & 3u))
@@ -293,7 +293,9 @@ extern "C" int gbs_dequantize(const gbs_plan_t* p, const void* codes, const floa
     DeviceGuard g;
     if (g.enter(p->device) != cudaSuccess) { cudaGetLastError(); return GBS_ERR_CUDA; }
     int e;
-    if ((flags & GBS_INVERSE_ROTATE) && gbs_tc_uvinv_supported(p))
+    if ((flags & GBS_INVERSE_ROTATE) && p->variant == GBS_VARIANT_TC_DENSE)
+        e = gbs_tc_denseinv_dequantize(p, codes, scales, n_rows, out, out_dtype, static_cast<cudaStream_t>(cuda_stream));
+    else if ((flags & GBS_INVERSE_ROTATE) && gbs_tc_uvinv_supported(p))
         e = gbs_tc_uvinv_dequantize(p, codes, scales, n_rows, out, out_dtype, static_cast<cudaStream_t>(cuda_stream));
     else if ((flags & GBS_INVERSE_ROTATE) && gbs_tc_rowinv_supported(p, scales))
         e = gbs_tc_rowinv_dequantize(p, codes, scales, n_rows, out, out_dtype, static_cast<cudaStream_t>(cuda_stream));

@@ -112,6 +112,11 @@ void gbs_tc_dense_image(const int8_t* hm, int m, unsigned short* img);
 int gbs_tc_dense_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
                                  float* scales, float* y_opt, cudaStream_t stream);
 
+// gbs_tc_denseinv.cu : gbs_dequantize with inverse rotation for the full order
+bool gbs_tc_denseinv_supported(const gbs_plan* p);
+int gbs_tc_denseinv_dequantize(const gbs_plan* p, const void* codes, const float* scales, int64_t n_rows, void* out,
+                               int out_dtype, cudaStream_t stream);
+
 // gbs_tc_row.cu
 bool gbs_tc_row_supported(const gbs_plan* p);
 int gbs_tc_row_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,

@@ -37,11 +37,20 @@ def test_full_paley_1544_against_the_dense_definition(bits, rows, alpha):
         yhat = plan.dequantize(codes, scales)
         q = unpack_codes(codes.cpu().numpy(), M, bits)
         np.testing.assert_allclose(yhat.cpu().double().numpy(), q * scales.cpu().double().numpy(), rtol=2e-7, atol=0)
+        # back to the input domain: xhat = (H^T yhat / sqrt(m))[0:d] against the oracle on the GPU's own codes and scales
+        want = oracle.dequantize_rows(codes.cpu().numpy(), scales.cpu().double().numpy(), D, M, M, bits, 0, inverse=True)
+        for dtype, tol in ((torch.float32, 2e-7), (torch.bfloat16, 2.0 ** -8)):
+            xhat = torch.full((rows + 1, D), float("nan"), dtype=dtype, device=DEV)
+            plan.dequantize(codes, scales, inverse=True, out=xhat[:rows])
+            torch.cuda.synchronize()
+            assert plan.device_status() == 0 and bool(torch.isnan(xhat[rows]).all())
+            got = xhat[:rows].cpu().double().numpy()
+            err = np.linalg.norm(got - want, axis=1) / np.maximum(np.linalg.norm(want, axis=1), 1e-300)
+            assert err.max() <= tol, err.max()
         # what this family does not serve is refused, not faulted
-        for call in (lambda: plan.clip_error(x.to(DEV), [0.5, 1.0]), lambda: plan.dequantize(codes, scales, inverse=True)):
-            with pytest.raises(binding.GbsError) as e:
-                call()
-            assert e.value.status == binding.GBS_ERR_UNSUPPORTED
+        with pytest.raises(binding.GbsError) as e:
+            plan.clip_error(x.to(DEV), [0.5, 1.0])
+        assert e.value.status == binding.GBS_ERR_UNSUPPORTED
 
 
 @pytest.mark.parametrize("d,m,bits,rows", [(256, 264, 3, 300), (120, 128, 4, 77), (368, 368, 4, 129)])
@@ -58,6 +67,12 @@ def test_other_full_orders_against_the_dense_definition(d, m, bits, rows):
         torch.cuda.synchronize()
         assert plan.device_status() == 0
         compare_rotate_quantize(x, ref, codes, scales, y, bits, 0, m, 0.9)
+        # and back: widths that are not a multiple of the kernel's 256-coordinate output blocks
+        want = oracle.dequantize_rows(codes.cpu().numpy(), scales.cpu().double().numpy(), d, m, m, bits, 0, inverse=True)
+        got = plan.dequantize(codes, scales, inverse=True).cpu().double().numpy()
+        assert got.shape == (rows, d) and plan.device_status() == 0
+        err = np.linalg.norm(got - want, axis=1) / np.maximum(np.linalg.norm(want, axis=1), 1e-300)
+        assert err.max() <= 2e-7, err.max()
 
 
 def test_full_paley_1544_with_256_token_tiles_sampled_rows():
