@@ -145,7 +145,10 @@ extern "C" int gbs_plan_create_ex(gbs_plan_t** out, int d, int d_pad, int m, int
         // the UV family with one symmetric scale per token also gets the image of the transpose, behind the
         // first one in the same allocation, for gbs_dequantize's inverse rotation on the tensor cores
         const bool with_t = tc_uv && p->group == 0 && !p->asym;
-        const size_t img_bytes = with_t ? 65536 : 32768;
+        // the wide family keeps the UVM image (clip scoring) and, where the register-resident kernel applies, its image
+        const char* no_uvr = getenv("GBS_NO_UVR");
+        const bool uvr = uvm_glog != 0 && !(no_uvr && no_uvr[0] == '1') && gbs_tc_uvr_supported(p);
+        const size_t img_bytes = with_t ? 65536 : (uvr ? 32768 + (size_t)gbs_tc_uvr_image_bytes(p) : 32768);
         unsigned char* img = (unsigned char*)malloc(img_bytes);
         if (!img) { cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC; }
         if (tc_uv) gbs_tc_uv_a_image(p, img);
@@ -164,16 +167,18 @@ extern "C" int gbs_plan_create_ex(gbs_plan_t** out, int d, int d_pad, int m, int
         }
         else if (tc_row) gbs_tc_sign_image(p->h_hm, 1, 7, 128, img);     // H_128 itself
         else gbs_tc_sign_image(p->h_hm, p->m, p->k - 5 - uvm_glog, p->d_pad >> (5 + uvm_glog), img);
+        if (uvr) gbs_tc_uvr_image(p, img + 32768);
         e = cudaMalloc(&p->d_aimg, img_bytes);
         if (e == cudaSuccess) e = cudaMemcpy(p->d_aimg, img, img_bytes, cudaMemcpyHostToDevice);
         free(img);
         if (e == cudaSuccess && with_t) p->d_aimg_t = p->d_aimg + 32768;
+        if (e == cudaSuccess && uvr) p->d_aimg_r = p->d_aimg + 32768;
         if (e != cudaSuccess) {
             cudaGetLastError();
             if (p->d_aimg) cudaFree(p->d_aimg);
             cudaFree(p->d_status); delete p; return GBS_ERR_ALLOC;
         }
-        p->variant = tc_uv ? GBS_VARIANT_TC_UV : (tc_row ? GBS_VARIANT_TC_ROW : GBS_VARIANT_TC_UVM);
+        p->variant = tc_uv ? GBS_VARIANT_TC_UV : (tc_row ? GBS_VARIANT_TC_ROW : (uvr ? GBS_VARIANT_TC_UVR : GBS_VARIANT_TC_UVM));
         p->uvm_glog = uvm_glog;
     }
     if (p->asym && p->variant != GBS_VARIANT_TC_ROW) {          // only the row family has the asymmetric quantizer
@@ -268,6 +273,8 @@ extern "C" int gbs_rotate_quantize(const gbs_plan_t* p, const void* x, int x_dty
         e = gbs_tc_dense_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
     else if (p->variant == GBS_VARIANT_TC_UV && x_dtype == GBS_DTYPE_BF16)
         e = gbs_tc_uv_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
+    else if (p->variant == GBS_VARIANT_TC_UVR && x_dtype == GBS_DTYPE_BF16)
+        e = gbs_tc_uvr_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
     else if (p->variant == GBS_VARIANT_TC_UVM && x_dtype == GBS_DTYPE_BF16)
         e = gbs_tc_uvm_rotate_quantize(p, x, n_rows, x_row_stride, codes, scales, y_opt, stream);
     else if (p->variant == GBS_VARIANT_TC_ROW && x_dtype == GBS_DTYPE_BF16)
@@ -334,7 +341,7 @@ extern "C" int gbs_clip_error(const gbs_plan_t* p, const void* x, int x_dtype, i
     else if (p->variant == GBS_VARIANT_TC_ROW && x_dtype == GBS_DTYPE_BF16)
         e = gbs_tc_row_clip_error(p, x, n_rows, x_row_stride, alphas_host, K, err_sum, err_rows_opt,
                                   static_cast<cudaStream_t>(cuda_stream));
-    else if (p->variant == GBS_VARIANT_TC_UVM && x_dtype == GBS_DTYPE_BF16)
+    else if ((p->variant == GBS_VARIANT_TC_UVM || p->variant == GBS_VARIANT_TC_UVR) && x_dtype == GBS_DTYPE_BF16)
         e = gbs_tc_uvm_clip_error(p, x, n_rows, x_row_stride, alphas_host, K, err_sum, err_rows_opt,
                                   static_cast<cudaStream_t>(cuda_stream));
     else

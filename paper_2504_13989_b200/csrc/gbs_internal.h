@@ -14,6 +14,7 @@ enum gbs_variant {
     GBS_VARIANT_GENERIC = 0,   // shared-memory FWHT on the plain ALUs; any supported (m, k), any dtype
     GBS_VARIANT_TC_UVM = 3,    // 4096 < d' = 32*G*U <= 32768, G in {2,4,8}: tensor cores + two register sweeps over TMEM
     GBS_VARIANT_TC_ROW = 2,    // d' = 128 (KV rows): X * H_128 on tcgen05 tensor cores, one thread owns one row
+    GBS_VARIANT_TC_UVR = 5,    // 4096 < d' = 128*U <= 32768, 80 <= U <= 256: tensor cores + the rest of the transform in registers
     GBS_VARIANT_TC_DENSE = 4,  // d' = m, a full Paley order (k = 0): X * H_m^T as a dense tcgen05 contraction, two sweeps
     GBS_VARIANT_TC_UV = 1,     // d' = U*32, U = m*2^j <= 128: (H_m (x) H_{2^j}) on tcgen05 tensor cores + H_32 in
                                // registers (bf16 rows)
@@ -36,6 +37,7 @@ struct gbs_plan {
     int asym;              // asymmetric quantizer (GBS_PLAN_ASYMMETRIC)
     int uvm_glog;          // UVM family: log2 of the number of 32-value chunks per tensor-core output row
     unsigned char* d_aimg; // device: pre-swizzled bf16 image of H_m (x) H_{2^j} for the tensor-core family (32 KB)
+    unsigned char* d_aimg_r; // device: image of H_m (x) H_{2^j} for the UVR family (behind the first one), or null
     unsigned char* d_aimg_t; // device: image of its transpose (UV family, one scale per token: inverse rotation), or null
     int a_colsum[128];     // column sums of H_m (x) H_{2^j} (UV family), for the inverse path's offset correction
     int* d_status;         // device status word: 0, or the code of the first bounded wait that expired
@@ -105,6 +107,13 @@ int gbs_tc_uvm_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
                                float* scales, float* y_opt, cudaStream_t stream);
 int gbs_tc_uvm_clip_error(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, const float* alphas, int K,
                           double* err_sum, float* err_rows, cudaStream_t stream);
+
+// gbs_tc_uvr.cu : rotate-quantize for wide rows with the register-resident epilogue (clip scoring stays with UVM)
+bool gbs_tc_uvr_supported(const gbs_plan* p);
+int gbs_tc_uvr_image_bytes(const gbs_plan* p);
+void gbs_tc_uvr_image(const gbs_plan* p, unsigned char* img);
+int gbs_tc_uvr_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows, int64_t stride, void* codes,
+                               float* scales, float* y_opt, cudaStream_t stream);
 
 // gbs_tc_dense.cu
 bool gbs_tc_dense_supported(const gbs_plan* p);

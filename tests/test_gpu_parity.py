@@ -297,7 +297,7 @@ def test_wide_family_shapes(d, d_pad, m, bits, alpha, rows, group):
     x = torch.from_numpy(xs.astype(np.float32)).to(torch.bfloat16)
     ref = oracle.rotate_quantize_rows(synth.to_oracle_array(x), d, d_pad, m, bits, group, alpha)
     with Plan(d, d_pad, m, bits, group, alpha) as plan:
-        assert plan.info.variant == 3, "the wide tensor-core family must be the one that runs for this plan"
+        assert plan.info.variant in (3, 5), "a wide tensor-core family must be the one that runs for this plan"
         codes, scales, y = _run_rq(plan, x.to(DEV), rows)
         assert plan.device_status() == 0
         stats = compare_rotate_quantize(x, ref, codes, scales, y, bits, group, d_pad)
