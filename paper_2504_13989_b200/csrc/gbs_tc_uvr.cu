@@ -46,10 +46,12 @@ constexpr int CTL_BYTES = 1024;
 
 struct Ctl {
     unsigned long long full[MAX_SLICES], empty[MAX_SLICES];
-    // tfull[s]: accumulator stage s written, for the warps of the first block (each of them sees every phase of the
-    // one stage it reads: a parity wait must never skip a phase); tfull2[t mod 4]: the same event for the warps of the
-    // second block, which take every second or fourth token.
-    unsigned long long tfull[4], tfull2[4], tempty[4], tbar[TSLOTS];
+    // A parity wait must never skip a phase of its barrier, so every barrier is indexed such that whoever waits on it
+    // takes part in each of its phases.  tfull[t mod 12]: the accumulators of token t are written (U <= 128: tokens
+    // twelve apart have the same issuing thread, the same epilogue warps and the same accumulator stage; U > 128:
+    // only indices 0 and 1 are used, by the warps of the first block); tfull2[t mod 4]: the same event for the warps of
+    // the second block, which take every second or fourth token; tempty[stage]: the stage has been read.
+    unsigned long long tfull[12], tfull2[4], tempty[4], tbar[TSLOTS];
     unsigned long long abar;
     __align__(16) float red[TSLOTS][8];          // [slot][slab]: max|.| of the slab (one scale per token)
     unsigned tmem_base;
@@ -163,16 +165,17 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvr_rq(const __grid_constant_
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n_tok = (int)P.n_rows;
     constexpr int tstride = TWO ? 2 * NCOLS : NCOLS;          // accumulator columns per token
-    // accumulator stages: two tokens of two blocks, or three tokens of one block (one stage per warp of a quadrant)
-    constexpr int tstages = TWO ? 2 : 3;
+    // accumulator stages: two tokens of two blocks, or four tokens of one block
+    constexpr int tstages = TWO ? 2 : 4;
+    constexpr int nfull = TWO ? 2 : 12;                       // tfull barriers in use
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < MAX_SLICES; ++s) {
             mbar_init(&S->full[s], 1);
             mbar_init(&S->empty[s], TWO ? 2 : 1);          // one commit per thread that contracts the slice
         }
+        for (int s = 0; s < 12; ++s) mbar_init(&S->tfull[s], 1);
         for (int s = 0; s < 4; ++s) {
-            mbar_init(&S->tfull[s], 1);
             mbar_init(&S->tfull2[s], 1);
             mbar_init(&S->tempty[s], (unsigned)P.slabs);
         }
@@ -231,10 +234,10 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvr_rq(const __grid_constant_
             const unsigned atom_jump = (unsigned)(P.atom_stride - 96) >> 4;     // from the last k-step of an atom to the next atom
             const bool odd = (P.ksteps & 1) != 0;                               // the last slice holds one k-step
             bool ok = mbar_wait_inline(&S->abort_flag, &S->abar, 0, P.status, 6);
-            int s = 0, it = 0, ts = 0;
+            int s = 0, it = 0, ts = 0, tf = 0;
             unsigned ph = 0, tph = 0;                 // tph: parity of the use count of stage ts
             for (int tk = blockIdx.x; ok && tk < n_tok; tk += gridDim.x, ++it, ts = (ts + 1 == tstages ? 0 : ts + 1),
-                                                         tph ^= (ts == 0 ? 1u : 0u)) {
+                                                         tph ^= (ts == 0 ? 1u : 0u), tf = (tf + 1 == nfull ? 0 : tf + 1)) {
                 if (!TWO && (it & 1) != issuer) {     // the other thread's token: step over its slices
                     for (int j = 0; j < P.nslices; ++j)
                         if (++s == P.n_ring) { s = 0; ph ^= 1; }
@@ -259,7 +262,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvr_rq(const __grid_constant_
                     umma_commit(&S->empty[s]);
                     if (++s == P.n_ring) { s = 0; ph ^= 1; }
                 }
-                if (ok) umma_commit((TWO && issuer) ? &S->tfull2[it & 3] : &S->tfull[ts]);
+                if (ok) umma_commit((TWO && issuer) ? &S->tfull2[it & 3] : &S->tfull[tf]);
             }
         }
       }
@@ -273,10 +276,11 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvr_rq(const __grid_constant_
         const int q = warp & 3;                   // TMEM lane quadrant this warp may access
         const int pr = (warp - 4) >> 2;           // which of the quadrant's three warps
         const unsigned tq = tmem_base + ((unsigned)(q * 32) << 16);
-        int it = 0, ts = 0, tb = 0;
-        unsigned tph = 0, tb_ph = 0;
+        int it = 0, ts = 0, tb = 0, tf = 0, set = 0;
+        unsigned tf_ph = 0, tb_ph = 0;
         for (long long row = blockIdx.x; row < P.n_rows;
-             row += gridDim.x, ++it, ts = (ts + 1 == tstages ? 0 : ts + 1), tph ^= (ts == 0 ? 1u : 0u),
+             row += gridDim.x, ++it, ts = (ts + 1 == tstages ? 0 : ts + 1), set = (set == 2 ? 0 : set + 1),
+                       tf = (tf + 1 == nfull ? 0 : tf + 1), tf_ph ^= (tf == 0 ? 1u : 0u),
                        tb = (tb + 1 == (TWO ? 4 : TSLOTS) ? 0 : tb + 1), tb_ph ^= (tb == 0 ? 1u : 0u)) {
             int slab = -1;
             if (TWO) {
@@ -286,7 +290,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvr_rq(const __grid_constant_
                     const int rel = q - rot_of(it, P.nb2);
                     if (rel >= 0 && rel < P.nb2) slab = 4 + rel;              // second block
                 }
-            } else if (ts == pr && q * 32 < P.U) {
+            } else if (set == pr && q * 32 < P.U) {
                 slab = q;
             }
             if (slab < 0) continue;
@@ -295,7 +299,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvr_rq(const __grid_constant_
             if (TWO && slab >= 4) {
                 if (!mbar_wait_inline(&S->abort_flag, &S->tfull2[it & 3], (it >> 2) & 1, P.status, 4)) break;
             } else {
-                if (!mbar_wait_inline(&S->abort_flag, &S->tfull[ts], tph, P.status, 4)) break;
+                if (!mbar_wait_inline(&S->abort_flag, &S->tfull[tf], tf_ph, P.status, 4)) break;
             }
             tc_fence_after();
             const unsigned tcol = tq + ts * tstride + (slab >= 4 ? NCOLS : 0);

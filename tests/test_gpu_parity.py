@@ -320,6 +320,33 @@ def test_wide_family_shapes(d, d_pad, m, bits, alpha, rows, group):
         np.testing.assert_allclose(erows.cpu().double().numpy(), rref, rtol=1e-4, atol=1e-12)
 
 
+@pytest.mark.parametrize("d,d_pad,m,bits,group", [
+    (16384, 16384, 1, 3, 0), (12288, 12288, 12, 4, 128), (14336, 14336, 28, 3, 0), (24576, 24576, 24, 4, 0),
+    (28672, 28672, 28, 3, 512), (32768, 32768, 1, 4, 0), (18944, 20480, 20, 3, 1024),
+])
+def test_wide_family_many_tokens_per_block(d, d_pad, m, bits, group):
+    """A batch that gives every block a dozen tokens and more (the accumulator stages, the shared-memory ring and
+    the rendezvous slots of the register-resident kernel all wrap several times): sampled rows against the oracle,
+    and the whole batch against a second run."""
+    rows = 148 * 13 + 5
+    g = torch.Generator().manual_seed(d + m + bits + group)
+    x = (torch.randn((rows, d), generator=g) * torch.rand((rows, 1), generator=g) * 3).to(torch.bfloat16)
+    x[7, :] = 0
+    pick = np.unique(np.concatenate([np.arange(4), np.arange(rows - 4, rows),
+                                     np.random.Generator(np.random.PCG64(rows + d)).integers(0, rows, 24), [7, 148, 149, 295, 296]]))
+    xs = x[pick].contiguous()
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(xs), d, d_pad, m, bits, group, 0.9)
+    with Plan(d, d_pad, m, bits, group, 0.9) as plan:
+        assert plan.info.variant in (3, 5)
+        codes, scales, y = _run_rq(plan, x.to(DEV), rows)
+        assert plan.device_status() == 0
+        idx = torch.from_numpy(pick).to(DEV)
+        print(compare_rotate_quantize(xs, ref, codes[idx], scales[idx], y[idx], bits, group, d_pad))
+        codes2, scales2, _ = _run_rq(plan, x.to(DEV), rows, want_y=False)
+        assert torch.equal(codes, codes2) and torch.equal(scales, scales2)
+        assert plan.device_status() == 0
+
+
 ROW_SHAPES = [
     # d, bits, group, alpha, rows, stride
     (128, 3, 0, 1.0, 1, 128),
