@@ -61,14 +61,14 @@ static_assert(sizeof(Ctl) <= CTL_BYTES, "control block");
 
 struct UvrParams {
     long long n_rows;
-    int U;                        // m * 2^j, a multiple of 16
+    int U;                        // m * 2^j
     int slabs;                    // ceil(U / 32)
     int nb2;                      // slabs of the second block (0 .. 4)
-    int ksteps;                   // U / 16
+    int ksteps;                   // ceil(U / 16): the contraction is padded with zero columns of A and zero rows of X
     int nslices;                  // ceil(U / 32)
     int n_ring;                   // slices of shared memory in use
     int a_bytes;                  // image of A
-    int atom_stride;              // bytes between the 64-column K atoms of the image: U * 128
+    int atom_stride;              // bytes between the 64-column K atoms of the image: U (rounded up to 8) * 128
     int code_row_bytes;
     int d_pad;
     int gsh;                      // GROUPED: scale group = 2^gsh chunks of 32 coordinates
@@ -393,6 +393,7 @@ int log2_chunks(int group)
     return gsh;
 }
 
+int image_rows(int U) { return (U + 7) & ~7; }             // lines per K atom: whole 8-line swizzle groups
 int image_rows_last(int U) { return U > 128 ? 256 : 128; }
 int image_atoms(int U) { return (U + 63) / 64; }
 
@@ -430,7 +431,7 @@ cudaError_t launch(int device, int grid, int smem, cudaStream_t stream, bool pdl
 int gbs_tc_uvr_image_bytes(const gbs_plan* p)
 {
     const int U = p->d_pad / NCOLS;
-    return ((image_atoms(U) - 1) * U + image_rows_last(U)) * 128;
+    return ((image_atoms(U) - 1) * image_rows(U) + image_rows_last(U)) * 128;
 }
 
 // Image of A = H_m (x) H_{2^j} (U x U, bf16 +-1, K-major, 128-byte swizzle), zero beyond U.
@@ -444,7 +445,7 @@ void gbs_tc_uvr_image(const gbs_plan* p, unsigned char* img)
             int sign = p->h_hm[(r >> j) * m + (k >> j)];
             if (__builtin_popcount((unsigned)(r & k & jm)) & 1) sign = -sign;
             const int atom = k >> 6, c = (k >> 3) & 7, e = k & 7;
-            const size_t off = (size_t)atom * U * 128 + (size_t)r * 128 + (size_t)((c ^ (r & 7)) << 4) + e * 2;
+            const size_t off = (size_t)atom * image_rows(U) * 128 + (size_t)r * 128 + (size_t)((c ^ (r & 7)) << 4) + e * 2;
             h[off / 2] = sign < 0 ? 0xBF80 : 0x3F80;
         }
 }
@@ -453,7 +454,7 @@ bool gbs_tc_uvr_supported(const gbs_plan* p)
 {
     if (p->asym || p->d_pad <= 4096 || p->d_pad % NCOLS != 0 || p->d % NCOLS != 0 || p->k < 7) return false;
     const int U = p->d_pad / NCOLS;
-    if (U > UMAX || U < 80 || U % 16 != 0) return false;
+    if (U > UMAX || U < 80) return false;          // U = m 2^j is a multiple of 4; fewer than 80 rows leave lane quadrants idle
     if (p->group != 0) {
         if (p->group < V || (p->group & (p->group - 1)) != 0 || p->group > 4096) return false;
     }
@@ -485,10 +486,10 @@ int gbs_tc_uvr_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
     P.U = U;
     P.slabs = (U + 31) / 32;
     P.nb2 = P.slabs > 4 ? P.slabs - 4 : 0;
-    P.ksteps = U / 16;
+    P.ksteps = (U + 15) / 16;
     P.nslices = (U + 31) / 32;
     P.a_bytes = gbs_tc_uvr_image_bytes(p);
-    P.atom_stride = U * 128;
+    P.atom_stride = image_rows(U) * 128;
     int ring = (p->smem_optin - 1024 - CTL_BYTES - P.a_bytes) / SLICE_BYTES;
     P.n_ring = ring < MAX_SLICES ? ring : MAX_SLICES;
     P.code_row_bytes = p->d_pad * p->bits / 8;
