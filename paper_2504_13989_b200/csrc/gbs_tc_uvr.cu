@@ -325,7 +325,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvr_rq(const __grid_constant_
             mc[3] = fwht32_absmax(r3);
             if (!lane_live) mc[0] = mc[1] = mc[2] = mc[3] = 0.f;       // rows beyond U hold nothing of this token
 
-            float a1[4];
+            float a1t = 0.f;                          // one scale per token: the same factor for every chunk
             if (GROUPED) {
                 if (P.gsh >= 1) {
                     mc[0] = mc[1] = fmaxf(mc[0], mc[1]);
@@ -339,7 +339,6 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvr_rq(const __grid_constant_
                 }
 #pragma unroll
                 for (int c = 0; c < 4; ++c) {
-                    a1[c] = (mc[c] > 0.f) ? __fdividef(P.c_half, mc[c]) : 0.f;
                     // one writer per group: its first chunk, in its first lane
                     const bool writer = (P.gsh <= 2) ? ((c & ((1 << P.gsh) - 1)) == 0)
                                                      : (c == 0 && (lane & ((1 << (P.gsh - 2)) - 1)) == 0);
@@ -356,15 +355,16 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvr_rq(const __grid_constant_
                 const float4* rp = reinterpret_cast<const float4*>(&S->red[tb][0]);
                 const float4 m0 = rp[0], m1 = rp[1];
                 const float M = fmaxf(fmaxf(fmaxf(m0.x, m0.y), fmaxf(m0.z, m0.w)), fmaxf(fmaxf(m1.x, m1.y), fmaxf(m1.z, m1.w)));
-                a1[0] = a1[1] = a1[2] = a1[3] = (M > 0.f) ? __fdividef(P.c_half, M) : 0.f;
+                a1t = (M > 0.f) ? __fdividef(P.c_half, M) : 0.f;
                 if (slab == 0 && lane == 0) P.scales[row] = P.c_scale * M;
             }
             if (lane_live) {
                 unsigned out[4 * BITS];
-                quantize_pack32<BITS>(r0, a1[0], out);
-                quantize_pack32<BITS>(r1, a1[1], out + BITS);
-                quantize_pack32<BITS>(r2, a1[2], out + 2 * BITS);
-                quantize_pack32<BITS>(r3, a1[3], out + 3 * BITS);
+                // per-group factors are formed chunk by chunk: four more live values would not fit the register budget
+                quantize_pack32<BITS>(r0, GROUPED ? ((mc[0] > 0.f) ? __fdividef(P.c_half, mc[0]) : 0.f) : a1t, out);
+                quantize_pack32<BITS>(r1, GROUPED ? ((mc[1] > 0.f) ? __fdividef(P.c_half, mc[1]) : 0.f) : a1t, out + BITS);
+                quantize_pack32<BITS>(r2, GROUPED ? ((mc[2] > 0.f) ? __fdividef(P.c_half, mc[2]) : 0.f) : a1t, out + 2 * BITS);
+                quantize_pack32<BITS>(r3, GROUPED ? ((mc[3] > 0.f) ? __fdividef(P.c_half, mc[3]) : 0.f) : a1t, out + 3 * BITS);
                 store_codes<BITS>(P.codes + row * P.code_row_bytes + (size_t)up * (NCOLS * BITS / 8), out);
                 if (P.y_opt) {
                     float* yo = P.y_opt + row * (long long)P.d_pad + (size_t)up * NCOLS;
