@@ -17,8 +17,9 @@
 //     per token the warps of the token meet once at an mbarrier.
 //   * Eight epilogue warps, two per lane quadrant: of each pair one takes the first block of even tokens and the
 //     second block's slab of odd tokens, the other the reverse, so every warp walks the tokens in order.
-//   * The token row reaches shared memory in slices of 32 u-rows (8 KB, two k-steps of the contraction) through a
-//     ring of up to 24 slices: a slice goes back to the TMA producer as soon as both blocks have contracted it.
+//   * The token row reaches shared memory in slices of 32 u-rows (8 KB, two k-steps of the contraction); a stage of
+//     the ring holds a token's slices (fewer where three such stages do not fit) behind one barrier and goes back to the
+//     TMA producer as soon as both blocks have contracted it.
 // Every wait is a bounded mbarrier wait; an expired wait records a code in the plan's status word and every role
 // leaves through the abort flag.
 #include <math.h>
@@ -66,7 +67,8 @@ struct UvrParams {
     int nb2;                      // slabs of the second block (0 .. 4)
     int ksteps;                   // ceil(U / 16): the contraction is padded with zero columns of A and zero rows of X
     int nslices;                  // ceil(U / 32)
-    int n_ring;                   // slices of shared memory in use
+    int g;                        // slices per shared-memory stage
+    int n_ring;                   // shared-memory stages in use
     int a_bytes;                  // image of A
     int atom_stride;              // bytes between the 64-column K atoms of the image: U (rounded up to 8) * 128
     int code_row_bytes;
@@ -206,20 +208,25 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvr_rq(const __grid_constant_
             unsigned ph = 0;
             bool ok = true;
             for (int tk = blockIdx.x; ok && tk < n_tok; tk += gridDim.x)
-                for (int j = 0; j < P.nslices; ++j) {
+                for (int j0 = 0; j0 < P.nslices; j0 += P.g) {
                     if (!mbar_wait_inline(&S->abort_flag, &S->empty[s], ph ^ 1, P.status, 1)) { ok = false; break; }
-                    mbar_arrive_expect_tx(&S->full[s], SLICE_BYTES);
-                    unsigned char* dst = ring + (size_t)s * SLICE_BYTES;
-                    tma_load_4d(dst, &tmap, &S->full[s], 0, 0, j * SLICE_ROWS, tk);
-                    tma_load_4d(dst + SLICE_BYTES / 2, &tmap, &S->full[s], 0, 1, j * SLICE_ROWS, tk);
+                    const int cnt = P.nslices - j0 < P.g ? P.nslices - j0 : P.g;
+                    mbar_arrive_expect_tx(&S->full[s], (unsigned)(cnt * SLICE_BYTES));
+                    // a stage: the first halves (64 coordinates) of its slices one after the other, then the second halves
+                    unsigned char* dst = ring + (size_t)s * P.g * SLICE_BYTES;
+                    for (int j = 0; j < cnt; ++j) {
+                        tma_load_4d(dst + j * (SLICE_BYTES / 2), &tmap, &S->full[s], 0, 0, (j0 + j) * SLICE_ROWS, tk);
+                        tma_load_4d(dst + (P.g + j) * (SLICE_BYTES / 2), &tmap, &S->full[s], 0, 1, (j0 + j) * SLICE_ROWS, tk);
+                    }
                     if (++s == P.n_ring) { s = 0; ph ^= 1; }
                 }
         }
       } else if (warp <= 2) {
         // ------------------------------ MMA issuers ------------------------------
-        // Two issuing threads on two schedulers: an issuing thread competes for issue slots with three epilogue warps
-        // whose butterflies rarely stall, and one thread alone does not keep the tensor pipe fed.  U > 128: thread 0
-        // contracts the first block of every token, thread 1 the second (a slice returns to the producer after both
+        // Two issuing threads on two schedulers: what costs an issuing thread time is not the MMAs (64 cycles each on the
+        // tensor pipe) but what stands between them (the poll of a stage's barrier, the commit that returns it, every
+        // instruction of its own loop), and one thread alone does not keep the epilogue fed.  U > 128: thread 0
+        // contracts the first block of every token, thread 1 the second (a stage returns to the producer after both
         // commits).  U <= 128: the threads take alternate tokens.
         if (lane == 0) {
             const int issuer = warp - 1;
@@ -227,42 +234,53 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvr_rq(const __grid_constant_
             // A: K-major, one 128-byte line per row and 64-column atom, 32 bytes per k-step.  B: N-major, atoms of 8
             // u-rows x 64 coordinates (1024 bytes), the other 64 coordinates of the slice 4 KB away.  Only the address
             // fields (bytes >> 4, low words) of the descriptors change between MMAs.
-            const unsigned long long ad0 = smem_desc(smem_u32(a_smem), 16, 1024, 2);
-            const unsigned long long bd0 = smem_desc(smem_u32(ring), SLICE_BYTES / 2, 1024, 2);
-            const unsigned ad_lo0 = (unsigned)ad0, ad_hi = (unsigned)(ad0 >> 32);
-            const unsigned bd_lo0 = (unsigned)bd0, bd_hi = (unsigned)(bd0 >> 32);
-            const unsigned atom_jump = (unsigned)(P.atom_stride - 96) >> 4;     // from the last k-step of an atom to the next atom
-            const bool odd = (P.ksteps & 1) != 0;                               // the last slice holds one k-step
+            // high words (1024 bytes between 8-row groups, descriptor version, 128-byte swizzle) are one constant;
+            // B's leading offset is the distance between the two 64-coordinate halves of a stage
+            constexpr unsigned D_HI = (1024u >> 4) | (1u << 14) | (2u << 29);
+            const unsigned ad_lo0 = ((smem_u32(a_smem) >> 4) & 0x3fffu) | ((16u >> 4) << 16);
+            const unsigned bd_lo0 = ((smem_u32(ring) >> 4) & 0x3fffu) | ((unsigned)(P.g * (SLICE_BYTES / 2) >> 4) << 16);
+            // few live values: the loop must fit the 32 registers this warpgroup keeps; a spill in it costs the tensor
+            // pipe more than any arithmetic
             bool ok = mbar_wait_inline(&S->abort_flag, &S->abar, 0, P.status, 6);
-            int s = 0, it = 0, ts = 0, tf = 0;
-            unsigned ph = 0, tph = 0;                 // tph: parity of the use count of stage ts
-            for (int tk = blockIdx.x; ok && tk < n_tok; tk += gridDim.x, ++it, ts = (ts + 1 == tstages ? 0 : ts + 1),
-                                                         tph ^= (ts == 0 ? 1u : 0u), tf = (tf + 1 == nfull ? 0 : tf + 1)) {
-                if (!TWO && (it & 1) != issuer) {     // the other thread's token: step over its slices
-                    for (int j = 0; j < P.nslices; ++j)
+            const int n_mine = ((int)blockIdx.x < n_tok) ? (n_tok - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
+            const int chunks = (P.nslices + P.g - 1) / P.g;
+            int s = 0;
+            unsigned ph = 0;
+            for (int it = 0; ok && it < n_mine; ++it) {
+                if (!TWO && (it & 1) != issuer) {     // the other thread's token: step over its stages
+                    for (int c = 0; c < chunks; ++c)
                         if (++s == P.n_ring) { s = 0; ph ^= 1; }
                     continue;
                 }
-                if (!mbar_wait_inline(&S->abort_flag, &S->tempty[ts], tph ^ 1, P.status, 3)) break;
+                const int ts = it & (tstages - 1);
+                if (!mbar_wait_inline(&S->abort_flag, &S->tempty[ts], ((it / tstages) & 1) ^ 1, P.status, 3)) break;
                 tc_fence_after();
                 const unsigned d = tmem_base + ts * tstride + (TWO ? issuer * NCOLS : 0);
                 // the second block's rows come from a window of the image that starts 128 - 32 rot rows into it
                 unsigned a_lo = ad_lo0 + ((TWO && issuer) ? (unsigned)((128 - 32 * rot_of(it, P.nb2)) * 128) >> 4 : 0u);
-                for (int j = 0; j < P.nslices; ++j) {
+                int kk = 0;                           // k-step of the token
+                for (int c = 0; c < chunks; ++c) {
                     if (!mbar_wait_inline(&S->abort_flag, &S->full[s], ph, P.status, 2)) { ok = false; break; }
                     tc_fence_after();
-                    const unsigned b_lo = bd_lo0 + (unsigned)s * (SLICE_BYTES >> 4);
-                    if (j == 0) umma_f16_words<false>(d, a_lo, ad_hi, b_lo, bd_hi, IDESC);
-                    else umma_f16_words<true>(d, a_lo, ad_hi, b_lo, bd_hi, IDESC);
-                    a_lo += 2u;
-                    if (!(odd && j == P.nslices - 1)) {
-                        umma_f16_words<true>(d, a_lo, ad_hi, b_lo + (16 * 128 >> 4), bd_hi, IDESC);
-                        a_lo += (j & 1) ? atom_jump : 2u;
+                    unsigned b_lo = bd_lo0 + (unsigned)(s * P.g) * (SLICE_BYTES >> 4);
+                    const int kend = kk + 2 * P.g < P.ksteps ? kk + 2 * P.g : P.ksteps;
+                    if (kk == 0) {
+                        umma_f16_words<false>(d, a_lo, D_HI, b_lo, D_HI, IDESC);
+                        a_lo += 2u;
+                        b_lo += 16 * 128 >> 4;
+                        kk = 1;
+                    }
+#pragma unroll 1
+                    for (; kk < kend; ++kk) {
+                        umma_f16_words<true>(d, a_lo, D_HI, b_lo, D_HI, IDESC);
+                        // every fourth k-step ends a 64-column atom of the image: on to the next atom
+                        a_lo += ((kk & 3) == 3) ? (unsigned)(P.atom_stride - 96) >> 4 : 2u;
+                        b_lo += 16 * 128 >> 4;
                     }
                     umma_commit(&S->empty[s]);
                     if (++s == P.n_ring) { s = 0; ph ^= 1; }
                 }
-                if (ok) umma_commit((TWO && issuer) ? &S->tfull2[it & 3] : &S->tfull[tf]);
+                if (ok) umma_commit((TWO && issuer) ? &S->tfull2[it & 3] : &S->tfull[TWO ? (it & 1) : it % 12]);
             }
         }
       }
@@ -490,8 +508,14 @@ int gbs_tc_uvr_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
     P.nslices = (U + 31) / 32;
     P.a_bytes = gbs_tc_uvr_image_bytes(p);
     P.atom_stride = image_rows(U) * 128;
-    int ring = (p->smem_optin - 1024 - CTL_BYTES - P.a_bytes) / SLICE_BYTES;
-    P.n_ring = ring < MAX_SLICES ? ring : MAX_SLICES;
+    const int ring = (p->smem_optin - 1024 - CTL_BYTES - P.a_bytes) / SLICE_BYTES;     // slices that fit
+    // A stage holds g slices behind one barrier: an issuing thread spends several hundred cycles on every poll and
+    // every commit, far more than on the MMAs of a slice.  As many slices as leave three stages, at most a token's.
+    P.g = ring / 3;
+    if (P.g < 1) P.g = 1;
+    if (P.g > P.nslices) P.g = P.nslices;
+    if (P.g > ring / 2) P.g = ring / 2;
+    P.n_ring = ring / P.g < MAX_SLICES ? ring / P.g : MAX_SLICES;
     P.code_row_bytes = p->d_pad * p->bits / 8;
     P.d_pad = p->d_pad;
     P.gsh = p->group ? log2_chunks(p->group) : 0;
@@ -504,7 +528,7 @@ int gbs_tc_uvr_rotate_quantize(const gbs_plan* p, const void* x, int64_t n_rows,
     P.scales = scales;
     P.y_opt = y_opt;
     P.status = p->d_status;
-    const int smem = 1024 + CTL_BYTES + P.a_bytes + P.n_ring * SLICE_BYTES;
+    const int smem = 1024 + CTL_BYTES + P.a_bytes + P.n_ring * P.g * SLICE_BYTES;
     const int grid = (int)(n_rows < p->sm_count ? n_rows : p->sm_count);
     const bool pdl = p->pdl != 0;
     cudaError_t e;
