@@ -15,8 +15,10 @@
 //     rounds, clips and packs (Sections 2.1, 3.1) 48 or 64 bytes of codes.  Scales per group of up to 128 coordinates
 //     never leave the thread, larger groups (up to 4096) are folded over neighbouring lanes by shuffles; for one scale
 //     per token the warps of the token meet once at an mbarrier.
-//   * Eight epilogue warps, two per lane quadrant: of each pair one takes the first block of even tokens and the
-//     second block's slab of odd tokens, the other the reverse, so every warp walks the tokens in order.
+//   * Twelve epilogue warps, three per lane quadrant (U > 128: two for the first block of even / odd tokens, one for
+//     the quadrant's slabs of the second block; U <= 128: every third token each), so every warp walks its tokens in
+//     order and no warp holds two consecutive tokens.  128 live values need about 160 registers: the first warpgroup
+//     (TMA producer, two MMA issuing threads) gives registers up, the three epilogue warpgroups take them.
 //   * The token row reaches shared memory in slices of 32 u-rows (8 KB, two k-steps of the contraction); a stage of
 //     the ring holds a token's slices (fewer where three such stages do not fit) behind one barrier and goes back to the
 //     TMA producer as soon as both blocks have contracted it.
