@@ -347,6 +347,28 @@ def test_wide_family_many_tokens_per_block(d, d_pad, m, bits, group):
         assert plan.device_status() == 0
 
 
+@pytest.mark.parametrize("d,d_pad,m,bits,group,rows", [
+    (16384, 16384, 1, 3, 0, 151), (18944, 20480, 20, 4, 0, 300), (12288, 12288, 12, 4, 128, 75), (28672, 28672, 28, 3, 512, 40),
+])
+def test_three_sweep_kernel_where_the_register_kernel_would_run(d, d_pad, m, bits, group, rows, monkeypatch):
+    """GBS_NO_UVR=1 at plan creation keeps a wide plan on the three-sweep kernel (it still serves clip scoring, groups
+    above 4096 and widths the register-resident kernel does not take): its rotate-quantize stays covered."""
+    monkeypatch.setenv("GBS_NO_UVR", "1")
+    rng = np.random.Generator(np.random.PCG64(d + 7 * m + bits + rows))
+    xs = rng.standard_t(3, size=(rows, d))
+    xs[:, rng.integers(0, d, 3)] *= 40
+    x = torch.from_numpy(xs.astype(np.float32)).to(torch.bfloat16)
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(x), d, d_pad, m, bits, group, 0.9)
+    with Plan(d, d_pad, m, bits, group, 0.9) as plan:
+        assert plan.info.variant == 3
+        codes, scales, y = _run_rq(plan, x.to(DEV), rows)
+        assert plan.device_status() == 0
+        print(compare_rotate_quantize(x, ref, codes, scales, y, bits, group, d_pad))
+    monkeypatch.delenv("GBS_NO_UVR")
+    with Plan(d, d_pad, m, bits, group, 0.9) as plan:
+        assert plan.info.variant == 5
+
+
 ROW_SHAPES = [
     # d, bits, group, alpha, rows, stride
     (128, 3, 0, 1.0, 1, 128),
