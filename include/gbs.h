@@ -83,8 +83,8 @@ typedef struct gbs_plan_info {
                                       4096 < d' = 32 * G * U <= 32768 (G in {2, 4, 8}, U as above, per-token
                                       scales, d a multiple of 32 * G), 4 = dense tensor-core contraction with the full
                                       Paley matrix (d' = m), 5 = as 3 where also d' = 128 * U with 80 <= U <= 256,
-                                      U % 16 == 0, d % 128 == 0 and group <= 4096: rotate-quantize keeps the rest of
-                                      the transform in registers (GBS_NO_UVR=1 forces 3) (set GBS_FORCE_GENERIC=1 in the
+                                      d % 128 == 0 and group <= 4096: rotate-quantize keeps the rest of the transform
+                                      in registers, clip scoring runs as in 3 (GBS_NO_UVR=1 forces 3) (set GBS_FORCE_GENERIC=1 in the
                                       environment before gbs_plan_create to force 0; GBS_NO_PDL=1 launches it
                                       without programmatic stream serialization) */
 } gbs_plan_info_t;
