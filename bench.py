@@ -691,6 +691,30 @@ def extras(device, stream, args, peak, sampler=None):
                                                                      "note": "library GEMM, context only"}
     del xq, wq
     torch.cuda.empty_cache()
+    # the full Paley order (width 1536 -> d' = m = 1544): the rotation is a dense contraction with H_m, forward in
+    # two sweeps (max|.|, then quantize: 2 x 2 m^2 flops per token), inverse in one (2 m d flops per token)
+    pd = Plan(1536, 1544, 1544, 3, 0, 0.9)
+    for n_d in (4096, 65536):
+        xd = (torch.randn((n_d, 1536), generator=torch.Generator().manual_seed(11)) * 0.5).to(torch.bfloat16).to(device)
+        od = pd.alloc_outputs(n_d, device)
+        ms = time_loop(lambda i: pd.rotate_quantize(xd, out=od, stream=stream), 4)
+        tf = 2.0 * 2.0 * n_d * 1544.0 * 1544.0 / ms / 1e9
+        out["paley1544_b3_%d_rows" % n_d] = {
+            "us_per_launch": ms * 1e3, "mrows_per_s": n_d / ms / 1e3, "kernel_family": pd.info.variant,
+            "roofline": {"bound": "tensor", "unit": "TFLOP/s", "achieved": tf, "peak": bf16_tf, "frac": tf / bf16_tf,
+                         "note": "two dense sweeps with H_1544 per token; peak = the %s bf16 figure" % bf16_kind}}
+        if True:
+            xh = torch.empty((n_d, 1536), dtype=torch.bfloat16, device=device)
+            ms = time_loop(lambda i: pd.dequantize(od[0], od[1], inverse=True, out=xh, stream=stream), 4)
+            tf = 2.0 * n_d * 1544.0 * 1536.0 / ms / 1e9
+            out["paley1544_b3_inverse_dequantize_%d_rows" % n_d] = {
+                "us_per_launch": ms * 1e3,
+                "roofline": {"bound": "tensor", "unit": "TFLOP/s", "achieved": tf, "peak": bf16_tf, "frac": tf / bf16_tf,
+                             "note": "codes unpacked to bf16 in the CTA, one dense contraction with H_1544"}}
+            del xh
+        del xd, od
+    del pd
+    torch.cuda.empty_cache()
     # clip-ratio scoring at the calibration size: K = 32 candidates over one full layer of 128 sequences x 2048
     # tokens x d = 4096 per launch, for each of 32 layers (its own seeded tensor each: seed 5 + layer)
     wc = synth.WORKLOADS["calib4096"]

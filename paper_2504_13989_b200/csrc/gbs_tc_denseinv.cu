@@ -135,32 +135,54 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_dense_inv(const __grid_consta
         }
     } else if (warp < 2 + UNPACK_WARPS) {
         // ------------------------------ unpack: one thread = one token row of the A tile ------------------------------
+        // The 64 codes of a stage are 8 * BITS bytes of the row, at any byte offset (rows of m * BITS / 8 bytes start
+        // wherever they start): the thread fetches the aligned words that cover them one stage ahead (the loads of the
+        // next stage are in flight while it waits for its buffer) and shifts them into place.
+        constexpr int NW = 2 * BITS + 1;          // aligned words that cover 8 * BITS bytes at any offset
         const int r = (warp - 2) * 32 + lane;
         int c = 0;
         bool ok = true;
+        unsigned raw[NW];
+        auto fetch = [&](const unsigned char* crow, bool live, int kc) {
+            const int k0 = kc * KC;
+            const unsigned char* src = crow + (long long)k0 * BITS / 8;
+            const unsigned* w0 = reinterpret_cast<const unsigned*>(reinterpret_cast<uintptr_t>(src) & ~(uintptr_t)3);
+            const unsigned char* end = crow + P.code_row_bytes;
+#pragma unroll
+            for (int i = 0; i < NW; ++i)          // words wholly beyond the row are not read (the last row ends the buffer)
+                raw[i] = (live && reinterpret_cast<const unsigned char*>(w0 + i) < end) ? __ldg(w0 + i) : 0u;
+        };
         for (int i = 0; ok && i < n_mine; ++i) {
             const long long row = ((long long)blockIdx.x + (long long)i * gridDim.x) * TM + r;
             const bool live = row < P.n_rows;
-            const unsigned char* crow = P.codes + row * P.code_row_bytes;
+            const unsigned char* crow = P.codes + (live ? row : 0) * P.code_row_bytes;
+            const unsigned sh = (unsigned)((reinterpret_cast<uintptr_t>(crow) & 3u) * 8u);   // kc * KC * BITS / 8 is a multiple of 4
+            fetch(crow, live, 0);
             for (int nb = 0; ok && nb < P.nblk; ++nb)
                 for (int kc = 0; kc < P.kchunks; ++kc, ++c) {
+                    unsigned f[2 * BITS];         // the stage's 8 * BITS bytes, in place
+#pragma unroll
+                    for (int w = 0; w < 2 * BITS; ++w) f[w] = __funnelshift_r(raw[w], raw[w + 1], sh);
+                    {
+                        const int kn = kc + 1 < P.kchunks ? kc + 1 : 0;      // next stage (of this block or the next)
+                        if (kc + 1 < P.kchunks || nb + 1 < P.nblk) fetch(crow, live, kn);
+                    }
                     const int s = c % STAGES;
                     ok = mbar_wait(&S->abort_flag, &S->empty[s], ((c / STAGES) & 1) ^ 1, P.status, 1);
                     if (!__all_sync(0xffffffffu, ok)) { ok = false; break; }
                     const unsigned base = smem_u32(S->a[s]) + (unsigned)r * 128u;
 #pragma unroll
                     for (int ch = 0; ch < 8; ++ch) {            // eight 16-byte chunks of eight codes each
-                        const int k0 = kc * KC + ch * 8;
                         unsigned w[4] = {0u, 0u, 0u, 0u};
-                        if (live && k0 < P.m) {                 // m is a multiple of 8: a chunk is whole or beyond the end
-                            const unsigned char* src = crow + (long long)k0 * BITS / 8;
-                            unsigned f = 0;
-#pragma unroll
-                            for (int bb = 0; bb < BITS; ++bb) f |= (unsigned)__ldg(src + bb) << (8 * bb);
+                        if (kc * KC + ch * 8 < P.m) {           // m is a multiple of 8: a chunk is whole or beyond the end
+                            // the chunk's 8 * BITS bits start at bit ch * 8 * BITS of f
+                            unsigned fld;
+                            if (BITS == 4) fld = f[ch];
+                            else fld = __funnelshift_r(f[(ch * 24) >> 5], f[((ch * 24) >> 5) + (((ch * 24) & 31) > 8 ? 1 : 0)], (ch * 24) & 31);   // 24 bits
 #pragma unroll
                             for (int e = 0; e < 8; e += 2) {
-                                const int q0 = ((int)(f << (32 - BITS * (e + 1)))) >> (32 - BITS);
-                                const int q1 = ((int)(f << (32 - BITS * (e + 2)))) >> (32 - BITS);
+                                const int q0 = ((int)(fld << (32 - BITS * (e + 1)))) >> (32 - BITS);
+                                const int q1 = ((int)(fld << (32 - BITS * (e + 2)))) >> (32 - BITS);
                                 w[e >> 1] = bf16_of_int(q0) | (bf16_of_int(q1) << 16);
                             }
                         }
@@ -191,7 +213,28 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_dense_inv(const __grid_consta
                     unsigned rr[32];
                     tmem_ld32_issue(lane_base + (unsigned)(buf * BN + c0), rr);
                     tmem_ld_wait(rr);
-                    if (live) {
+                    if (live && c0 + 32 <= width) {                 // rows of d elements, d a multiple of 8: 16-byte stores
+                        if (sizeof(OutT) == 4) {
+                            float4* o4 = reinterpret_cast<float4*>(reinterpret_cast<float*>(orow) + nb * BN + c0);
+#pragma unroll
+                            for (int e = 0; e < 8; ++e)
+                                o4[e] = make_float4(__uint_as_float(rr[4 * e]) * sc, __uint_as_float(rr[4 * e + 1]) * sc,
+                                                    __uint_as_float(rr[4 * e + 2]) * sc, __uint_as_float(rr[4 * e + 3]) * sc);
+                        } else {
+                            uint4* o4 = reinterpret_cast<uint4*>(reinterpret_cast<__nv_bfloat16*>(orow) + nb * BN + c0);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                unsigned w[4];
+#pragma unroll
+                                for (int h = 0; h < 4; ++h) {
+                                    const __nv_bfloat162 v2 = __floats2bfloat162_rn(__uint_as_float(rr[8 * e + 2 * h]) * sc,
+                                                                                    __uint_as_float(rr[8 * e + 2 * h + 1]) * sc);
+                                    w[h] = *reinterpret_cast<const unsigned*>(&v2);
+                                }
+                                o4[e] = make_uint4(w[0], w[1], w[2], w[3]);
+                            }
+                        }
+                    } else if (live) {
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
                             if (c0 + e < width) {
