@@ -222,6 +222,16 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uvr_rq(const __grid_constant_
                     }
                     if (++s == P.n_ring) { s = 0; ph ^= 1; }
                 }
+            if (!ok) {
+                // Leaving through the abort flag: the copies this thread started may still be on their way into this
+                // block's shared memory.  Give each armed stage a short, bounded time to complete before the block ends
+                // (walking back from the stage that would have been armed next; a stage never armed passes at once).
+                const unsigned long long t0 = global_ns();
+                for (int n = 0; n < P.n_ring; ++n) {
+                    if (--s < 0) { s = P.n_ring - 1; ph ^= 1; }
+                    while (!mbar_try_wait(&S->full[s], ph) && global_ns() - t0 < 2000000ull) {}
+                }
+            }
         }
       } else if (warp <= 2) {
         // ------------------------------ MMA issuers ------------------------------
