@@ -72,6 +72,16 @@ __device__ __forceinline__ bool mbar_wait(volatile int* abort_flag, void* bar, u
     return mbar_wait_slow(abort_flag, bar, parity, status, code, watch_abort);
 }
 
+// A producer that leaves its loop through the abort flag has copies on their way into the block's shared memory.  It
+// gives the stages it armed (uses it_next - 1, it_next - 2, .. of a ring of n_stages `full` barriers; use i fills stage
+// i % n_stages in phase (i / n_stages) & 1) a bounded time, two milliseconds in all, to complete before the block ends.
+__device__ __noinline__ void drain_copies(unsigned long long* full, int n_stages, int it_next)
+{
+    const unsigned long long t0 = global_ns();
+    for (int i = it_next - 1; i >= 0 && i >= it_next - n_stages; --i)
+        while (!mbar_try_wait(&full[i % n_stages], (unsigned)(i / n_stages) & 1u) && global_ns() - t0 < 2000000ull) {}
+}
+
 __device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, void* bar, int c0, int c1, int c2)
 {
     asm volatile(

@@ -129,6 +129,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_dense_rq(const __grid_constan
                     }
                 }
             }
+            if (!ok) drain_copies(S->full, STAGES, c);
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------

@@ -101,6 +101,8 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_dense_inv(const __grid_consta
                         for (int j = 0; j < BN / 64; ++j)        // 64 output coordinates x 64 rotated coordinates each
                             tma_load_2d(S->b[s] + j * (KC * 128), &hmap, &S->full[s], nb * BN + j * 64, kc * KC);
                     }
+            // (a stage's barrier also counts the unpacking warps, which may have left: the time limit ends the wait)
+            if (!ok) drain_copies(S->full, STAGES, c);
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------

@@ -126,6 +126,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_row_rq(const __grid_constant_
                 tma_load_2d(S->x[s], &tmap, &S->full[s], 0, t * TILE);
                 tma_load_2d(S->x[s] + TILE_BYTES / 2, &tmap, &S->full[s], 64, t * TILE);
             }
+            if (S->abort_flag) drain_copies(S->full, STAGES, it);
         }
     } else if (warp == 1) {
         // ------------------------------ MMA issuer ------------------------------

@@ -195,6 +195,7 @@ __global__ void __launch_bounds__(THREADS, 1) k_tc_uv_rq(const __grid_constant__
                 mbar_arrive_expect_tx(&S->full[s], stage_bytes);
                 tma_load_3d(S->b[s], &tmap, &S->full[s], 0, 0, g * TOK);
             }
+            if (S->abort_flag) drain_copies(S->full, STAGES, it);
         }
     } else if (warp == 1 || warp >= 2 + EPI_WARPS) {
         // ------------------------------ MMA issuers ------------------------------

@@ -228,6 +228,7 @@ __global__ void __launch_bounds__(threads_for(GLOG), 1) k_tc_uvm_rq(const __grid
                     tma_load_4d(S->b + (size_t)s * P.stage_bytes + (size_t)c * (P.stage_bytes >> GLOG), &tmap,
                                 &S->full[s], 0, c, 0, tk);
             }
+            if (S->abort_flag) drain_copies(S->full, nst, it);
         }
     } else if (warp == 1 || warp >= 2 + EPI_WARPS) {
         constexpr int NISS = issuers_for(GLOG);
