@@ -119,3 +119,35 @@ def test_rotated_domain_dequantize_at_launch_sizes_of_both_forms(name, rows, bit
         got = out[idx].cpu().double().numpy()
         tol = 2e-7 if dtype == torch.float32 else 2.0 ** -8
         np.testing.assert_allclose(got, want, rtol=tol, atol=1e-30 if not asym else 1e-6 * np.abs(want).max())
+
+
+@pytest.mark.parametrize("bits,group", [(3, 0), (4, 128)])
+def test_mlp_width_long_batch_sampled_rows(bits, group):
+    """Sixteen batches' worth of MLP rows (65 536 x 18944 -> 20480) in one launch: every block of the wide kernel walks
+    several hundred tokens, so every ring, stage and barrier index wraps many times; the oracle checks the first and last
+    rows and a random sample, and every code of every row must lie in [-D, D]."""
+    w = synth.WORKLOADS["mlp18944"]
+    rows = 65536
+    x = synth.make_device("mlp18944", rows, device=DEV)
+    pick = np.unique(np.concatenate([np.arange(3), np.arange(rows - 3, rows),
+                                     np.random.Generator(np.random.PCG64(bits + group)).integers(0, rows, 26)]))
+    xs = x[torch.from_numpy(pick).to(DEV)].cpu()
+    ref = oracle.rotate_quantize_rows(synth.to_oracle_array(xs), w.d, w.d_pad, w.m, bits, group, w.alpha)
+    with Plan(w.d, w.d_pad, w.m, bits, group, w.alpha) as plan:
+        codes, scales, _ = plan.rotate_quantize(x)
+        torch.cuda.synchronize()
+        assert plan.device_status() == 0
+        idx = torch.from_numpy(pick).to(DEV)
+        print(compare_rotate_quantize(xs, ref, codes[idx], scales[idx], None, bits, group, w.d_pad, alpha=w.alpha))
+        # the code range over the whole tensor, on the device: no field of any row outside [-D, D]
+        D = (1 << (bits - 1)) - 1
+        flat = codes.view(-1)
+        if bits == 4:
+            lo, hi = (flat & 15).to(torch.int16), (flat >> 4).to(torch.int16)
+            for f in (lo, hi):
+                q = torch.where(f >= 8, f - 16, f)
+                assert int(q.min()) >= -D and int(q.max()) <= D
+        else:
+            sample = codes[:: 97].cpu().numpy()
+            q = unpack_codes(sample.reshape(sample.shape[0], -1), w.d_pad, bits)
+            assert q.min() >= -D and q.max() <= D
