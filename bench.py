@@ -645,6 +645,10 @@ def extras(device, stream, args, peak, sampler=None):
         xb = synth.make_host(name).repeat(reps, 1)
         out["%s_b3_65536rows" % name] = rq_leg(name, 3, xb=xb)
         del xb
+    # the wide kernel away from the launch boundaries: four MLP batches tiled into one launch
+    xb = synth.make_host("mlp18944").repeat(4, 1)
+    out["mlp18944_b4_16384rows"] = rq_leg("mlp18944", 4, xb=xb)
+    del xb
     # dequantize on the headline workload, with the plain fill of the same output bytes beside it
     w = synth.WORKLOADS["llama4096"]
     x = synth.make_host("llama4096").to(device)
